@@ -1,0 +1,161 @@
+/*
+ * aqt.h -- C ABI of the quantized linear layer (native integer quantization, arXiv 2203.15952).
+ *
+ * The layer: dynamic abs-max symmetric quantization of activations to int8 / int4 codes plus
+ * scales (Fig. 2, Section 2.2), pre-quantized per-output-channel int4 / int8 weights, an integer
+ * matmul with int32 accumulation (Section 1: native integer operations), and de-quantization by
+ * multiplying with the scales (Section 2.2) fused with bias, activation and residual.
+ *
+ * Conventions
+ *  - Every function returns an int status: AQT_OK or a negative AQT_ERR_* code.  Nothing throws.
+ *  - Unless a parameter says "host", every pointer is a DEVICE pointer owned by the caller.  The
+ *    library allocates no device memory; scratch space is passed in as `workspace`.
+ *  - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the legacy default
+ *    stream) of the current device and is not synchronised.  Argument errors are reported
+ *    synchronously by the return value and nothing is enqueued; device-side failures (a bounded
+ *    wait that ran out) are recorded in a device status word read by aqt_device_status().
+ *  - Outputs must not alias inputs.  Inputs must be finite (NaN / Inf: codes unspecified).
+ *  - Matrices are row-major.  x is [M, K]; weights are handed over as W^T = [N, K] with K
+ *    contiguous (row n = output channel n), so y = x . W with W = [K, N].
+ *  - 4-bit codes are two's-complement nibbles, two per byte along K: even k in the low nibble,
+ *    odd k in the high nibble.  The paper states only the resulting model sizes (Tables 1, 2);
+ *    this layout is the library's.
+ *  - Built for sm_100a only.  A call on another device returns AQT_ERR_UNSUPPORTED.
+ */
+#ifndef AQT_H_
+#define AQT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AQT_VERSION 100
+
+/* status codes */
+#define AQT_OK 0
+#define AQT_ERR_BADARG (-1)      /* null pointer, negative size, unknown enum value, odd K for int4 */
+#define AQT_ERR_ALIGN (-2)       /* a base pointer or row pitch violates the stated alignment       */
+#define AQT_ERR_UNSUPPORTED (-3) /* device is not sm_100, or a size is beyond the stated limits      */
+#define AQT_ERR_WORKSPACE (-4)   /* workspace missing or smaller than aqt_workspace_bytes()          */
+#define AQT_ERR_CUDA (-5)        /* a CUDA runtime / driver call failed                             */
+#define AQT_ERR_TIMEOUT (-6)     /* a bounded device-side wait ran out (reported by aqt_device_status) */
+
+/* which axis aqt_quantize reduces over (Fig. 2: reduce_max(abs(input), axis, keepdims=True)) */
+#define AQT_AXIS_ROW 0    /* reduce over columns: one scale per row       -> scale_out[rows] */
+#define AQT_AXIS_COL 1    /* reduce over rows: one scale per column       -> scale_out[cols] */
+#define AQT_AXIS_TENSOR 2 /* reduce over all elements: one scale          -> scale_out[1]    */
+
+/* rounding of scaled values to codes */
+#define AQT_ROUND_HALF_UP_FLOOR 0 /* floor(v + 0.5), the sum rounded in binary32 (Fig. 2)  */
+#define AQT_ROUND_NEAREST_EVEN 1  /* IEEE 754 round-to-nearest, ties to even               */
+
+/* granularity of the activation scale handed to the matmul */
+#define AQT_SCALE_ROW 0    /* s_x[M], one per row (reduced over K) */
+#define AQT_SCALE_TENSOR 1 /* s_x[1]                               */
+
+/* epilogue activation (not part of the paper; Conformer module definitions) */
+#define AQT_ACT_NONE 0
+#define AQT_ACT_SWISH 1     /* a = z * sigmoid(z)                                              */
+#define AQT_ACT_GLU 2       /* a[j] = z[j] * sigmoid(z[j + N/2]), j < N/2; output has N/2 columns */
+#define AQT_ACT_GLU_SWISH 3 /* Swish applied to the GLU output                                  */
+
+/* operations for aqt_workspace_bytes */
+#define AQT_OP_QMATMUL 1
+#define AQT_OP_LINEAR_FWD 2
+
+int aqt_version(void);
+const char* aqt_status_string(int status);
+
+/*
+ * aqt_quantize -- Fig. 2, quantize(input, axis), and its int4 form (Section 2.2: divide the
+ * abs-max by 7 instead of 127).
+ *   amax  = max |x| over the reduced axis;  scale = amax / qmax, qmax = 127 (bits 8) or 7 (bits 4)
+ *   v     = x / scale (0 where scale == 0, "divide_no_nan"), IEEE binary32 division
+ *   code  = floor(v + 0.5) or nearest-even(v) per `rounding`, clipped to +-qmax as a guard
+ * x         [rows, cols] fp32, row pitch ld elements (ld >= cols).
+ * q_out     pack == 0: int8 [rows, cols] dense (both bit widths use an int8 container, as the
+ *           figure's cast does).  pack == 1 (bits == 4 only, cols even): uint8 [rows, cols/2].
+ * scale_out fp32, extent given by `axis` (see AQT_AXIS_*).  For AQT_AXIS_COL and
+ *           AQT_AXIS_TENSOR it also serves as the abs-max accumulator while the call runs.
+ * Alignment: none required; 16-byte aligned x with ld % 4 == 0 and cols % 4 == 0 takes the
+ * vectorised path.  rows or cols == 0 is a no-op.
+ */
+int aqt_quantize(const float* x, int64_t rows, int64_t cols, int64_t ld, int bits, int axis, int rounding,
+                 int pack, void* q_out, float* scale_out, void* stream);
+
+/*
+ * aqt_pack_int4 / aqt_unpack_int4 -- 4-bit storage of codes (the paper reports only model sizes,
+ * Tables 1 and 2; nibble order as stated at the top).  q is int8 [rows, cols] with values in
+ * [-8, 7]; packed is uint8 [rows, cols/2]; cols must be even (AQT_ERR_BADARG otherwise).
+ * Unpacking sign-extends each nibble, which is exact.
+ */
+int aqt_pack_int4(const int8_t* q, int64_t rows, int64_t cols, uint8_t* packed, void* stream);
+int aqt_unpack_int4(const uint8_t* packed, int64_t rows, int64_t cols, int8_t* q, void* stream);
+
+/*
+ * aqt_qmatmul -- integer matmul on codes with the de-quantizing epilogue (Section 1: native
+ * integer matmul; Section 2.2: de-quantize by multiplying with the scales):
+ *   acc[m][n] = sum_k xq[m][k] * wq[n][k]                      exact, int32
+ *   z[m][n]   = fma(float(acc) * s_x[m or 0], s_w[n], bias[n]) binary32, bias = 0 if NULL
+ *   a         = act(z)                                         see AQT_ACT_*
+ *   y         = residual ? fma(residual_scale, a, residual) : a
+ * xq        bits_a == 8: int8 [M, K];  bits_a == 4: uint8 [M, K/2] packed.
+ * s_x       fp32 [M] (AQT_SCALE_ROW) or [1] (AQT_SCALE_TENSOR).
+ * wq        W^T codes: bits_w == 8: int8 [N, K];  bits_w == 4: uint8 [N, K/2] packed.
+ * s_w       fp32 [N];  bias fp32 [N] or NULL.
+ * residual  fp32 [M, N_out] with row pitch ldr, or NULL.  N_out = N, or N/2 for the GLU forms.
+ * y         fp32 [M, N_out], row pitch ldy.
+ * acc_debug NULL, or int32 [M, N] dense: receives the raw accumulators (for parity checks).
+ * workspace at least aqt_workspace_bytes(AQT_OP_QMATMUL, ...) bytes, 256-byte aligned; holds the
+ *           sign-extended copy of each 4-bit operand.  May be NULL when both operands are 8-bit.
+ * Limits: K % 32 == 0; N % 4 == 0 (N % 8 == 0 for GLU); ldy % 4 == 0, ldr % 4 == 0; xq, wq, y,
+ * residual, s_w, bias 16-byte aligned; M, N, K < 2^31 and M*N < 2^40.  K <= 133 000 keeps every
+ * accumulator inside int32.  M == 0 or N == 0 is a no-op.
+ */
+int aqt_qmatmul(const void* xq, const float* s_x, int s_x_kind, const void* wq, const float* s_w,
+                const float* bias, const float* residual, int64_t ldr, float residual_scale, int64_t M,
+                int64_t N, int64_t K, int bits_a, int bits_w, int act, float* y, int64_t ldy,
+                int32_t* acc_debug, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * aqt_linear_fwd -- the whole layer for fp32 activations: aqt_quantize(x, axis = K) with a
+ * per-row or per-tensor dynamic scale, then aqt_qmatmul (same arguments and limits).
+ * x         fp32 [M, K], row pitch ldx.
+ * workspace at least aqt_workspace_bytes(AQT_OP_LINEAR_FWD, ...) bytes, 256-byte aligned; holds
+ *           the activation codes and scales between the two steps and what aqt_qmatmul needs.
+ */
+int aqt_linear_fwd(const float* x, int64_t ldx, const void* wq, const float* s_w, const float* bias,
+                   const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K,
+                   int bits_a, int bits_w, int a_scale_kind, int rounding, int act, float* y, int64_t ldy,
+                   void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * aqt_linear_fwd_host -- aqt_linear_fwd for callers whose activations live in HOST memory.
+ * x_host    host fp32 [M, K] dense; y_host host fp32 [M, N_out] dense (pinned memory makes the
+ *           copies asynchronous).  Weights, scales, bias stay device pointers.
+ * workspace device memory, at least aqt_workspace_bytes(AQT_OP_LINEAR_FWD, ...) + 4*M*K + 4*M*N_out
+ *           bytes: the device copies of x and y are placed behind the layer's own scratch.
+ * The call enqueues the host-to-device copy, the layer, and the device-to-host copy on `stream`
+ * and returns without synchronising.
+ */
+int aqt_linear_fwd_host(const float* x_host, const void* wq, const float* s_w, const float* bias, int64_t M,
+                        int64_t N, int64_t K, int bits_a, int bits_w, int a_scale_kind, int rounding, int act,
+                        float* y_host, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Scratch bytes needed by `op` (AQT_OP_*) at these sizes; 0 if none.  Host-only, no CUDA call. */
+size_t aqt_workspace_bytes(int op, int64_t M, int64_t N, int64_t K, int bits_a, int bits_w);
+
+/*
+ * aqt_device_status -- synchronises `stream`, copies the device status word to *status_out (host
+ * pointer) and clears it.  AQT_OK, or AQT_ERR_TIMEOUT if a kernel gave up on a bounded wait since
+ * the last call (its output is then undefined).  Returns AQT_ERR_CUDA if the copy itself failed.
+ */
+int aqt_device_status(void* stream, int* status_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AQT_H_ */

@@ -1,0 +1,197 @@
+"""Thin Python binding of the C ABI in include/aqt.h: same names, argument marshalling only.
+
+Every step of the quantized linear layer runs in the CUDA library; torch is used here for device
+memory and the current stream.  There is no CPU fallback: if the shared library is missing the
+import of any entry point fails with an error that says how to build it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+from . import build as _build
+
+# enums of include/aqt.h
+AQT_OK = 0
+AXIS_ROW, AXIS_COL, AXIS_TENSOR = 0, 1, 2
+ROUND_HALF_UP_FLOOR, ROUND_NEAREST_EVEN = 0, 1
+SCALE_ROW, SCALE_TENSOR = 0, 1
+ACT_NONE, ACT_SWISH, ACT_GLU, ACT_GLU_SWISH = 0, 1, 2, 3
+OP_QMATMUL, OP_LINEAR_FWD = 1, 2
+
+EXPORTS = ("aqt_version", "aqt_status_string", "aqt_quantize", "aqt_pack_int4", "aqt_unpack_int4", "aqt_qmatmul",
+           "aqt_linear_fwd", "aqt_linear_fwd_host", "aqt_workspace_bytes", "aqt_device_status")
+
+
+class AqtError(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        self.status = status
+        super().__init__("%s failed: %d (%s)" % (fn, status, status_string(status)))
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libaqt.so (built in-tree by paper_2203_15952_b200.build).  Never falls back."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB_PATH
+        if not os.path.exists(path):
+            raise ImportError("CUDA library %s is missing; build it with `python -m paper_2203_15952_b200.build` "
+                              "(needs nvcc). There is no CPU fallback." % path)
+        L = ctypes.CDLL(path)
+        L.aqt_status_string.restype = ctypes.c_char_p
+        L.aqt_workspace_bytes.restype = ctypes.c_size_t
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().aqt_status_string(int(status)).decode()
+
+
+def _check(fn: str, status: int) -> None:
+    if status != AQT_OK:
+        raise AqtError(fn, status)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return ctypes.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _i64(v) -> ctypes.c_int64:
+    return ctypes.c_int64(int(v))
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _n_out(N: int, act: int) -> int:
+    return N // 2 if act in (ACT_GLU, ACT_GLU_SWISH) else N
+
+
+def aqt_version() -> int:
+    return int(lib().aqt_version())
+
+
+def aqt_workspace_bytes(op: int, M: int, N: int, K: int, bits_a: int, bits_w: int) -> int:
+    return int(lib().aqt_workspace_bytes(int(op), _i64(M), _i64(N), _i64(K), int(bits_a), int(bits_w)))
+
+
+def aqt_device_status(stream=None) -> int:
+    out = ctypes.c_int(0)
+    _check("aqt_device_status", lib().aqt_device_status(_stream(stream), ctypes.byref(out)))
+    return out.value
+
+
+def aqt_quantize(x: torch.Tensor, bits: int, axis: int = AXIS_ROW, rounding: int = ROUND_NEAREST_EVEN,
+                 pack: bool = False, q_out: Optional[torch.Tensor] = None, scale_out: Optional[torch.Tensor] = None,
+                 stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Fig. 2 quantize(input, axis) on the GPU.  x: fp32 [rows, cols] (last dim contiguous)."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.dim() == 2 and (x.shape[1] <= 1 or x.stride(1) == 1)
+    rows, cols = x.shape
+    ld = x.stride(0) if rows > 1 else max(cols, 1)
+    if q_out is None:
+        q_out = torch.empty((rows, cols // 2), dtype=torch.uint8, device=x.device) if pack else \
+            torch.empty((rows, cols), dtype=torch.int8, device=x.device)
+    n_scale = rows if axis == AXIS_ROW else (cols if axis == AXIS_COL else 1)
+    if scale_out is None:
+        scale_out = torch.empty(n_scale, dtype=torch.float32, device=x.device)
+    _check("aqt_quantize", lib().aqt_quantize(_ptr(x), _i64(rows), _i64(cols), _i64(ld), int(bits), int(axis), int(rounding),
+                                              int(bool(pack)), _ptr(q_out), _ptr(scale_out), _stream(stream)))
+    return q_out, scale_out
+
+
+def aqt_pack_int4(q: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    assert q.is_cuda and q.dtype == torch.int8 and q.dim() == 2 and q.is_contiguous()
+    rows, cols = q.shape
+    if out is None:
+        out = torch.empty((rows, cols // 2), dtype=torch.uint8, device=q.device)
+    _check("aqt_pack_int4", lib().aqt_pack_int4(_ptr(q), _i64(rows), _i64(cols), _ptr(out), _stream(stream)))
+    return out
+
+
+def aqt_unpack_int4(packed: torch.Tensor, cols: int, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    assert packed.is_cuda and packed.dtype == torch.uint8 and packed.dim() == 2 and packed.is_contiguous()
+    rows = packed.shape[0]
+    if out is None:
+        out = torch.empty((rows, cols), dtype=torch.int8, device=packed.device)
+    _check("aqt_unpack_int4", lib().aqt_unpack_int4(_ptr(packed), _i64(rows), _i64(cols), _ptr(out), _stream(stream)))
+    return out
+
+
+def _workspace(need: int, workspace: Optional[torch.Tensor], device) -> Optional[torch.Tensor]:
+    if need == 0:
+        return workspace
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=device)
+    return workspace
+
+
+def aqt_qmatmul(xq: torch.Tensor, s_x: torch.Tensor, wq: torch.Tensor, s_w: torch.Tensor,
+                bias: Optional[torch.Tensor] = None, residual: Optional[torch.Tensor] = None, residual_scale: float = 1.0,
+                *, K: int, bits_a: int = 8, bits_w: int = 8, act: int = ACT_NONE, s_x_kind: int = SCALE_ROW,
+                y: Optional[torch.Tensor] = None, acc_debug: Optional[torch.Tensor] = None,
+                workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Integer matmul on codes + de-quantizing epilogue.  xq [M, K] int8 or [M, K/2] uint8 packed;
+    wq [N, K] int8 or [N, K/2] uint8 packed.  Returns y fp32 [M, N_out]."""
+    M, N = xq.shape[0], wq.shape[0]
+    n_out = _n_out(N, act)
+    if y is None:
+        y = torch.empty((M, n_out), dtype=torch.float32, device=xq.device)
+    need = aqt_workspace_bytes(OP_QMATMUL, M, N, K, bits_a, bits_w)
+    workspace = _workspace(need, workspace, xq.device)
+    _check("aqt_qmatmul", lib().aqt_qmatmul(
+        _ptr(xq), _ptr(s_x), int(s_x_kind), _ptr(wq), _ptr(s_w), _ptr(bias), _ptr(residual),
+        _i64(residual.stride(0) if residual is not None else 0), ctypes.c_float(residual_scale), _i64(M), _i64(N), _i64(K),
+        int(bits_a), int(bits_w), int(act), _ptr(y), _i64(y.stride(0)), _ptr(acc_debug), _ptr(workspace),
+        ctypes.c_size_t(0 if workspace is None else workspace.numel()), _stream(stream)))
+    return y
+
+
+def aqt_linear_fwd(x: torch.Tensor, wq: torch.Tensor, s_w: torch.Tensor, bias: Optional[torch.Tensor] = None,
+                   residual: Optional[torch.Tensor] = None, residual_scale: float = 1.0, *, bits_a: int = 8,
+                   bits_w: int = 8, a_scale_kind: int = SCALE_ROW, rounding: int = ROUND_NEAREST_EVEN,
+                   act: int = ACT_NONE, y: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                   stream=None) -> torch.Tensor:
+    """The whole layer: dynamic activation quantization, integer matmul, epilogue.  x fp32 [M, K]."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.dim() == 2 and x.stride(1) == 1
+    M, K = x.shape
+    N = wq.shape[0]
+    n_out = _n_out(N, act)
+    if y is None:
+        y = torch.empty((M, n_out), dtype=torch.float32, device=x.device)
+    need = aqt_workspace_bytes(OP_LINEAR_FWD, M, N, K, bits_a, bits_w)
+    workspace = _workspace(need, workspace, x.device)
+    _check("aqt_linear_fwd", lib().aqt_linear_fwd(
+        _ptr(x), _i64(x.stride(0)), _ptr(wq), _ptr(s_w), _ptr(bias), _ptr(residual),
+        _i64(residual.stride(0) if residual is not None else 0), ctypes.c_float(residual_scale), _i64(M), _i64(N), _i64(K),
+        int(bits_a), int(bits_w), int(a_scale_kind), int(rounding), int(act), _ptr(y), _i64(y.stride(0)), _ptr(workspace),
+        ctypes.c_size_t(workspace.numel()), _stream(stream)))
+    return y
+
+
+def linear_fwd_host_workspace_bytes(M: int, N: int, K: int, bits_a: int, bits_w: int, act: int) -> int:
+    r256 = lambda v: (v + 255) // 256 * 256
+    return r256(aqt_workspace_bytes(OP_LINEAR_FWD, M, N, K, bits_a, bits_w)) + r256(4 * M * K) + r256(4 * M * _n_out(N, act))
+
+
+def aqt_linear_fwd_host(x_host: torch.Tensor, wq: torch.Tensor, s_w: torch.Tensor, bias: Optional[torch.Tensor],
+                        y_host: torch.Tensor, workspace: torch.Tensor, *, bits_a: int = 8, bits_w: int = 8,
+                        a_scale_kind: int = SCALE_ROW, rounding: int = ROUND_NEAREST_EVEN, act: int = ACT_NONE,
+                        stream=None) -> torch.Tensor:
+    """aqt_linear_fwd with x and y in (pinned) host memory; copies are enqueued on the stream."""
+    assert not x_host.is_cuda and not y_host.is_cuda and x_host.is_contiguous() and y_host.is_contiguous()
+    M, K = x_host.shape
+    N = wq.shape[0]
+    _check("aqt_linear_fwd_host", lib().aqt_linear_fwd_host(
+        _ptr(x_host), _ptr(wq), _ptr(s_w), _ptr(bias), _i64(M), _i64(N), _i64(K), int(bits_a), int(bits_w),
+        int(a_scale_kind), int(rounding), int(act), _ptr(y_host), _ptr(workspace), ctypes.c_size_t(workspace.numel()),
+        _stream(stream)))
+    return y_host

@@ -1,0 +1,247 @@
+// C ABI of the quantized linear layer: argument validation and kernel launches.
+// Single translation unit: the kernels live in the headers included below.
+#include "aqt_common.cuh"
+#include "pack.cuh"
+#include "qgemm_sm100.cuh"
+#include "quantize.cuh"
+
+using namespace aqt;
+
+namespace {
+
+// The kernels use tcgen05 / TMEM and exist for compute capability 10.x only.
+int check_device() {
+  static int cached = 1;  // 1 = not yet known
+  if (cached == 1) {
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return AQT_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return AQT_ERR_CUDA;
+    cached = (major == 10) ? AQT_OK : AQT_ERR_UNSUPPORTED;
+  }
+  return cached;
+}
+
+bool bits_ok(int b) { return b == 4 || b == 8; }
+bool act_ok(int a) { return a >= AQT_ACT_NONE && a <= AQT_ACT_GLU_SWISH; }
+bool is_glu(int a) { return a == AQT_ACT_GLU || a == AQT_ACT_GLU_SWISH; }
+
+size_t ws_qmatmul(int64_t M, int64_t N, int64_t K, int bits_a, int bits_w) {
+  size_t b = 0;
+  if (bits_a == 4) b += round_up((size_t)M * (size_t)K, 256);
+  if (bits_w == 4) b += round_up((size_t)N * (size_t)K, 256);
+  return b;
+}
+size_t ws_linear(int64_t M, int64_t N, int64_t K, int bits_w) {
+  return round_up((size_t)M * (size_t)K, 256) + round_up((size_t)M * 4, 256) + ws_qmatmul(0, N, K, 8, bits_w);
+}
+
+int validate_matmul_shape(int64_t M, int64_t N, int64_t K, int bits_a, int bits_w, int act, int s_x_kind) {
+  if (M < 0 || N < 0 || K <= 0) return AQT_ERR_BADARG;
+  if (!bits_ok(bits_a) || !bits_ok(bits_w) || !act_ok(act)) return AQT_ERR_BADARG;
+  if (s_x_kind != AQT_SCALE_ROW && s_x_kind != AQT_SCALE_TENSOR) return AQT_ERR_BADARG;
+  if (K % 32 != 0 || N % 4 != 0 || (is_glu(act) && N % 8 != 0)) return AQT_ERR_BADARG;
+  if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 31) || M * N >= (1ll << 40)) return AQT_ERR_UNSUPPORTED;
+  return AQT_OK;
+}
+
+// Codes already in int8 containers for A; B possibly packed.  ws holds B's unpacked copy.
+int qmatmul_i8a(const int8_t* a_codes, const float* s_x, int s_x_kind, const void* wq, const float* s_w, const float* bias,
+                const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K, int bits_w,
+                int act, float* y, int64_t ldy, int32_t* acc_debug, uint8_t* ws, cudaStream_t st) {
+  const int8_t* b_codes = reinterpret_cast<const int8_t*>(wq);
+  if (bits_w == 4) {
+    int rc = launch_unpack_int4(reinterpret_cast<const uint8_t*>(wq), N * K / 2, reinterpret_cast<int8_t*>(ws), st);
+    if (rc != AQT_OK) return rc;
+    b_codes = reinterpret_cast<const int8_t*>(ws);
+  }
+  GemmParams p;
+  p.s_x = s_x;
+  p.s_w = s_w;
+  p.bias = bias;
+  p.residual = residual;
+  p.acc_debug = acc_debug;
+  p.ldr = ldr;
+  p.residual_scale = residual_scale;
+  p.s_x_kind = s_x_kind;
+  p.act = act;
+  p.M = (int)M;
+  p.N = (int)N;
+  p.K = (int)K;
+  p.n_out = is_glu(act) ? (int)(N / 2) : (int)N;
+  p.tiles_m = p.tiles_n = p.k_blocks = 0;
+  return launch_qgemm(a_codes, b_codes, y, ldy, p, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+int aqt_version(void) { return AQT_VERSION; }
+
+const char* aqt_status_string(int status) {
+  switch (status) {
+    case AQT_OK: return "ok";
+    case AQT_ERR_BADARG: return "bad argument";
+    case AQT_ERR_ALIGN: return "misaligned pointer or pitch";
+    case AQT_ERR_UNSUPPORTED: return "unsupported device or size";
+    case AQT_ERR_WORKSPACE: return "workspace missing or too small";
+    case AQT_ERR_CUDA: return "CUDA call failed";
+    case AQT_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+size_t aqt_workspace_bytes(int op, int64_t M, int64_t N, int64_t K, int bits_a, int bits_w) {
+  if (M < 0 || N < 0 || K < 0) return 0;
+  if (op == AQT_OP_QMATMUL) return ws_qmatmul(M, N, K, bits_a, bits_w);
+  if (op == AQT_OP_LINEAR_FWD) return ws_linear(M, N, K, bits_w);
+  return 0;
+}
+
+int aqt_quantize(const float* x, int64_t rows, int64_t cols, int64_t ld, int bits, int axis, int rounding, int pack,
+                 void* q_out, float* scale_out, void* stream) {
+  if (rows < 0 || cols < 0 || ld < cols || !bits_ok(bits)) return AQT_ERR_BADARG;
+  if (axis != AQT_AXIS_ROW && axis != AQT_AXIS_COL && axis != AQT_AXIS_TENSOR) return AQT_ERR_BADARG;
+  if (rounding != AQT_ROUND_HALF_UP_FLOOR && rounding != AQT_ROUND_NEAREST_EVEN) return AQT_ERR_BADARG;
+  if (pack != 0 && pack != 1) return AQT_ERR_BADARG;
+  if (pack == 1 && (bits != 4 || cols % 2 != 0)) return AQT_ERR_BADARG;
+  if (rows == 0 || cols == 0) return AQT_OK;
+  if (x == nullptr || q_out == nullptr || scale_out == nullptr) return AQT_ERR_BADARG;
+  if (!is_aligned(x, 4) || !is_aligned(scale_out, 4)) return AQT_ERR_ALIGN;
+  int rc = check_device();
+  if (rc != AQT_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const int qmax = qmax_of(bits);
+  if (rounding == AQT_ROUND_HALF_UP_FLOOR) {
+    return pack ? launch_quantize_axis<AQT_ROUND_HALF_UP_FLOOR, true>(x, rows, cols, ld, qmax, axis, q_out, scale_out, st)
+                : launch_quantize_axis<AQT_ROUND_HALF_UP_FLOOR, false>(x, rows, cols, ld, qmax, axis, q_out, scale_out, st);
+  }
+  return pack ? launch_quantize_axis<AQT_ROUND_NEAREST_EVEN, true>(x, rows, cols, ld, qmax, axis, q_out, scale_out, st)
+              : launch_quantize_axis<AQT_ROUND_NEAREST_EVEN, false>(x, rows, cols, ld, qmax, axis, q_out, scale_out, st);
+}
+
+int aqt_pack_int4(const int8_t* q, int64_t rows, int64_t cols, uint8_t* packed, void* stream) {
+  if (rows < 0 || cols < 0 || cols % 2 != 0) return AQT_ERR_BADARG;
+  if (rows == 0 || cols == 0) return AQT_OK;
+  if (q == nullptr || packed == nullptr) return AQT_ERR_BADARG;
+  int rc = check_device();
+  if (rc != AQT_OK) return rc;
+  return launch_pack_int4(q, rows * cols / 2, packed, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int aqt_unpack_int4(const uint8_t* packed, int64_t rows, int64_t cols, int8_t* q, void* stream) {
+  if (rows < 0 || cols < 0 || cols % 2 != 0) return AQT_ERR_BADARG;
+  if (rows == 0 || cols == 0) return AQT_OK;
+  if (q == nullptr || packed == nullptr) return AQT_ERR_BADARG;
+  int rc = check_device();
+  if (rc != AQT_OK) return rc;
+  return launch_unpack_int4(packed, rows * cols / 2, q, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int aqt_qmatmul(const void* xq, const float* s_x, int s_x_kind, const void* wq, const float* s_w, const float* bias,
+                const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K, int bits_a,
+                int bits_w, int act, float* y, int64_t ldy, int32_t* acc_debug, void* workspace, size_t workspace_bytes,
+                void* stream) {
+  int rc = validate_matmul_shape(M, N, K, bits_a, bits_w, act, s_x_kind);
+  if (rc != AQT_OK) return rc;
+  if (M == 0 || N == 0) return AQT_OK;
+  const int64_t n_out = is_glu(act) ? N / 2 : N;
+  if (xq == nullptr || s_x == nullptr || wq == nullptr || s_w == nullptr || y == nullptr) return AQT_ERR_BADARG;
+  if (ldy < n_out || (residual != nullptr && ldr < n_out)) return AQT_ERR_BADARG;
+  if (!is_aligned(xq, 16) || !is_aligned(wq, 16) || !is_aligned(y, 16) || !is_aligned(s_w, 16) || !is_aligned(s_x, 4) ||
+      (bias != nullptr && !is_aligned(bias, 16)) || (residual != nullptr && !is_aligned(residual, 16)) ||
+      (acc_debug != nullptr && !is_aligned(acc_debug, 4)))
+    return AQT_ERR_ALIGN;
+  if (ldy % 4 != 0 || (residual != nullptr && ldr % 4 != 0)) return AQT_ERR_ALIGN;
+  const size_t need = ws_qmatmul(M, N, K, bits_a, bits_w);
+  if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return AQT_ERR_WORKSPACE;
+  if (need > 0 && !is_aligned(workspace, 256)) return AQT_ERR_ALIGN;
+  rc = check_device();
+  if (rc != AQT_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  const int8_t* a_codes = reinterpret_cast<const int8_t*>(xq);
+  if (bits_a == 4) {
+    rc = launch_unpack_int4(reinterpret_cast<const uint8_t*>(xq), M * K / 2, reinterpret_cast<int8_t*>(ws), st);
+    if (rc != AQT_OK) return rc;
+    a_codes = reinterpret_cast<const int8_t*>(ws);
+    ws += round_up((size_t)M * (size_t)K, 256);
+  }
+  return qmatmul_i8a(a_codes, s_x, s_x_kind, wq, s_w, bias, residual, ldr, residual_scale, M, N, K, bits_w, act, y, ldy,
+                     acc_debug, ws, st);
+}
+
+int aqt_linear_fwd(const float* x, int64_t ldx, const void* wq, const float* s_w, const float* bias, const float* residual,
+                   int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K, int bits_a, int bits_w,
+                   int a_scale_kind, int rounding, int act, float* y, int64_t ldy, void* workspace, size_t workspace_bytes,
+                   void* stream) {
+  int rc = validate_matmul_shape(M, N, K, bits_a, bits_w, act, a_scale_kind);
+  if (rc != AQT_OK) return rc;
+  if (rounding != AQT_ROUND_HALF_UP_FLOOR && rounding != AQT_ROUND_NEAREST_EVEN) return AQT_ERR_BADARG;
+  if (M == 0 || N == 0) return AQT_OK;
+  const int64_t n_out = is_glu(act) ? N / 2 : N;
+  if (x == nullptr || wq == nullptr || s_w == nullptr || y == nullptr) return AQT_ERR_BADARG;
+  if (ldx < K || ldy < n_out || (residual != nullptr && ldr < n_out)) return AQT_ERR_BADARG;
+  if (!is_aligned(x, 4) || !is_aligned(wq, 16) || !is_aligned(y, 16) || !is_aligned(s_w, 16) ||
+      (bias != nullptr && !is_aligned(bias, 16)) || (residual != nullptr && !is_aligned(residual, 16)))
+    return AQT_ERR_ALIGN;
+  if (ldy % 4 != 0 || (residual != nullptr && ldr % 4 != 0)) return AQT_ERR_ALIGN;
+  const size_t need = ws_linear(M, N, K, bits_w);
+  if (workspace == nullptr || workspace_bytes < need) return AQT_ERR_WORKSPACE;
+  if (!is_aligned(workspace, 256)) return AQT_ERR_ALIGN;
+  rc = check_device();
+  if (rc != AQT_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  int8_t* codes = reinterpret_cast<int8_t*>(ws);
+  float* s_x = reinterpret_cast<float*>(ws + round_up((size_t)M * (size_t)K, 256));
+  uint8_t* ws_mm = ws + round_up((size_t)M * (size_t)K, 256) + round_up((size_t)M * 4, 256);
+  // Step 1 (Fig. 2): dynamic quantization of the activations over K; 4-bit codes stay in int8
+  // containers between the two kernels, which is what the figure's cast produces.
+  const int axis = a_scale_kind == AQT_SCALE_ROW ? AQT_AXIS_ROW : AQT_AXIS_TENSOR;
+  rc = aqt_quantize(x, M, K, ldx, bits_a, axis, rounding, 0, codes, s_x, stream);
+  if (rc != AQT_OK) return rc;
+  // Step 2: integer matmul + de-quantizing epilogue.
+  return qmatmul_i8a(codes, s_x, a_scale_kind, wq, s_w, bias, residual, ldr, residual_scale, M, N, K, bits_w, act, y, ldy,
+                     nullptr, ws_mm, st);
+}
+
+int aqt_linear_fwd_host(const float* x_host, const void* wq, const float* s_w, const float* bias, int64_t M, int64_t N,
+                        int64_t K, int bits_a, int bits_w, int a_scale_kind, int rounding, int act, float* y_host,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = validate_matmul_shape(M, N, K, bits_a, bits_w, act, a_scale_kind);
+  if (rc != AQT_OK) return rc;
+  if (M == 0 || N == 0) return AQT_OK;
+  if (x_host == nullptr || y_host == nullptr) return AQT_ERR_BADARG;
+  const int64_t n_out = is_glu(act) ? N / 2 : N;
+  const size_t layer = round_up(ws_linear(M, N, K, bits_w), 256);
+  const size_t xb = round_up((size_t)M * K * 4, 256), yb = round_up((size_t)M * n_out * 4, 256);
+  if (workspace == nullptr || workspace_bytes < layer + xb + yb) return AQT_ERR_WORKSPACE;
+  if (!is_aligned(workspace, 256)) return AQT_ERR_ALIGN;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  float* x_dev = reinterpret_cast<float*>(ws + layer);
+  float* y_dev = reinterpret_cast<float*>(ws + layer + xb);
+  AQT_RETURN_IF_CUDA(cudaMemcpyAsync(x_dev, x_host, (size_t)M * K * 4, cudaMemcpyHostToDevice, st));
+  rc = aqt_linear_fwd(x_dev, K, wq, s_w, bias, nullptr, 0, 0.0f, M, N, K, bits_a, bits_w, a_scale_kind, rounding, act, y_dev,
+                      n_out, ws, layer, stream);
+  if (rc != AQT_OK) return rc;
+  AQT_RETURN_IF_CUDA(cudaMemcpyAsync(y_host, y_dev, (size_t)M * n_out * 4, cudaMemcpyDeviceToHost, st));
+  return AQT_OK;
+}
+
+int aqt_device_status(void* stream, int* status_out) {
+  if (status_out == nullptr) return AQT_ERR_BADARG;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  AQT_RETURN_IF_CUDA(cudaStreamSynchronize(st));
+  int v = 0;
+  AQT_RETURN_IF_CUDA(cudaMemcpyFromSymbol(&v, g_device_status, sizeof(int)));
+  if (v != 0) {
+    const int zero = 0;
+    AQT_RETURN_IF_CUDA(cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)));
+  }
+  *status_out = v;
+  return AQT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,93 @@
+// Shared host/device helpers of the quantized-linear library (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <stdlib.h>
+
+#include "../../include/aqt.h"
+
+namespace aqt {
+
+// Device status word: kernels record a bounded wait that ran out here; the host reads and
+// clears it in aqt_device_status().  One word per loaded library image and device.
+__device__ int g_device_status = 0;
+
+// With AQT_DEBUG set in the environment, failing CUDA calls are described on stderr.
+inline bool debug_enabled() {
+  static int on = -1;
+  if (on < 0) on = (getenv("AQT_DEBUG") != nullptr) ? 1 : 0;
+  return on == 1;
+}
+inline int cuda_fail(cudaError_t e, const char* what, int line) {
+  if (debug_enabled()) fprintf(stderr, "[aqt] %s (line %d): %s\n", what, line, cudaGetErrorString(e));
+  return AQT_ERR_CUDA;
+}
+
+#define AQT_RETURN_IF_CUDA(expr)                                      \
+  do {                                                                \
+    cudaError_t _e = (expr);                                          \
+    if (_e != cudaSuccess) return cuda_fail(_e, #expr, __LINE__);     \
+  } while (0)
+
+// Status of the launch just issued.
+#define AQT_LAUNCH_STATUS() (aqt::launch_status(__LINE__))
+inline int launch_status(int line) {
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? AQT_OK : cuda_fail(e, "kernel launch", line);
+}
+
+inline bool is_aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+__host__ __device__ inline int qmax_of(int bits) { return bits == 8 ? 127 : 7; }
+
+// Per-scale constants of the quantizer of Fig. 2 for one reduced group (row, column or tensor).
+// The figure divides every element by the scale in binary32.  The quotient x / s is formed here
+// as the correctly rounded binary32 value by one multiply and two fused multiply-adds against
+// the correctly rounded reciprocal r = RN(1/s): q0 = RN(x r), e = x - q0 s (exact in an fma),
+// v = RN(q0 + e r).  That sequence returns RN(x / s) whenever no intermediate leaves the normal
+// range, which `fast` records; otherwise elements take the IEEE division instruction sequence.
+struct ScaleCtx {
+  float s;    // scale = amax / qmax
+  float r;    // RN(1 / s), valid when fast
+  bool fast;  // amax within [2^-60, 2^60]
+};
+
+__device__ __forceinline__ ScaleCtx make_scale_ctx(float amax, int qmax) {
+  ScaleCtx c;
+  c.s = __fdiv_rn(amax, (float)qmax);
+  c.fast = (amax >= 8.6736174e-19f) && (amax <= 1.1529215e18f);
+  c.r = c.fast ? __frcp_rn(c.s) : 0.0f;
+  return c;
+}
+
+// One element of Fig. 2 after the scale is known: divide_no_nan, round, guard clip.
+template <int ROUNDING>
+__device__ __forceinline__ int quantize_elem(float x, const ScaleCtx& c, int qmax) {
+  float v;
+  if (c.fast) {
+    float q0 = __fmul_rn(x, c.r);
+    float e = __fmaf_rn(-q0, c.s, x);
+    v = __fmaf_rn(e, c.r, q0);
+  } else {
+    v = (c.s == 0.0f) ? 0.0f : __fdiv_rn(x, c.s);
+  }
+  int q;
+  if (ROUNDING == AQT_ROUND_HALF_UP_FLOOR) {
+    q = __float2int_rd(__fadd_rn(v, 0.5f));
+  } else {
+    q = __float2int_rn(v);
+  }
+  return max(-qmax, min(qmax, q));
+}
+
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+}  // namespace aqt

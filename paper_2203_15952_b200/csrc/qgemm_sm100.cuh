@@ -1,0 +1,558 @@
+// Integer GEMM on quantization codes with the de-quantizing epilogue, for sm_100a.
+//
+//   acc[m][n] = sum_k xq[m][k] * wq[n][k]      tcgen05.mma kind::i8, int32 accumulators in TMEM
+//   z = fma(float(acc) * s_x, s_w[n], bias[n]);  y = residual + residual_scale * act(z)
+//
+// One persistent CTA per SM walks output tiles of 128 x BN.  Warp roles:
+//   warp 0        TMA producer: A (activation codes) and B (weight codes) k-blocks of 128 bytes
+//                 into a ring of shared-memory stages, 128-byte swizzled, K-major
+//   warp 1        MMA issuer: one thread issues four K=32 MMAs per k-block into one of two TMEM
+//                 accumulator buffers and commits the stage back to the producer
+//   warps 2..9    epilogue: TMEM -> registers -> de-quantize / bias / activation / residual ->
+//                 swizzled shared staging -> TMA store; overlaps the next tile's MMAs
+// Every wait on an mbarrier is bounded by a wall-clock limit; on expiry the CTA records
+// AQT_ERR_TIMEOUT in the device status word, leaves its loops, frees its TMEM and returns.
+#pragma once
+
+#include <cuda.h>
+
+#include "aqt_common.cuh"
+
+namespace aqt {
+
+constexpr int kBM = 128;         // tile rows = TMEM lanes
+constexpr int kBK = 128;         // bytes (= int8 elements) of K per pipeline stage: one swizzle row
+constexpr int kMmaK = 32;        // K of one tcgen05.mma kind::i8
+constexpr int kEpiWarps = 8;     // two warps per TMEM lane quadrant
+constexpr int kGemmThreads = 32 * (2 + kEpiWarps);
+constexpr int kStoreBoxRows = 32;
+constexpr int kStoreBoxCols = 32;                                  // fp32: 128 bytes = one swizzle row
+constexpr int kStageBufBytes = kStoreBoxRows * kStoreBoxCols * 4;  // 4 KB
+constexpr int kStageBufsPerWarp = 1;  // 8 warps x 4 KB; the pipeline stages take the rest of shared memory
+constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
+
+template <int BN>
+struct GemmCfg {
+  static constexpr int kABytes = kBM * kBK;
+  static constexpr int kBBytes = BN * kBK;
+  static constexpr int kStages = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
+  static constexpr int kTmemCols = 2 * BN;  // two accumulator buffers; a power of two >= 32
+  static constexpr int kEpiBytes = kEpiWarps * kStageBufsPerWarp * kStageBufBytes;
+  static constexpr int kSmemBytes = kStages * (kABytes + kBBytes) + kEpiBytes + 1024;  // + alignment slack
+  static_assert(kSmemBytes + 512 <= 232448, "pipeline + staging must fit the 227 KB a CTA can opt into");
+};
+
+struct GemmParams {
+  const float* s_x;
+  const float* s_w;
+  const float* bias;
+  const float* residual;
+  int32_t* acc_debug;
+  int64_t ldr;
+  float residual_scale;
+  int s_x_kind;
+  int act;
+  int M, N, K;
+  int n_out;    // N, or N / 2 for the GLU forms
+  int tiles_m, tiles_n, k_blocks;
+};
+
+// ------------------------------------------------------------------------------------------------
+// PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return done != 0;
+}
+
+// Bounded wait.  Returns false if the CTA is aborting or the limit passed (and then sets both
+// the CTA's abort flag and the device status word).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint64_t t_start) {
+  for (uint32_t spin = 1;; ++spin) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((spin & 0xFF) == 0) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t_start > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicExch(&g_device_status, AQT_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* m) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
+}
+// 2-D tiled load into this CTA's shared memory, completion counted in bytes on `bar`.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* m, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(m)), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(
+                   reinterpret_cast<uint64_t>(m)),
+               "r"(c0), "r"(c1), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void tma_store_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// Arrive on an mbarrier once all MMAs issued so far by this thread have completed.
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, 128 x N x 32, signed 8-bit operands, int32 accumulate.
+__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp receives lane (base + i).
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand tile whose rows are 128 bytes, stored with the
+// 128-byte swizzle (what the TMA load writes); 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);  // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                    // leading-dimension offset: not used by swizzled K-major
+  d |= (uint64_t)(1024 >> 4) << 32;          // stride between 8-row groups
+  d |= (uint64_t)1 << 46;                    // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                    // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: D int32, A and B signed 8-bit, both K-major, M = 128, N = BN.
+__host__ __device__ constexpr uint32_t idesc_i8(int bn) {
+  return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Epilogue math
+
+__device__ __forceinline__ float sigmoid_f(float z) {
+  // 1 / (1 + e^-z): accurate exp (2 ulp), approximate reciprocal (1 ulp)
+  return __fdividef(1.0f, 1.0f + expf(-z));
+}
+
+__device__ __forceinline__ float4 ld4_guard(const float* base, int n, int limit, float fill) {
+  if (base == nullptr) return make_float4(fill, fill, fill, fill);
+  if (n + 3 < limit) return __ldg(reinterpret_cast<const float4*>(base + n));
+  float4 r;
+  r.x = n + 0 < limit ? __ldg(base + n + 0) : fill;
+  r.y = n + 1 < limit ? __ldg(base + n + 1) : fill;
+  r.z = n + 2 < limit ? __ldg(base + n + 2) : fill;
+  r.w = n + 3 < limit ? __ldg(base + n + 3) : fill;
+  return r;
+}
+
+// z for 32 consecutive accumulator columns starting at global column n0 (s_w / bias index).
+__device__ __forceinline__ void dequant32(const uint32_t (&acc)[32], float sx, const float* s_w, const float* bias,
+                                          int n0, int N, float (&z)[32]) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const float4 w = ld4_guard(s_w, n0 + 4 * j, N, 0.0f);
+    const float4 b = ld4_guard(bias, n0 + 4 * j, N, 0.0f);
+    z[4 * j + 0] = __fmaf_rn(__fmul_rn(__int2float_rn((int)acc[4 * j + 0]), sx), w.x, b.x);
+    z[4 * j + 1] = __fmaf_rn(__fmul_rn(__int2float_rn((int)acc[4 * j + 1]), sx), w.y, b.y);
+    z[4 * j + 2] = __fmaf_rn(__fmul_rn(__int2float_rn((int)acc[4 * j + 2]), sx), w.z, b.z);
+    z[4 * j + 3] = __fmaf_rn(__fmul_rn(__int2float_rn((int)acc[4 * j + 3]), sx), w.w, b.w);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// The kernel
+
+template <int BN>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                const __grid_constant__ CUtensorMap tm_y, const GemmParams p) {
+  using Cfg = GemmCfg<BN>;
+  constexpr int STAGES = Cfg::kStages;
+  constexpr int HALF = BN / 2;
+
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t full_bar[STAGES];
+  __shared__ uint64_t empty_bar[STAGES];
+  __shared__ uint64_t tmem_full_bar[2];
+  __shared__ uint64_t tmem_empty_bar[2];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms need 1024-byte alignment
+  const uint32_t smem_a = smem_base;
+  const uint32_t smem_b = smem_base + STAGES * Cfg::kABytes;
+  const uint32_t smem_epi = smem_b + STAGES * Cfg::kBBytes;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint64_t t_start = global_timer_ns();
+  const bool glu = (p.act == AQT_ACT_GLU) || (p.act == AQT_ACT_GLU_SWISH);
+  const int total_tiles = p.tiles_m * p.tiles_n;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    tma_prefetch_desc(&tm_a);
+    tma_prefetch_desc(&tm_b);
+    tma_prefetch_desc(&tm_y);
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&tmem_full_bar[b]), 1);
+      mbar_init(smem_u32(&tmem_empty_bar[b]), kEpiWarps);
+    }
+    fence_barrier_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&tmem_base_slot), Cfg::kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
+        // B rows of the two half-tiles: adjacent output channels, or (value, gate) halves for GLU
+        const int row0 = glu ? tn * HALF : tn * BN;
+        const int row1 = glu ? p.N / 2 + tn * HALF : tn * BN + HALF;
+        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+          if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1, &abort_flag, t_start)) { ok = false; break; }
+          const uint32_t bar = smem_u32(&full_bar[s]);
+          mbar_arrive_expect_tx(bar, Cfg::kABytes + Cfg::kBBytes);
+          tma_load_2d(smem_a + s * Cfg::kABytes, &tm_a, kb * kBK, tm * kBM, bar);
+          tma_load_2d(smem_b + s * Cfg::kBBytes, &tm_b, kb * kBK, row0, bar);
+          tma_load_2d(smem_b + s * Cfg::kBBytes + HALF * kBK, &tm_b, kb * kBK, row1, bar);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_i8(BN);
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+        const uint32_t buf = tcount & 1, aph = (tcount >> 1) & 1;
+        if (!mbar_wait(smem_u32(&tmem_empty_bar[buf]), aph ^ 1, &abort_flag, t_start)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * BN;
+        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+          if (!mbar_wait(smem_u32(&full_bar[s]), ph, &abort_flag, t_start)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t a_desc = smem_desc_k_major_sw128(smem_a + s * Cfg::kABytes);
+          const uint64_t b_desc = smem_desc_k_major_sw128(smem_b + s * Cfg::kBBytes);
+#pragma unroll
+          for (int kk = 0; kk < kBK / kMmaK; ++kk) {
+            // advancing K inside the 128-byte swizzle row: +32 bytes = +2 in the 16-byte address field
+            tc_mma_i8(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+          }
+          tc_commit(smem_u32(&empty_bar[s]));  // stage reusable once these MMAs have read it
+        }
+        if (ok) tc_commit(smem_u32(&tmem_full_bar[buf]));  // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps
+    const int ew = warp - 2;
+    const int quad = warp & 3;            // TMEM lane quadrant this warp may read
+    const int chalf = ew >> 2;            // which half of the tile's output columns
+    const uint32_t my_stage = smem_epi + ew * kStageBufsPerWarp * kStageBufBytes;
+    const int out_cols_tile = glu ? HALF : BN;       // output columns per tile
+    const int chunks = out_cols_tile / 32 / 2;       // 32-column chunks per epilogue warp
+    uint32_t tcount = 0, store_count = 0;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tcount) {
+      const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
+      const uint32_t buf = tcount & 1, aph = (tcount >> 1) & 1;
+      if (!mbar_wait(smem_u32(&tmem_full_bar[buf]), aph, &abort_flag, t_start)) break;
+      tc_fence_after();
+      const int m = tm * kBM + quad * 32 + lane;
+      const bool row_ok = m < p.M;
+      const float sx = (p.s_x_kind == AQT_SCALE_ROW) ? (row_ok ? __ldg(p.s_x + m) : 0.0f) : __ldg(p.s_x);
+      const uint32_t lane_addr = tmem_base + buf * BN + ((uint32_t)(quad * 32) << 16);
+      const int out0 = tn * out_cols_tile;  // first output column of the tile
+
+      for (int c = 0; c < chunks; ++c) {
+        const int col = (chalf * chunks + c) * 32;  // column offset inside the tile's output
+        float a[32];
+        uint32_t acc[32];
+        if (!glu) {
+          const int n0 = tn * BN + col;
+          tmem_ld_32x32(lane_addr + col, acc);
+          tmem_ld_wait();
+          if (p.acc_debug != nullptr && row_ok) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (n0 + j < p.N) p.acc_debug[(int64_t)m * p.N + n0 + j] = (int32_t)acc[j];
+          }
+          dequant32(acc, sx, p.s_w, p.bias, n0, p.N, a);
+          if (p.act == AQT_ACT_SWISH) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) a[j] = a[j] * sigmoid_f(a[j]);
+          }
+        } else {
+          const int nv = out0 + col;            // value channel
+          const int ng = p.N / 2 + out0 + col;  // gate channel
+          float g[32];
+          tmem_ld_32x32(lane_addr + col, acc);
+          tmem_ld_wait();
+          if (p.acc_debug != nullptr && row_ok) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (nv + j < p.N / 2) p.acc_debug[(int64_t)m * p.N + nv + j] = (int32_t)acc[j];
+          }
+          dequant32(acc, sx, p.s_w, p.bias, nv, p.N / 2, a);
+          tmem_ld_32x32(lane_addr + HALF + col, acc);
+          tmem_ld_wait();
+          if (p.acc_debug != nullptr && row_ok) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (ng + j < p.N) p.acc_debug[(int64_t)m * p.N + ng + j] = (int32_t)acc[j];
+          }
+          dequant32(acc, sx, p.s_w, p.bias, ng, p.N, g);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            a[j] = a[j] * sigmoid_f(g[j]);
+            if (p.act == AQT_ACT_GLU_SWISH) a[j] = a[j] * sigmoid_f(a[j]);
+          }
+        }
+        const int oc = out0 + col;  // first global output column of this chunk
+        if (p.residual != nullptr && row_ok) {
+          const float* rrow = p.residual + (int64_t)m * p.ldr;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float4 r = ld4_guard(rrow, oc + 4 * j, p.n_out, 0.0f);
+            a[4 * j + 0] = __fmaf_rn(p.residual_scale, a[4 * j + 0], r.x);
+            a[4 * j + 1] = __fmaf_rn(p.residual_scale, a[4 * j + 1], r.y);
+            a[4 * j + 2] = __fmaf_rn(p.residual_scale, a[4 * j + 2], r.z);
+            a[4 * j + 3] = __fmaf_rn(p.residual_scale, a[4 * j + 3], r.w);
+          }
+        }
+        // staging buffer free once the bulk store that last used it has read it
+        const uint32_t sbuf = my_stage + (store_count % kStageBufsPerWarp) * kStageBufBytes;
+        if (lane == 0) tma_store_wait_read<kStageBufsPerWarp - 1>();
+        __syncwarp();
+        // row `lane` of the 32 x 32 box; 16-byte chunk j sits at (j ^ (row & 7)) under the 128-byte swizzle
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t dst = sbuf + lane * 128 + ((j ^ (lane & 7)) << 4);
+          asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(a[4 * j]), "f"(a[4 * j + 1]),
+                       "f"(a[4 * j + 2]), "f"(a[4 * j + 3])
+                       : "memory");
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          // boxes that start inside the output are clipped at its edges by the copy engine
+          if (oc < p.n_out && tm * kBM + quad * 32 < p.M) tma_store_2d(&tm_y, sbuf, oc, tm * kBM + quad * 32);
+          tma_store_commit();
+        }
+        ++store_count;
+      }
+      // this warp has read its part of the accumulator buffer
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[buf]));
+    }
+    if (lane == 0) tma_store_wait_all();
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (abort_flag && threadIdx.x == 0) {
+    // give bulk copies that were in flight when a wait gave up time to land before smem is released
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 200000ull) {
+    }
+  }
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, Cfg::kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Host side: tensor maps and launch
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_tiled() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(sym);
+  }
+  return fn;
+}
+
+// 2-D row-major tensor [rows, cols] with `pitch_bytes` between rows; box [box_rows, box_cols];
+// 128-byte swizzle (box_cols * elem_bytes must be 128).
+static int make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const void* base, uint64_t rows,
+                       uint64_t cols, uint64_t pitch_bytes, uint32_t box_rows, uint32_t box_cols) {
+  EncodeTiledFn enc = get_encode_tiled();
+  if (enc == nullptr) {
+    if (debug_enabled()) fprintf(stderr, "[aqt] driver entry point for tensor map encoding not found\n");
+    return AQT_ERR_CUDA;
+  }
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {pitch_bytes};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  (void)elem_bytes;
+  CUresult r = enc(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS && debug_enabled())
+    fprintf(stderr, "[aqt] tensor map encode failed: CUresult %d (rows %llu cols %llu pitch %llu box %u x %u base %p)\n", (int)r,
+            (unsigned long long)rows, (unsigned long long)cols, (unsigned long long)pitch_bytes, box_rows, box_cols, base);
+  return r == CUDA_SUCCESS ? AQT_OK : AQT_ERR_CUDA;
+}
+
+static int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
+  }
+  return n;
+}
+
+// Rounds of a persistent grid over the tiles: fewer rounds of fuller waves win.
+static int pick_bn(int64_t M, int64_t N, bool glu, int sms) {
+  const int64_t tiles_m = ceil_div(M, kBM);
+  int best_bn = 128;
+  double best_cost = 1e300;
+  const int cands[3] = {256, 128, 64};
+  for (int i = 0; i < 3; ++i) {
+    const int bn = cands[i];
+    if (glu && bn == 64) continue;  // GLU output box needs at least 32 columns per half-tile warp pair
+    const int64_t tiles = tiles_m * ceil_div(N, bn);
+    const int64_t rounds = ceil_div(tiles, sms);
+    // per-tile cost: proportional to BN, plus a fixed per-tile overhead worth ~24 columns
+    const double cost = (double)rounds * (bn + 24);
+    if (cost < best_cost) {
+      best_cost = cost;
+      best_bn = bn;
+    }
+  }
+  return best_bn;
+}
+
+template <int BN>
+static int launch_qgemm_bn(const int8_t* a, const int8_t* b, float* y, int64_t ldy, const GemmParams& p0, cudaStream_t st) {
+  using Cfg = GemmCfg<BN>;
+  GemmParams p = p0;
+  p.tiles_m = (int)ceil_div(p.M, kBM);
+  p.tiles_n = (int)ceil_div(p.N, BN);
+  p.k_blocks = (int)ceil_div(p.K, kBK);
+  CUtensorMap tm_a, tm_b, tm_y;
+  int rc = make_map_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a, (uint64_t)p.M, (uint64_t)p.K, (uint64_t)p.K, kBM, kBK);
+  if (rc != AQT_OK) return rc;
+  rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, b, (uint64_t)p.N, (uint64_t)p.K, (uint64_t)p.K, BN / 2, kBK);
+  if (rc != AQT_OK) return rc;
+  rc = make_map_2d(&tm_y, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, y, (uint64_t)p.M, (uint64_t)p.n_out, (uint64_t)ldy * 4,
+                   kStoreBoxRows, kStoreBoxCols);
+  if (rc != AQT_OK) return rc;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (debug_enabled()) {
+      cudaFuncAttributes fa;
+      int dev = 0, optin = 0;
+      cudaGetDevice(&dev);
+      cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+      cudaError_t e = cudaFuncGetAttributes(&fa, qgemm_i8_kernel<BN>);
+      fprintf(stderr, "[aqt] qgemm<%d>: get-attr %s static smem %zu regs %d max dyn %d; device opt-in max %d; asking %d\n", BN,
+              cudaGetErrorString(e), fa.sharedSizeBytes, fa.numRegs, fa.maxDynamicSharedSizeBytes, optin, Cfg::kSmemBytes);
+    }
+    AQT_RETURN_IF_CUDA(cudaFuncSetAttribute(qgemm_i8_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
+    attr_set = true;
+  }
+  const int sms = sm_count();
+  if (sms <= 0) return AQT_ERR_CUDA;
+  const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
+  const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+  qgemm_i8_kernel<BN><<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tm_a, tm_b, tm_y, p);
+  return AQT_LAUNCH_STATUS();
+}
+
+// a: int8 [M, K] codes; b: int8 [N, K] codes (both dense, 16-byte aligned, K % 16 == 0).
+static int launch_qgemm(const int8_t* a, const int8_t* b, float* y, int64_t ldy, const GemmParams& p, cudaStream_t st) {
+  const bool glu = (p.act == AQT_ACT_GLU) || (p.act == AQT_ACT_GLU_SWISH);
+  const int bn = pick_bn(p.M, p.N, glu, sm_count() > 0 ? sm_count() : 148);
+  if (bn == 256) return launch_qgemm_bn<256>(a, b, y, ldy, p, st);
+  if (bn == 128) return launch_qgemm_bn<128>(a, b, y, ldy, p, st);
+  return launch_qgemm_bn<64>(a, b, y, ldy, p, st);
+}
+
+}  // namespace aqt

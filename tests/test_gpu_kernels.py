@@ -1,0 +1,220 @@
+"""Parity of each CUDA kernel against the CPU oracle, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+from paper_2203_15952_b200 import binding as aqt
+from paper_2203_15952_b200 import inputs as gen
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+
+
+def _status_ok():
+    assert aqt.aqt_device_status() == 0
+
+
+# ----------------------------------------------------------------------------- quantizer
+
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("rounding", [orc.ROUND_HALF_UP_FLOOR, orc.ROUND_NEAREST_EVEN])
+@pytest.mark.parametrize("shape", [(64, 256), (300, 512), (131, 1024), (70, 2048), (33, 4096), (40, 96), (17, 4100), (9, 37), (5, 8192)])
+def test_quantize_rows_bit_exact(bits, rounding, shape):
+    x = gen.normal(1, 100 + bits, shape[0], shape[1], std=1.7)
+    x[0, :] = 0.0                                     # zero row
+    x[1, 0] = 1e-41                                   # subnormal element
+    if shape[0] > 3:
+        x[2, :] *= 1e-30                              # tiny row (slow division path)
+        x[3, :] *= 1e25                               # huge row
+    q_ref, s_ref = orc.quantize(x, bits, orc.AXIS_ROW, rounding)
+    q, s = aqt.aqt_quantize(_dev(x), bits, aqt.AXIS_ROW, rounding)
+    assert np.array_equal(s.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    assert np.array_equal(q.cpu().numpy(), q_ref)
+    if shape[1] % 2 == 0 and bits == 4:
+        qp, s2 = aqt.aqt_quantize(_dev(x), 4, aqt.AXIS_ROW, rounding, pack=True)
+        assert np.array_equal(qp.cpu().numpy(), orc.pack_int4(q_ref))
+        assert np.array_equal(s2.cpu().numpy(), s_ref)
+
+
+def test_quantize_ties_and_half_ulp_cases():
+    """Exact ties and values one ulp either side of them, on the GPU's division sequence."""
+    base = np.arange(-127, 127, dtype=np.float32) + 0.5
+    vals = np.concatenate([base, np.nextafter(base, np.float32(1e9)), np.nextafter(base, np.float32(-1e9)), [127.0]]).astype(np.float32)
+    vals = np.concatenate([vals, np.zeros((-len(vals)) % 4, np.float32)])
+    x = np.stack([vals, vals * np.float32(3.0), vals * np.float32(0.1), vals * np.float32(1e-3)])
+    for rounding in (orc.ROUND_HALF_UP_FLOOR, orc.ROUND_NEAREST_EVEN):
+        q_ref, s_ref = orc.quantize(x, 8, orc.AXIS_ROW, rounding)
+        q, s = aqt.aqt_quantize(_dev(x), 8, aqt.AXIS_ROW, rounding)
+        assert np.array_equal(s.cpu().numpy(), s_ref) and np.array_equal(q.cpu().numpy(), q_ref)
+
+
+def test_quantize_strided_rows():
+    big = gen.normal(2, 5, 50, 640)
+    xd = _dev(big)[:, :512]
+    q_ref, s_ref = orc.quantize(np.ascontiguousarray(big[:, :512]), 8, orc.AXIS_ROW)
+    q, s = aqt.aqt_quantize(xd, 8, aqt.AXIS_ROW)
+    assert np.array_equal(q.cpu().numpy(), q_ref) and np.array_equal(s.cpu().numpy(), s_ref)
+
+
+@pytest.mark.parametrize("axis", [orc.AXIS_COL, orc.AXIS_TENSOR])
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("shape", [(64, 256), (512, 2048), (37, 53), (1000, 6)])
+def test_quantize_col_and_tensor_axes_bit_exact(axis, bits, shape):
+    x = gen.normal(3, 7, shape[0], shape[1], std=0.05)
+    for rounding in (orc.ROUND_HALF_UP_FLOOR, orc.ROUND_NEAREST_EVEN):
+        q_ref, s_ref = orc.quantize(x, bits, axis, rounding)
+        q, s = aqt.aqt_quantize(_dev(x), bits, axis, rounding)
+        assert np.array_equal(s.cpu().numpy(), s_ref) and np.array_equal(q.cpu().numpy(), q_ref)
+    if bits == 4 and shape[1] % 2 == 0:
+        qp, _ = aqt.aqt_quantize(_dev(x), 4, axis, orc.ROUND_NEAREST_EVEN, pack=True)
+        assert np.array_equal(qp.cpu().numpy(), orc.pack_int4(orc.quantize(x, 4, axis)[0]))
+
+
+def test_quantize_heavy_tailed_rows():
+    x = gen.student_t3(0, 77, 256, 1024)
+    q_ref, s_ref = orc.quantize(x, 8, orc.AXIS_ROW)
+    q, s = aqt.aqt_quantize(_dev(x), 8, aqt.AXIS_ROW)
+    assert np.array_equal(q.cpu().numpy(), q_ref) and np.array_equal(s.cpu().numpy(), s_ref)
+
+
+# ----------------------------------------------------------------------------- pack / unpack
+
+@pytest.mark.parametrize("shape", [(225, 2), (7, 90), (128, 512), (3, 4098), (1, 16)])
+def test_pack_unpack_bit_exact(shape):
+    rng = np.random.default_rng(shape[0])
+    q = rng.integers(-7, 8, shape).astype(np.int8)
+    packed_ref = orc.pack_int4(q)
+    packed = aqt.aqt_pack_int4(_dev(q))
+    assert np.array_equal(packed.cpu().numpy(), packed_ref)
+    assert np.array_equal(aqt.aqt_unpack_int4(packed, shape[1]).cpu().numpy(), q)
+    assert np.array_equal(aqt.aqt_unpack_int4(_dev(packed_ref), shape[1]).cpu().numpy(), orc.unpack_int4(packed_ref, shape[1]))
+
+
+# ----------------------------------------------------------------------------- integer matmul + epilogue
+
+def _codes(rng, rows, K, bits):
+    qm = 127 if bits == 8 else 7
+    return rng.integers(-qm, qm + 1, (rows, K)).astype(np.int8)
+
+
+def _run_qmatmul(M, N, K, bits_a, bits_w, act, with_bias, with_res, s_x_kind=aqt.SCALE_ROW, seed=0, extremes=False):
+    rng = np.random.default_rng(seed + 1000 * M + N + K)
+    xq = _codes(rng, M, K, bits_a)
+    wq = _codes(rng, N, K, bits_w)
+    if extremes:
+        xq[0, :] = 127 if bits_a == 8 else 7
+        wq[0, :] = 127 if bits_w == 8 else 7
+        wq[1 % N, :] = -wq[0, :]
+    s_x = rng.uniform(1e-3, 5e-2, M if s_x_kind == aqt.SCALE_ROW else 1).astype(np.float32)
+    s_w = rng.uniform(1e-4, 5e-3, N).astype(np.float32)
+    bias = (rng.standard_normal(N) * 0.1).astype(np.float32) if with_bias else None
+    n_out = N // 2 if act in (aqt.ACT_GLU, aqt.ACT_GLU_SWISH) else N
+    res = rng.standard_normal((M, n_out)).astype(np.float32) if with_res else None
+    acc_ref = orc.int_matmul(xq, wq)
+    y_ref = orc.epilogue_f32(acc_ref, s_x, s_x_kind, s_w, bias, res, 0.5, act)
+    y64 = orc.epilogue_f64(acc_ref, s_x, s_x_kind, s_w, bias, res, 0.5, act)
+
+    xq_d = _dev(orc.pack_int4(xq)) if bits_a == 4 else _dev(xq)
+    wq_d = _dev(orc.pack_int4(wq)) if bits_w == 4 else _dev(wq)
+    acc_d = torch.full((M, N), -12345, dtype=torch.int32, device=DEV)
+    y_d = torch.full((M, n_out), float("nan"), dtype=torch.float32, device=DEV)
+    aqt.aqt_qmatmul(xq_d, _dev(s_x), wq_d, _dev(s_w), None if bias is None else _dev(bias),
+                    None if res is None else _dev(res), 0.5, K=K, bits_a=bits_a, bits_w=bits_w, act=act,
+                    s_x_kind=s_x_kind, y=y_d, acc_debug=acc_d)
+    _status_ok()
+    acc = acc_d.cpu().numpy()
+    y = y_d.cpu().numpy()
+    assert np.array_equal(acc.astype(np.int64), acc_ref), "accumulators differ: %d of %d" % ((acc != acc_ref).sum(), acc.size)
+    if act == aqt.ACT_NONE:
+        assert np.array_equal(y.view(np.uint32), y_ref.view(np.uint32))          # only IEEE ops: bit-exact
+    else:
+        assert np.isfinite(y).all()
+        # float tolerance: 1e-6 relative to the larger of the result and the terms it is formed from
+        z = orc.epilogue_f64(acc_ref, s_x, s_x_kind, s_w, bias, None, 0.0, aqt.ACT_NONE)
+        mag = np.abs(y64)
+        zmag = np.abs(z[:, :n_out]) if z.shape[1] != n_out else np.abs(z)
+        mag = np.maximum(mag, zmag)
+        if res is not None:
+            mag = np.maximum(mag, np.abs(res))
+        assert np.all(np.abs(y - y64) <= 1e-6 * mag + 1e-30), float(np.max(np.abs(y - y64) / (mag + 1e-30)))
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 64, 128), (128, 128, 128), (128, 256, 128), (128, 256, 512), (256, 512, 256)])
+def test_qmatmul_single_tiles_int8(M, N, K):
+    _run_qmatmul(M, N, K, 8, 8, aqt.ACT_NONE, False, False, extremes=True)
+
+
+@pytest.mark.parametrize("M,N,K", [(64, 256, 256), (200, 192, 96), (1000, 520, 160), (129, 36, 32), (1, 4, 32), (333, 1536, 512)])
+def test_qmatmul_ragged_shapes(M, N, K):
+    _run_qmatmul(M, N, K, 8, 8, aqt.ACT_NONE, True, True)
+
+
+@pytest.mark.parametrize("bits_a,bits_w", [(8, 4), (4, 4), (4, 8)])
+@pytest.mark.parametrize("M,N,K", [(384, 512, 512), (130, 200, 2048)])
+def test_qmatmul_int4_operands(bits_a, bits_w, M, N, K):
+    _run_qmatmul(M, N, K, bits_a, bits_w, aqt.ACT_NONE, True, False, extremes=True)
+
+
+@pytest.mark.parametrize("act", [aqt.ACT_SWISH, aqt.ACT_GLU, aqt.ACT_GLU_SWISH])
+@pytest.mark.parametrize("M,N,K", [(256, 512, 256), (300, 1024, 512), (100, 136, 64)])
+def test_qmatmul_activations(act, M, N, K):
+    _run_qmatmul(M, N, K, 8, 4, act, True, True)
+
+
+def test_qmatmul_per_tensor_scale_and_deep_k():
+    _run_qmatmul(256, 256, 4096, 8, 8, aqt.ACT_NONE, True, False, s_x_kind=aqt.SCALE_TENSOR, extremes=True)
+
+
+def test_qmatmul_many_tiles_persistent_loop():
+    """More tiles than SMs, so every CTA walks several tiles and both accumulator buffers."""
+    _run_qmatmul(128 * 40, 2048, 512, 8, 8, aqt.ACT_SWISH, False, False)
+    _run_qmatmul(128 * 37 + 5, 512, 2048, 8, 8, aqt.ACT_NONE, False, True)
+
+
+# ----------------------------------------------------------------------------- whole layer
+
+@pytest.mark.parametrize("bits_a,bits_w,kind", [(8, 8, aqt.SCALE_TENSOR), (8, 4, aqt.SCALE_ROW), (4, 4, aqt.SCALE_ROW)])
+@pytest.mark.parametrize("rounding", [orc.ROUND_HALF_UP_FLOOR, orc.ROUND_NEAREST_EVEN])
+def test_linear_fwd_matches_oracle(bits_a, bits_w, kind, rounding):
+    M, K, N = 200, 512, 384
+    x = gen.normal(4, 1, M, K)
+    wt = gen.weight(4, 2, K, N)
+    bias = gen.normal(4, 3, 1, N, std=0.01)[0]
+    wq, s_w = orc.quantize(wt, bits_w, orc.AXIS_ROW, rounding)
+    y_ref = orc.linear_fwd(x, wq, s_w, bias=bias, bits_a=bits_a, a_scale_kind=kind, rounding=rounding)
+    # weights prepared on the GPU as well: quantize over K per output channel, pack if 4-bit
+    wq_d, sw_d = aqt.aqt_quantize(_dev(wt), bits_w, aqt.AXIS_ROW, rounding, pack=(bits_w == 4))
+    assert np.array_equal(sw_d.cpu().numpy(), s_w)
+    y = aqt.aqt_linear_fwd(_dev(x), wq_d, sw_d, _dev(bias), bits_a=bits_a, bits_w=bits_w, a_scale_kind=kind,
+                           rounding=rounding)
+    _status_ok()
+    assert np.array_equal(y.cpu().numpy().view(np.uint32), y_ref.view(np.uint32))
+
+
+def test_linear_fwd_host_buffers():
+    M, K, N = 256, 256, 256
+    x = gen.normal(5, 1, M, K)
+    wt = gen.weight(5, 2, K, N)
+    wq, s_w = orc.quantize(wt, 8, orc.AXIS_ROW)
+    y_ref = orc.linear_fwd(x, wq, s_w, act=orc.ACT_SWISH)
+    xh = torch.from_numpy(x).pin_memory()
+    yh = torch.empty((M, N), dtype=torch.float32).pin_memory()
+    ws = torch.empty(aqt.linear_fwd_host_workspace_bytes(M, N, K, 8, 8, aqt.ACT_SWISH), dtype=torch.uint8, device=DEV)
+    aqt.aqt_linear_fwd_host(xh, _dev(wq), _dev(s_w), None, yh, ws, act=aqt.ACT_SWISH)
+    _status_ok()
+    y = yh.numpy()
+    assert np.all(np.abs(y - y_ref) <= 1e-6 * np.maximum(np.abs(y_ref), 1e-3) + 1e-30)
+
+
+def test_status_codes_on_device():
+    x = torch.zeros((128, 128), dtype=torch.int8, device=DEV)
+    s = torch.ones(128, dtype=torch.float32, device=DEV)
+    with pytest.raises(aqt.AqtError) as e:
+        aqt.aqt_qmatmul(x, s, torch.zeros((128, 64), dtype=torch.uint8, device=DEV), s, K=128, bits_w=4,
+                        workspace=torch.empty(16, dtype=torch.uint8, device=DEV))
+    assert e.value.status == -4
