@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark of the quantized linear hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python -m torch.distributed.run --nnodes=1 --nproc-per-node N --master-addr 127.0.0.1 \
+        --master-port P bench.py --gpus N --steps K --warmup W
+
+Workload: the Conformer feed-forward pair (d_model 512 -> 2048 Swish -> 512, batch 32 x 400
+frames, int4 per-channel weights, int8 per-row dynamic activations), synthetic seeded inputs.
+One step = one pass of the whole path over one batch:
+    quantize(x) -> integer GEMM + de-quantize + Swish -> quantize(u) -> integer GEMM + de-quantize.
+Prints ONE JSON line (rank 0).  With N > 1 every rank runs the same batch size on its own GPU
+(rows are independent under per-row scales, so the path shards with no collective): weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "quantized Conformer linear TOPS (int4 weights, int8 activations)"
+UNIT = "TOPS"
+CFG = 2  # the Conformer FFN pair; fits one GPU many times over
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc, self.gpu = None, gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons, power = [], [], set(), []
+        for line in out.strip().splitlines():
+            f = [v.strip() for v in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "power_w_max": max(power), "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+def _dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# ------------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on the host cores
+
+def _oracle_weights(w, specs):
+    from oracle import conformer_ref as ref
+    from paper_2203_15952_b200 import inputs as gen
+    out = []
+    for i, s in enumerate(specs):
+        wq, sw = ref.prepare_weight(gen.layer_weight(w, 0, i, s), s.bits_w)
+        out.append((wq, sw, gen.layer_bias(w, 0, i, s)))
+    return out
+
+
+def _oracle_time_rows(w, specs, wts, rows: int, offset: int = 0) -> float:
+    """Seconds the oracle takes for the whole path on `rows` rows of the workload."""
+    from oracle import conformer_ref as ref
+    from paper_2203_15952_b200 import inputs as gen
+    sel = [(offset + i) % w.M for i in range(rows)]
+    x = gen.workload_input(w, row_subset=sel)
+    t0 = time.perf_counter()
+    ref.ffn_pair(specs, wts, x)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(budget_s: float = 15.0):
+    """Oracle throughput on a bounded row sample (rows are independent under per-row scales, so
+    rows / time is the oracle's rate for this path, not an extrapolation of other work)."""
+    import oracle as orc
+    from paper_2203_15952_b200 import inputs as gen
+    w = gen.WORKLOADS[CFG]
+    specs = gen.workload_layers(w)
+    wts = _oracle_weights(w, specs)
+    probe_rows = 128
+    t_probe = _oracle_time_rows(w, specs, wts, probe_rows)
+    # 10-30 s of CPU work: as many rows as the budget allows, in passes of at most M rows
+    rows_total = int(max(probe_rows, probe_rows * budget_s / max(t_probe, 1e-6))) // 64 * 64
+    rows, t, off = 0, 0.0, probe_rows
+    while rows < rows_total and t < 2 * budget_s:
+        n = min(w.M, rows_total - rows)
+        t += _oracle_time_rows(w, specs, wts, n, offset=off)
+        rows += n
+        off += n
+    ops_per_row = sum(2 * s.N * s.K for s in specs)
+    return {"value": rows * ops_per_row / t / 1e12, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+            "sample": "%d rows (batch of %d, rows cycled) of the FFN pair, whole path (quantize, int matmul, epilogue, twice), %.1f s" % (rows, w.M, t),
+            "frames_per_s": rows / t}
+
+
+def run_reference(args):
+    rank, world, _ = _dist_env()
+    if rank != 0:
+        return 0
+    import oracle as orc
+    from paper_2203_15952_b200 import inputs as gen
+    w = gen.WORKLOADS[CFG]
+    specs = gen.workload_layers(w)
+    wts = _oracle_weights(w, specs)
+    ops_per_row = sum(2 * s.N * s.K for s in specs)
+    t_probe = _oracle_time_rows(w, specs, wts, 128)
+    # a step = a row sample sized so that warm-up + steps finish within about two minutes
+    per_step_budget = 100.0 / max(1, args.steps + args.warmup)
+    rows = int(max(64, min(w.M, 128 * per_step_budget / max(t_probe, 1e-6)))) // 64 * 64
+    for i in range(args.warmup):
+        _oracle_time_rows(w, specs, wts, rows, offset=i * rows)
+    t = 0.0
+    for i in range(args.steps):
+        t += _oracle_time_rows(w, specs, wts, rows, offset=(args.warmup + i) * rows)
+    value = args.steps * rows * ops_per_row / t / 1e12
+    sample = "%d of %d rows per step, whole FFN-pair path on the CPU oracle" % (rows, w.M)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": {"workload": w.name, "rows_per_step": rows, "note": "CPU oracle on host cores; bounded row sample"},
+            "frames_per_s": args.steps * rows / t,
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2203_15952_b200 import binding as aqt
+    from paper_2203_15952_b200 import inputs as gen
+    from paper_2203_15952_b200.encoder import QuantLinear
+
+    rank, world, local = _dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = gen.WORKLOADS[CFG]
+    specs = gen.workload_layers(w)
+    M = w.M
+    # every rank works on its own batch of M rows (seeded by rank): weak scaling, no collective
+    seed = rank
+    layers = []
+    for i, s in enumerate(specs):
+        wt = torch.from_numpy(gen.layer_weight(w, 0, i, s, seed=0)).to(dev)
+        layers.append(QuantLinear.from_float(s, wt))
+    R = 6  # rotating input/output sets: x + u + y of one step exceed the 126 MB L2 already
+    x_host = gen.workload_input(w, seed=seed)
+    xs = [torch.from_numpy(x_host).to(dev) for _ in range(R)]
+    ys = [torch.empty((M, specs[1].N), dtype=torch.float32, device=dev) for _ in range(R)]
+    u = torch.empty((M, specs[0].N), dtype=torch.float32, device=dev)
+    q1 = torch.empty((M, specs[0].K), dtype=torch.int8, device=dev)
+    q2 = torch.empty((M, specs[1].K), dtype=torch.int8, device=dev)
+    s1 = torch.empty(M, dtype=torch.float32, device=dev)
+    s2 = torch.empty(M, dtype=torch.float32, device=dev)
+    ws = torch.empty(max(aqt.aqt_workspace_bytes(aqt.OP_QMATMUL, M, s.N, s.K, s.bits_a, s.bits_w) for s in specs) + 256,
+                     dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+    names = ["quantize(x) 12800x512", "qmatmul 512->2048 swish", "quantize(u) 12800x2048", "qmatmul 2048->512"]
+
+    # pre-marshalled C-ABI calls (one set per rotating buffer) so that Python stays ahead of the GPU
+    calls = []
+    for r in range(R):
+        calls.append((
+            aqt.bind_quantize(xs[r], specs[0].bits_a, aqt.AXIS_ROW, aqt.ROUND_NEAREST_EVEN, False, q1, s1),
+            aqt.bind_qmatmul(q1, s1, layers[0].wq, layers[0].s_w, None, None, 1.0, specs[0].K, 8, specs[0].bits_w, specs[0].act,
+                             aqt.SCALE_ROW, u, ws),
+            aqt.bind_quantize(u, specs[1].bits_a, aqt.AXIS_ROW, aqt.ROUND_NEAREST_EVEN, False, q2, s2),
+            aqt.bind_qmatmul(q2, s2, layers[1].wq, layers[1].s_w, None, None, 1.0, specs[1].K, 8, specs[1].bits_w, specs[1].act,
+                             aqt.SCALE_ROW, ys[r], ws)))
+
+    def step(i, events=None):
+        c = calls[i % R]
+        if events is None:
+            c[0](); c[1](); c[2](); c[3]()
+            return
+        events[0].record(stream)
+        for j in range(4):
+            c[j]()
+            events[j + 1].record(stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    if aqt.aqt_device_status() != 0:
+        raise SystemExit("device status reports a failed wait during warm-up")
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    barrier()
+    for i in range(args.steps):
+        step(i, evs[i])
+    barrier()
+    total_ms = evs[0][0].elapsed_time(evs[-1][4])
+    clocks = sampler.stop() if rank == 0 else None
+    status = aqt.aqt_device_status()
+
+    per_call_ms = [statistics.mean(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(args.steps)) for j in range(4)]
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    ops_step = sum(2 * M * s.N * s.K for s in specs)
+    value = world * args.steps * ops_step / (total_ms * 1e-3) / 1e12
+
+    # ---- end to end: host buffers through the C ABI, copies inside the timed region (per rank)
+    xh = torch.from_numpy(x_host).pin_memory()
+    yh = torch.empty((M, specs[1].N), dtype=torch.float32).pin_memory()
+    ws_a = torch.empty(aqt.linear_fwd_host_workspace_bytes(M, specs[0].N, specs[0].K, 8, 4, specs[0].act, True, False),
+                       dtype=torch.uint8, device=dev)
+    ws_b = torch.empty(aqt.linear_fwd_host_workspace_bytes(M, specs[1].N, specs[1].K, 8, 4, specs[1].act, False, True),
+                       dtype=torch.uint8, device=dev)
+
+    def e2e_step():
+        aqt.aqt_linear_fwd_host(xh, layers[0].wq, layers[0].s_w, None, u, ws_a, bits_a=8, bits_w=4, act=specs[0].act)
+        aqt.aqt_linear_fwd_host(u, layers[1].wq, layers[1].s_w, None, yh, ws_b, bits_a=8, bits_w=4, act=specs[1].act)
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e_value = world * args.steps * ops_step / (float(te.item()) * 1e-3) / 1e12
+
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank != 0:
+        return 0
+
+    # ---- roofline of the dominant call (largest share of the step)
+    peak, peak_kind = _peaks()
+    s0, s1_ = specs
+    alg_bytes = [
+        4 * M * s0.K + M * s0.K + 4 * M,                                              # quantize(x): read fp32, write codes + scales
+        M * s0.K + s0.K * s0.N // 2 + 8 * s0.N + 4 * M + 4 * M * s0.N,                # GEMM 1: codes, int4 weights, scales, fp32 out
+        4 * M * s1_.K + M * s1_.K + 4 * M,                                            # quantize(u)
+        M * s1_.K + s1_.K * s1_.N // 2 + 8 * s1_.N + 4 * M + 4 * M * s1_.N,           # GEMM 2
+    ]
+    kernels = [{"call": names[j], "ms": per_call_ms[j], "algorithmic_bytes": alg_bytes[j],
+                "gbs": alg_bytes[j] / (per_call_ms[j] * 1e-3) / 1e9, "share": per_call_ms[j] / sum(per_call_ms)} for j in range(4)]
+    dom = max(range(4), key=lambda j: per_call_ms[j])
+    achieved = kernels[dom]["gbs"]
+    roofline = {"bound": "hbm", "kernel": names[dom], "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "peak_source": "of " + peak_kind, "traffic": None, "calls": kernels}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int8", "data": "synthetic",
+            "config": {"workload": w.name, "M": M, "d_model": w.d, "ff": w.ff, "bits_w": 4, "bits_a": 8, "a_scale": "per-row",
+                       "rounding": "nearest-even", "l2": "rotating %d input/output sets; x + u + y of one step (157 MB) exceed the 126 MB L2" % R,
+                       "parallelism": "replicas x%d (rows sharded, no collective)" % world},
+            "frames_per_s": world * args.steps * M / (total_ms * 1e-3),
+            "clocks": clocks, "device_status": status,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 4 * M * s0.K, "d2h_bytes_per_step": 4 * M * s1_.N,
+                    "ms_per_step": float(te.item()) / args.steps},
+            "gpu_launches": args.steps * 6, "sum_call_ms_per_step": sum(per_call_ms),
+            "roofline": roofline}
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline()
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -133,17 +133,22 @@ int aqt_linear_fwd(const float* x, int64_t ldx, const void* wq, const float* s_w
                    void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * aqt_linear_fwd_host -- aqt_linear_fwd for callers whose activations live in HOST memory.
- * x_host    host fp32 [M, K] dense; y_host host fp32 [M, N_out] dense (pinned memory makes the
- *           copies asynchronous).  Weights, scales, bias stay device pointers.
- * workspace device memory, at least aqt_workspace_bytes(AQT_OP_LINEAR_FWD, ...) + 4*M*K + 4*M*N_out
- *           bytes: the device copies of x and y are placed behind the layer's own scratch.
- * The call enqueues the host-to-device copy, the layer, and the device-to-host copy on `stream`
- * and returns without synchronising.
+ * aqt_linear_fwd_host -- aqt_linear_fwd for callers whose activations live in HOST memory
+ * (Section 2.2's layer, unchanged; only where x and y live differs).
+ * x         fp32 [M, K] dense: a host pointer if x_on_host != 0, else a device pointer.
+ * y         fp32 [M, N_out] dense: a host pointer if y_on_host != 0, else a device pointer.
+ *           Pinned host memory makes the copies asynchronous.  Weights, scales and bias are
+ *           device pointers as everywhere else.  No residual input.
+ * workspace device memory, at least aqt_workspace_bytes(AQT_OP_LINEAR_FWD, ...) rounded up to
+ *           256, plus 4*M*K rounded up to 256 if x_on_host, plus 4*M*N_out if y_on_host: the
+ *           device copies of x and y are placed behind the layer's own scratch, in that order.
+ * The call enqueues the host-to-device copy, the layer and the device-to-host copy on `stream`
+ * and returns without synchronising.  Chaining two calls (host -> device, device -> host) runs a
+ * two-layer block with only its input and output crossing the bus.
  */
-int aqt_linear_fwd_host(const float* x_host, const void* wq, const float* s_w, const float* bias, int64_t M,
-                        int64_t N, int64_t K, int bits_a, int bits_w, int a_scale_kind, int rounding, int act,
-                        float* y_host, void* workspace, size_t workspace_bytes, void* stream);
+int aqt_linear_fwd_host(const float* x, int x_on_host, const void* wq, const float* s_w, const float* bias,
+                        int64_t M, int64_t N, int64_t K, int bits_a, int bits_w, int a_scale_kind, int rounding,
+                        int act, float* y, int y_on_host, void* workspace, size_t workspace_bytes, void* stream);
 
 /* Scratch bytes needed by `op` (AQT_OP_*) at these sizes; 0 if none.  Host-only, no CUDA call. */
 size_t aqt_workspace_bytes(int op, int64_t M, int64_t N, int64_t K, int bits_a, int bits_w);

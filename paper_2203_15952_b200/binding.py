@@ -76,6 +76,44 @@ def _n_out(N: int, act: int) -> int:
     return N // 2 if act in (ACT_GLU, ACT_GLU_SWISH) else N
 
 
+def bind(fn_name: str, *cargs):
+    """Pre-marshalled call: returns a zero-argument callable that invokes entry point `fn_name`
+    with the given ctypes arguments and raises AqtError on a non-zero status.  For launch-rate
+    sensitive loops (the arguments, including the stream, are fixed at bind time)."""
+    fn = getattr(lib(), fn_name)
+
+    def call():
+        st = fn(*cargs)
+        if st != AQT_OK:
+            raise AqtError(fn_name, st)
+    return call
+
+
+def bind_quantize(x, bits, axis, rounding, pack, q_out, scale_out, stream=None):
+    rows, cols = x.shape
+    return bind("aqt_quantize", _ptr(x), _i64(rows), _i64(cols), _i64(x.stride(0)), int(bits), int(axis), int(rounding),
+                int(bool(pack)), _ptr(q_out), _ptr(scale_out), _stream(stream))
+
+
+def bind_qmatmul(xq, s_x, wq, s_w, bias, residual, residual_scale, K, bits_a, bits_w, act, s_x_kind, y, workspace,
+                 stream=None):
+    M, N = xq.shape[0], wq.shape[0]
+    return bind("aqt_qmatmul", _ptr(xq), _ptr(s_x), int(s_x_kind), _ptr(wq), _ptr(s_w), _ptr(bias), _ptr(residual),
+                _i64(residual.stride(0) if residual is not None else 0), ctypes.c_float(residual_scale), _i64(M), _i64(N),
+                _i64(K), int(bits_a), int(bits_w), int(act), _ptr(y), _i64(y.stride(0)), _ptr(None), _ptr(workspace),
+                ctypes.c_size_t(0 if workspace is None else workspace.numel()), _stream(stream))
+
+
+def bind_linear_fwd(x, wq, s_w, bias, residual, residual_scale, bits_a, bits_w, a_scale_kind, rounding, act, y, workspace,
+                    stream=None):
+    M, K = x.shape
+    N = wq.shape[0]
+    return bind("aqt_linear_fwd", _ptr(x), _i64(x.stride(0)), _ptr(wq), _ptr(s_w), _ptr(bias), _ptr(residual),
+                _i64(residual.stride(0) if residual is not None else 0), ctypes.c_float(residual_scale), _i64(M), _i64(N),
+                _i64(K), int(bits_a), int(bits_w), int(a_scale_kind), int(rounding), int(act), _ptr(y), _i64(y.stride(0)),
+                _ptr(workspace), ctypes.c_size_t(workspace.numel()), _stream(stream))
+
+
 def aqt_version() -> int:
     return int(lib().aqt_version())
 
@@ -177,21 +215,28 @@ def aqt_linear_fwd(x: torch.Tensor, wq: torch.Tensor, s_w: torch.Tensor, bias: O
     return y
 
 
-def linear_fwd_host_workspace_bytes(M: int, N: int, K: int, bits_a: int, bits_w: int, act: int) -> int:
+def linear_fwd_host_workspace_bytes(M: int, N: int, K: int, bits_a: int, bits_w: int, act: int,
+                                    x_on_host: bool = True, y_on_host: bool = True) -> int:
     r256 = lambda v: (v + 255) // 256 * 256
-    return r256(aqt_workspace_bytes(OP_LINEAR_FWD, M, N, K, bits_a, bits_w)) + r256(4 * M * K) + r256(4 * M * _n_out(N, act))
+    need = r256(aqt_workspace_bytes(OP_LINEAR_FWD, M, N, K, bits_a, bits_w))
+    if x_on_host:
+        need += r256(4 * M * K)
+    if y_on_host:
+        need += r256(4 * M * _n_out(N, act))
+    return need
 
 
-def aqt_linear_fwd_host(x_host: torch.Tensor, wq: torch.Tensor, s_w: torch.Tensor, bias: Optional[torch.Tensor],
-                        y_host: torch.Tensor, workspace: torch.Tensor, *, bits_a: int = 8, bits_w: int = 8,
+def aqt_linear_fwd_host(x: torch.Tensor, wq: torch.Tensor, s_w: torch.Tensor, bias: Optional[torch.Tensor],
+                        y: torch.Tensor, workspace: torch.Tensor, *, bits_a: int = 8, bits_w: int = 8,
                         a_scale_kind: int = SCALE_ROW, rounding: int = ROUND_NEAREST_EVEN, act: int = ACT_NONE,
                         stream=None) -> torch.Tensor:
-    """aqt_linear_fwd with x and y in (pinned) host memory; copies are enqueued on the stream."""
-    assert not x_host.is_cuda and not y_host.is_cuda and x_host.is_contiguous() and y_host.is_contiguous()
-    M, K = x_host.shape
+    """aqt_linear_fwd with x and/or y in (pinned) host memory; copies are enqueued on the stream.
+    Whether a tensor is on the host is read from the tensor itself."""
+    assert x.is_contiguous() and y.is_contiguous() and x.dtype == torch.float32 and y.dtype == torch.float32
+    M, K = x.shape
     N = wq.shape[0]
     _check("aqt_linear_fwd_host", lib().aqt_linear_fwd_host(
-        _ptr(x_host), _ptr(wq), _ptr(s_w), _ptr(bias), _i64(M), _i64(N), _i64(K), int(bits_a), int(bits_w),
-        int(a_scale_kind), int(rounding), int(act), _ptr(y_host), _ptr(workspace), ctypes.c_size_t(workspace.numel()),
-        _stream(stream)))
-    return y_host
+        _ptr(x), int(not x.is_cuda), _ptr(wq), _ptr(s_w), _ptr(bias), _i64(M), _i64(N), _i64(K), int(bits_a), int(bits_w),
+        int(a_scale_kind), int(rounding), int(act), _ptr(y), int(not y.is_cuda), _ptr(workspace),
+        ctypes.c_size_t(workspace.numel()), _stream(stream)))
+    return y

@@ -206,27 +206,33 @@ int aqt_linear_fwd(const float* x, int64_t ldx, const void* wq, const float* s_w
                      nullptr, ws_mm, st);
 }
 
-int aqt_linear_fwd_host(const float* x_host, const void* wq, const float* s_w, const float* bias, int64_t M, int64_t N,
-                        int64_t K, int bits_a, int bits_w, int a_scale_kind, int rounding, int act, float* y_host,
-                        void* workspace, size_t workspace_bytes, void* stream) {
+int aqt_linear_fwd_host(const float* x, int x_on_host, const void* wq, const float* s_w, const float* bias, int64_t M,
+                        int64_t N, int64_t K, int bits_a, int bits_w, int a_scale_kind, int rounding, int act, float* y,
+                        int y_on_host, void* workspace, size_t workspace_bytes, void* stream) {
   int rc = validate_matmul_shape(M, N, K, bits_a, bits_w, act, a_scale_kind);
   if (rc != AQT_OK) return rc;
   if (M == 0 || N == 0) return AQT_OK;
-  if (x_host == nullptr || y_host == nullptr) return AQT_ERR_BADARG;
+  if (x == nullptr || y == nullptr) return AQT_ERR_BADARG;
   const int64_t n_out = is_glu(act) ? N / 2 : N;
   const size_t layer = round_up(ws_linear(M, N, K, bits_w), 256);
-  const size_t xb = round_up((size_t)M * K * 4, 256), yb = round_up((size_t)M * n_out * 4, 256);
+  const size_t xb = x_on_host ? round_up((size_t)M * K * 4, 256) : 0;
+  const size_t yb = y_on_host ? round_up((size_t)M * n_out * 4, 256) : 0;
   if (workspace == nullptr || workspace_bytes < layer + xb + yb) return AQT_ERR_WORKSPACE;
   if (!is_aligned(workspace, 256)) return AQT_ERR_ALIGN;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
-  float* x_dev = reinterpret_cast<float*>(ws + layer);
-  float* y_dev = reinterpret_cast<float*>(ws + layer + xb);
-  AQT_RETURN_IF_CUDA(cudaMemcpyAsync(x_dev, x_host, (size_t)M * K * 4, cudaMemcpyHostToDevice, st));
+  const float* x_dev = x;
+  float* y_dev = y;
+  if (x_on_host) {
+    float* xd = reinterpret_cast<float*>(ws + layer);
+    AQT_RETURN_IF_CUDA(cudaMemcpyAsync(xd, x, (size_t)M * K * 4, cudaMemcpyHostToDevice, st));
+    x_dev = xd;
+  }
+  if (y_on_host) y_dev = reinterpret_cast<float*>(ws + layer + xb);
   rc = aqt_linear_fwd(x_dev, K, wq, s_w, bias, nullptr, 0, 0.0f, M, N, K, bits_a, bits_w, a_scale_kind, rounding, act, y_dev,
                       n_out, ws, layer, stream);
   if (rc != AQT_OK) return rc;
-  AQT_RETURN_IF_CUDA(cudaMemcpyAsync(y_host, y_dev, (size_t)M * n_out * 4, cudaMemcpyDeviceToHost, st));
+  if (y_on_host) AQT_RETURN_IF_CUDA(cudaMemcpyAsync(y, y_dev, (size_t)M * n_out * 4, cudaMemcpyDeviceToHost, st));
   return AQT_OK;
 }
 

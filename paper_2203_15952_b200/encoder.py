@@ -1,0 +1,149 @@
+"""Chains of quantized linears on the GPU: FFN pair, Conformer block, encoder stack.
+
+Every arithmetic step is a call into the C ABI (binding.aqt_*); this module only owns buffers and
+the order of calls.  The dataflow is the stand-in block used by the workloads: the parts of a
+Conformer block that are not weight-bearing linears (attention scores, depthwise convolution,
+normalisation) are not on the quantized path (Section 3.3 quantizes the encoder's linears only)
+and are replaced by the identity:
+
+    h <- h + 1/2 * W_a2 . Swish(W_a1 . h)          feed-forward module a
+    q, k, v <- W_q . h, W_k . h, W_v . h            attention projections
+    h <- h + W_o . v
+    c <- Swish(GLU(W_pw1 . h))                      convolution module, pointwise 1
+    h <- h + W_pw2 . c                              pointwise 2
+    h <- h + 1/2 * W_b2 . Swish(W_b1 . h)          feed-forward module b
+
+Residual adds are fp32 and are fused into the epilogue of the producing linear.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Dict, List, Optional
+
+import torch
+
+from . import binding as aqt
+from .inputs import LinearSpec
+
+
+@dataclass
+class QuantLinear:
+    """Pre-quantized weights of one linear: codes W^T [N, K] (nibble-packed when 4-bit), one
+    fp32 scale per output channel (Section 2.2, channel-wise), optional fp32 bias."""
+    spec: LinearSpec
+    wq: torch.Tensor
+    s_w: torch.Tensor
+    bias: Optional[torch.Tensor]
+
+    @classmethod
+    def from_float(cls, spec: LinearSpec, wt: torch.Tensor, bias: Optional[torch.Tensor] = None,
+                   rounding: int = aqt.ROUND_NEAREST_EVEN) -> "QuantLinear":
+        """wt: fp32 W^T [N, K] on the GPU.  Quantizes over K per output channel with the same
+        quantizer the activations use (Fig. 2), packing 4-bit codes two per byte."""
+        assert wt.shape == (spec.N, spec.K)
+        wq, s_w = aqt.aqt_quantize(wt, spec.bits_w, aqt.AXIS_ROW, rounding, pack=(spec.bits_w == 4))
+        return cls(spec, wq, s_w, bias)
+
+    @property
+    def weight_bytes(self) -> int:
+        return self.wq.numel() + 4 * self.s_w.numel()
+
+
+class LayerRunner:
+    """Owns the scratch workspace shared by all layers of a workload and runs single layers."""
+
+    def __init__(self, M: int, layers: List[QuantLinear], device, a_scale_kind: int = aqt.SCALE_ROW,
+                 rounding: int = aqt.ROUND_NEAREST_EVEN):
+        self.M, self.device, self.a_scale_kind, self.rounding = M, device, a_scale_kind, rounding
+        need = max(aqt.aqt_workspace_bytes(aqt.OP_LINEAR_FWD, M, l.spec.N, l.spec.K, l.spec.bits_a, l.spec.bits_w) for l in layers)
+        self.workspace = torch.empty(need, dtype=torch.uint8, device=device)
+
+    def __call__(self, layer: QuantLinear, x: torch.Tensor, y: torch.Tensor, residual: Optional[torch.Tensor] = None,
+                 residual_scale: float = 1.0) -> torch.Tensor:
+        s = layer.spec
+        return aqt.aqt_linear_fwd(x, layer.wq, layer.s_w, layer.bias, residual, residual_scale, bits_a=s.bits_a,
+                                  bits_w=s.bits_w, a_scale_kind=self.a_scale_kind, rounding=self.rounding, act=s.act,
+                                  y=y, workspace=self.workspace)
+
+
+class FfnPair:
+    """y = W_2 . Swish(W_1 . x): the second layer re-quantizes the first layer's fp32 output."""
+
+    def __init__(self, M: int, layers: List[QuantLinear], device, **kw):
+        assert len(layers) == 2
+        self.layers = layers
+        self.run = LayerRunner(M, layers, device, **kw)
+        self.u = torch.empty((M, layers[0].spec.n_out), dtype=torch.float32, device=device)
+
+    def forward(self, x: torch.Tensor, y: torch.Tensor) -> torch.Tensor:
+        self.run(self.layers[0], x, self.u)
+        return self.run(self.layers[1], self.u, y)
+
+    @property
+    def ops(self) -> int:
+        return sum(2 * self.run.M * l.spec.N * l.spec.K for l in self.layers)
+
+
+class ConformerBlockLinears:
+    """The ten linears of one block in the stand-in dataflow above.  Buffers are allocated once
+    and shared by every block of a stack."""
+
+    def __init__(self, M: int, d: int, ff: int, layers_for_sizing: List[QuantLinear], device, **kw):
+        self.M, self.d, self.ff = M, d, ff
+        self.run = LayerRunner(M, layers_for_sizing, device, **kw)
+        f32 = dict(dtype=torch.float32, device=device)
+        self.u = torch.empty((M, ff), **f32)
+        self.q = torch.empty((M, d), **f32)
+        self.k = torch.empty((M, d), **f32)
+        self.v = torch.empty((M, d), **f32)
+        self.c = torch.empty((M, d), **f32)
+        self.h_a = torch.empty((M, d), **f32)
+        self.h_b = torch.empty((M, d), **f32)
+
+    def forward(self, layers: List[QuantLinear], h_in: torch.Tensor, h_out: torch.Tensor,
+                keep: Optional[Dict[str, torch.Tensor]] = None) -> torch.Tensor:
+        """h_in -> h_out (distinct buffers, neither h_a nor h_b).  `keep`, if given, receives
+        clones of every intermediate keyed by layer name (for parity checks)."""
+        L, run = layers, self.run
+
+        def note(name, t):
+            if keep is not None:
+                keep[name] = t.clone()
+
+        run(L[0], h_in, self.u); note(L[0].spec.name, self.u)
+        run(L[1], self.u, self.h_a, residual=h_in, residual_scale=0.5); note(L[1].spec.name, self.h_a)
+        run(L[2], self.h_a, self.q); note(L[2].spec.name, self.q)
+        run(L[3], self.h_a, self.k); note(L[3].spec.name, self.k)
+        run(L[4], self.h_a, self.v); note(L[4].spec.name, self.v)
+        run(L[5], self.v, self.h_b, residual=self.h_a, residual_scale=1.0); note(L[5].spec.name, self.h_b)
+        run(L[6], self.h_b, self.c); note(L[6].spec.name, self.c)
+        run(L[7], self.c, self.h_a, residual=self.h_b, residual_scale=1.0); note(L[7].spec.name, self.h_a)
+        run(L[8], self.h_a, self.u); note(L[8].spec.name, self.u)
+        run(L[9], self.u, h_out, residual=self.h_a, residual_scale=0.5); note(L[9].spec.name, h_out)
+        return h_out
+
+    def ops(self, layers: List[QuantLinear]) -> int:
+        return sum(2 * self.M * l.spec.N * l.spec.K for l in layers)
+
+
+class EncoderStack:
+    """n_blocks blocks in sequence, ping-ponging the residual stream between two buffers."""
+
+    def __init__(self, M: int, d: int, ff: int, blocks: List[List[QuantLinear]], device, **kw):
+        self.blocks = blocks
+        self.block = ConformerBlockLinears(M, d, ff, blocks[0], device, **kw)
+        self.h0 = torch.empty((M, d), dtype=torch.float32, device=device)
+        self.h1 = torch.empty((M, d), dtype=torch.float32, device=device)
+
+    def forward(self, x: torch.Tensor) -> torch.Tensor:
+        """x is read only; the result lives in one of the stack's own buffers."""
+        src = x
+        for b, layers in enumerate(self.blocks):
+            dst = self.h0 if b % 2 == 0 else self.h1
+            self.block.forward(layers, src, dst)
+            src = dst
+        return src
+
+    @property
+    def ops(self) -> int:
+        return sum(self.block.ops(layers) for layers in self.blocks)
