@@ -46,7 +46,7 @@ int validate_matmul_shape(int64_t M, int64_t N, int64_t K, int bits_a, int bits_
 
 // Codes already in int8 containers for A; B possibly packed.  ws holds B's unpacked copy.
 int qmatmul_i8a(const int8_t* a_codes, const float* s_x, int s_x_kind, const void* wq, const float* s_w, const float* bias,
-                const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K, int bits_w,
+                const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K, int bits_a, int bits_w,
                 int act, float* y, int64_t ldy, int32_t* acc_debug, uint8_t* ws, cudaStream_t st) {
   const int8_t* b_codes = reinterpret_cast<const int8_t*>(wq);
   if (bits_w == 4) {
@@ -69,6 +69,8 @@ int qmatmul_i8a(const int8_t* a_codes, const float* s_x, int s_x_kind, const voi
   p.K = (int)K;
   p.n_out = is_glu(act) ? (int)(N / 2) : (int)N;
   p.tiles_m = p.tiles_n = p.k_blocks = 0;
+  // |acc| <= K * qmax_a * qmax_w (codes never reach -qmax - 1, Section 2.2's symmetric range)
+  p.small_acc = (K * (int64_t)qmax_of(bits_a) * qmax_of(bits_w) < (1ll << 22)) ? 1 : 0;
   return launch_qgemm(a_codes, b_codes, y, ldy, p, st);
 }
 
@@ -167,8 +169,8 @@ int aqt_qmatmul(const void* xq, const float* s_x, int s_x_kind, const void* wq, 
     a_codes = reinterpret_cast<const int8_t*>(ws);
     ws += round_up((size_t)M * (size_t)K, 256);
   }
-  return qmatmul_i8a(a_codes, s_x, s_x_kind, wq, s_w, bias, residual, ldr, residual_scale, M, N, K, bits_w, act, y, ldy,
-                     acc_debug, ws, st);
+  return qmatmul_i8a(a_codes, s_x, s_x_kind, wq, s_w, bias, residual, ldr, residual_scale, M, N, K, bits_a, bits_w, act, y,
+                     ldy, acc_debug, ws, st);
 }
 
 int aqt_linear_fwd(const float* x, int64_t ldx, const void* wq, const float* s_w, const float* bias, const float* residual,
@@ -202,8 +204,8 @@ int aqt_linear_fwd(const float* x, int64_t ldx, const void* wq, const float* s_w
   rc = aqt_quantize(x, M, K, ldx, bits_a, axis, rounding, 0, codes, s_x, stream);
   if (rc != AQT_OK) return rc;
   // Step 2: integer matmul + de-quantizing epilogue.
-  return qmatmul_i8a(codes, s_x, a_scale_kind, wq, s_w, bias, residual, ldr, residual_scale, M, N, K, bits_w, act, y, ldy,
-                     nullptr, ws_mm, st);
+  return qmatmul_i8a(codes, s_x, a_scale_kind, wq, s_w, bias, residual, ldr, residual_scale, M, N, K, bits_a, bits_w, act, y,
+                     ldy, nullptr, ws_mm, st);
 }
 
 int aqt_linear_fwd_host(const float* x, int x_on_host, const void* wq, const float* s_w, const float* bias, int64_t M,

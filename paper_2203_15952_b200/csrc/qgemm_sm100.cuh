@@ -9,7 +9,8 @@
 //   warp 1        MMA issuer: one thread issues four K=32 MMAs per k-block into one of two TMEM
 //                 accumulator buffers and commits the stage back to the producer
 //   warps 2..9    epilogue: TMEM -> registers -> de-quantize / bias / activation / residual ->
-//                 swizzled shared staging -> TMA store; overlaps the next tile's MMAs
+//                 swizzled shared staging -> TMA store; overlaps the next tile's MMAs.  The
+//                 residual tile is fetched by TMA into the same staging buffer beforehand.
 // Every wait on an mbarrier is bounded by a wall-clock limit; on expiry the CTA records
 // AQT_ERR_TIMEOUT in the device status word, leaves its loops, frees its TMEM and returns.
 #pragma once
@@ -23,22 +24,30 @@ namespace aqt {
 constexpr int kBM = 128;         // tile rows = TMEM lanes
 constexpr int kBK = 128;         // bytes (= int8 elements) of K per pipeline stage: one swizzle row
 constexpr int kMmaK = 32;        // K of one tcgen05.mma kind::i8
-constexpr int kEpiWarps = 8;     // two warps per TMEM lane quadrant
-constexpr int kGemmThreads = 32 * (2 + kEpiWarps);
+constexpr int kStageBufsPerWarp = 2;  // a warp fills one output staging buffer while the other is being stored
 constexpr int kStoreBoxRows = 32;
 constexpr int kStoreBoxCols = 32;                                  // fp32: 128 bytes = one swizzle row
 constexpr int kStageBufBytes = kStoreBoxRows * kStoreBoxCols * 4;  // 4 KB
-constexpr int kStageBufsPerWarp = 1;  // 8 warps x 4 KB; the pipeline stages take the rest of shared memory
-constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
+constexpr int kScaleSlabFloats = 2 * 32 * 4;                       // per-warp s_w and bias slices: up to 4 chunks of 32
+constexpr uint64_t kWaitLimitNs = 2000000000ull;                   // 2 s
 
-template <int BN>
+// BN: tile width.  STAGES: depth of the operand ring.  EW: epilogue warps, 4 (one per TMEM lane
+// quadrant) or 8 (two per quadrant, each taking half of the tile's columns).  Shallow-K shapes are
+// bound by the epilogue and take EW = 8; deep-K shapes are bound by operand loads and give the
+// shared memory of four staging warps to the ring.
+template <int BN, int STAGES, int EW>
 struct GemmCfg {
+  static constexpr int kThreads = 32 * (2 + EW);
   static constexpr int kABytes = kBM * kBK;
   static constexpr int kBBytes = BN * kBK;
-  static constexpr int kStages = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
+  static constexpr int kStages = STAGES;
   static constexpr int kTmemCols = 2 * BN;  // two accumulator buffers; a power of two >= 32
-  static constexpr int kEpiBytes = kEpiWarps * kStageBufsPerWarp * kStageBufBytes;
-  static constexpr int kSmemBytes = kStages * (kABytes + kBBytes) + kEpiBytes + 1024;  // + alignment slack
+  static constexpr int kEpiBytes = EW * kStageBufsPerWarp * kStageBufBytes;
+  // With EW == 8 each warp keeps its s_w / bias slices in shared memory; with EW == 4 the scales
+  // are read through L1 instead (the epilogue is a small part of a deep-K tile).
+  static constexpr bool kScaleSlab = (EW == 8);
+  static constexpr int kScaleBytes = kScaleSlab ? EW * kScaleSlabFloats * 4 : 0;
+  static constexpr int kSmemBytes = STAGES * (kABytes + kBBytes) + kEpiBytes + kScaleBytes + 1024;  // + alignment slack
   static_assert(kSmemBytes + 512 <= 232448, "pipeline + staging must fit the 227 KB a CTA can opt into");
 };
 
@@ -55,6 +64,7 @@ struct GemmParams {
   int M, N, K;
   int n_out;    // N, or N / 2 for the GLU forms
   int tiles_m, tiles_n, k_blocks;
+  int small_acc;  // every |accumulator| < 2^22: the int -> float conversion can use the exponent trick
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -183,52 +193,101 @@ __host__ __device__ constexpr uint32_t idesc_i8(int bn) {
 // ------------------------------------------------------------------------------------------------
 // Epilogue math
 
-__device__ __forceinline__ float sigmoid_f(float z) {
-  // 1 / (1 + e^-z): accurate exp (2 ulp), approximate reciprocal (1 ulp)
-  return __fdividef(1.0f, 1.0f + expf(-z));
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+  float y;
+  asm("rcp.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 
-__device__ __forceinline__ float4 ld4_guard(const float* base, int n, int limit, float fill) {
-  if (base == nullptr) return make_float4(fill, fill, fill, fill);
+// sigmoid(z) = 1 / (1 + e^-z).  e^-z = 2^t with t = -z log2(e) formed in two pieces (the rounded
+// product and its exact remainder) so that the exponent's rounding error does not grow with |z|;
+// the special-function unit supplies 2^t and the reciprocal.  Relative error about 4e-7.
+// z is clamped at -87 so that e^-z stays finite (sigmoid is below 2e-38 there).
+__device__ __forceinline__ float sigmoid_f(float z) {
+  const float kHi = -1.4426950216293335f;     // RN(-log2 e)
+  const float kLo = -1.9259629911266175e-8f;  // -log2 e - kHi
+  const float zc = fmaxf(z, -87.0f);
+  const float t = __fmul_rn(zc, kHi);
+  float r = __fmaf_rn(zc, kHi, -t);
+  r = __fmaf_rn(zc, kLo, r);
+  const float e = ex2_approx(t);
+  const float en = __fmaf_rn(e, r * 0.69314718f, e);  // 2^(t + r) ~ 2^t (1 + r ln 2)
+  return rcp_approx(1.0f + en);
+}
+
+// int32 accumulator -> float, round-to-nearest-even (exact below 2^24).  With SMALL the caller
+// guarantees |acc| < 2^22: adding the integer to the bit pattern of 1.5 * 2^23 and subtracting
+// that constant is exact and stays off the conversion unit.
+template <bool SMALL>
+__device__ __forceinline__ float acc_to_float(uint32_t acc) {
+  if (SMALL) return __int_as_float(0x4B400000 + (int)acc) - 12582912.0f;
+  return __int2float_rn((int)acc);
+}
+
+// z[i] = fma(float(acc[i]) * sx, s_w[i], bias[i]) for 32 consecutive columns whose scales and
+// biases sit at `sw_smem` / `b_smem` (shared-memory byte addresses, 16-byte aligned).
+template <bool SMALL>
+__device__ __forceinline__ void dequant32(const uint32_t (&acc)[32], float sx, uint32_t sw_smem, uint32_t b_smem, float (&z)[32]) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    float w0, w1, w2, w3, b0, b1, b2, b3;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(w0), "=f"(w1), "=f"(w2), "=f"(w3) : "r"(sw_smem + 16 * j));
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(b0), "=f"(b1), "=f"(b2), "=f"(b3) : "r"(b_smem + 16 * j));
+    z[4 * j + 0] = __fmaf_rn(__fmul_rn(acc_to_float<SMALL>(acc[4 * j + 0]), sx), w0, b0);
+    z[4 * j + 1] = __fmaf_rn(__fmul_rn(acc_to_float<SMALL>(acc[4 * j + 1]), sx), w1, b1);
+    z[4 * j + 2] = __fmaf_rn(__fmul_rn(acc_to_float<SMALL>(acc[4 * j + 2]), sx), w2, b2);
+    z[4 * j + 3] = __fmaf_rn(__fmul_rn(acc_to_float<SMALL>(acc[4 * j + 3]), sx), w3, b3);
+  }
+}
+
+__device__ __forceinline__ float4 ld4_guard(const float* base, int n, int limit) {
+  if (base == nullptr) return make_float4(0.f, 0.f, 0.f, 0.f);
   if (n + 3 < limit) return __ldg(reinterpret_cast<const float4*>(base + n));
   float4 r;
-  r.x = n + 0 < limit ? __ldg(base + n + 0) : fill;
-  r.y = n + 1 < limit ? __ldg(base + n + 1) : fill;
-  r.z = n + 2 < limit ? __ldg(base + n + 2) : fill;
-  r.w = n + 3 < limit ? __ldg(base + n + 3) : fill;
+  r.x = n + 0 < limit ? __ldg(base + n + 0) : 0.f;
+  r.y = n + 1 < limit ? __ldg(base + n + 1) : 0.f;
+  r.z = n + 2 < limit ? __ldg(base + n + 2) : 0.f;
+  r.w = n + 3 < limit ? __ldg(base + n + 3) : 0.f;
   return r;
 }
 
-// z for 32 consecutive accumulator columns starting at global column n0 (s_w / bias index).
-__device__ __forceinline__ void dequant32(const uint32_t (&acc)[32], float sx, const float* s_w, const float* bias,
-                                          int n0, int N, float (&z)[32]) {
+// The same with scales and biases read from global memory (warp-uniform addresses, served by L1).
+template <bool SMALL>
+__device__ __forceinline__ void dequant32_gmem(const uint32_t (&acc)[32], float sx, const float* s_w, const float* bias, int n0,
+                                               int limit, float (&z)[32]) {
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    const float4 w = ld4_guard(s_w, n0 + 4 * j, N, 0.0f);
-    const float4 b = ld4_guard(bias, n0 + 4 * j, N, 0.0f);
-    z[4 * j + 0] = __fmaf_rn(__fmul_rn(__int2float_rn((int)acc[4 * j + 0]), sx), w.x, b.x);
-    z[4 * j + 1] = __fmaf_rn(__fmul_rn(__int2float_rn((int)acc[4 * j + 1]), sx), w.y, b.y);
-    z[4 * j + 2] = __fmaf_rn(__fmul_rn(__int2float_rn((int)acc[4 * j + 2]), sx), w.z, b.z);
-    z[4 * j + 3] = __fmaf_rn(__fmul_rn(__int2float_rn((int)acc[4 * j + 3]), sx), w.w, b.w);
+    const float4 w = ld4_guard(s_w, n0 + 4 * j, limit);
+    const float4 b = ld4_guard(bias, n0 + 4 * j, limit);
+    z[4 * j + 0] = __fmaf_rn(__fmul_rn(acc_to_float<SMALL>(acc[4 * j + 0]), sx), w.x, b.x);
+    z[4 * j + 1] = __fmaf_rn(__fmul_rn(acc_to_float<SMALL>(acc[4 * j + 1]), sx), w.y, b.y);
+    z[4 * j + 2] = __fmaf_rn(__fmul_rn(acc_to_float<SMALL>(acc[4 * j + 2]), sx), w.z, b.z);
+    z[4 * j + 3] = __fmaf_rn(__fmul_rn(acc_to_float<SMALL>(acc[4 * j + 3]), sx), w.w, b.w);
   }
 }
 
 // ------------------------------------------------------------------------------------------------
 // The kernel
 
-template <int BN>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+template <int BN, int STAGES, int EW, bool SMALL, bool DEBUG>
+__global__ void __launch_bounds__(32 * (2 + EW), 1)
 qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                const __grid_constant__ CUtensorMap tm_y, const GemmParams p) {
-  using Cfg = GemmCfg<BN>;
-  constexpr int STAGES = Cfg::kStages;
+                const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_r, const GemmParams p) {
+  using Cfg = GemmCfg<BN, STAGES, EW>;
   constexpr int HALF = BN / 2;
+  constexpr int SBUFS = kStageBufsPerWarp;
 
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full_bar[STAGES];
   __shared__ uint64_t empty_bar[STAGES];
   __shared__ uint64_t tmem_full_bar[2];
   __shared__ uint64_t tmem_empty_bar[2];
+  __shared__ uint64_t res_bar[EW][SBUFS];  // residual tile landed in a warp's staging buffer
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
@@ -236,6 +295,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   const uint32_t smem_a = smem_base;
   const uint32_t smem_b = smem_base + STAGES * Cfg::kABytes;
   const uint32_t smem_epi = smem_b + STAGES * Cfg::kBBytes;
+  const uint32_t smem_scale = smem_epi + Cfg::kEpiBytes;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -248,14 +308,17 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     tma_prefetch_desc(&tm_a);
     tma_prefetch_desc(&tm_b);
     tma_prefetch_desc(&tm_y);
+    if (p.residual != nullptr) tma_prefetch_desc(&tm_r);
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&full_bar[s]), 1);
       mbar_init(smem_u32(&empty_bar[s]), 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&tmem_full_bar[b]), 1);
-      mbar_init(smem_u32(&tmem_empty_bar[b]), kEpiWarps);
+      mbar_init(smem_u32(&tmem_empty_bar[b]), EW);
     }
+    for (int w = 0; w < EW; ++w)
+      for (int b = 0; b < SBUFS; ++b) mbar_init(smem_u32(&res_bar[w][b]), 1);
     fence_barrier_init();
     fence_proxy_async_smem();
   }
@@ -319,83 +382,157 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   } else {
     // ------------------------------------------------------------------ epilogue warps
     const int ew = warp - 2;
-    const int quad = warp & 3;            // TMEM lane quadrant this warp may read
-    const int chalf = ew >> 2;            // which half of the tile's output columns
-    const uint32_t my_stage = smem_epi + ew * kStageBufsPerWarp * kStageBufBytes;
-    const int out_cols_tile = glu ? HALF : BN;       // output columns per tile
-    const int chunks = out_cols_tile / 32 / 2;       // 32-column chunks per epilogue warp
+    const int quad = warp & 3;  // TMEM lane quadrant this warp may read
+    const int chalf = ew >> 2;  // which half of the tile's output columns (always 0 with four warps)
+    const uint32_t my_stage = smem_epi + ew * SBUFS * kStageBufBytes;
+    const uint32_t my_sw = smem_scale + ew * kScaleSlabFloats * 4;   // s_w slices of this warp's chunks
+    const uint32_t my_bias = my_sw + (kScaleSlabFloats / 2) * 4;     // bias slices
+    const int out_cols_tile = glu ? HALF : BN;      // output columns per tile
+    const int chunks = out_cols_tile / 32 / (EW / 4);  // 32-column chunks per epilogue warp and tile
+    const bool has_res = p.residual != nullptr;
+    const int n_value_limit = glu ? p.N / 2 : p.N;
     uint32_t tcount = 0, store_count = 0;
+
+    // residual prefetch for the very first chunk of this warp
+    if (has_res && lane == 0 && (int)blockIdx.x < total_tiles) {
+      const int tm0 = blockIdx.x / p.tiles_n, tn0 = blockIdx.x - tm0 * p.tiles_n;
+      const int oc0 = tn0 * out_cols_tile + chalf * chunks * 32, r0 = tm0 * kBM + quad * 32;
+      const uint32_t bar = smem_u32(&res_bar[ew][0]);
+      mbar_arrive_expect_tx(bar, kStageBufBytes);
+      tma_load_2d(my_stage, &tm_r, oc0 < p.n_out ? oc0 : 0, r0 < p.M ? r0 : 0, bar);
+    }
+
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tcount) {
       const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
       const uint32_t buf = tcount & 1, aph = (tcount >> 1) & 1;
-      if (!mbar_wait(smem_u32(&tmem_full_bar[buf]), aph, &abort_flag, t_start)) break;
-      tc_fence_after();
+      const int out0 = tn * out_cols_tile;  // first output column of the tile
       const int m = tm * kBM + quad * 32 + lane;
       const bool row_ok = m < p.M;
+
+      // this warp's s_w / bias slices for the tile -> shared memory (before the accumulator is ready)
+      __syncwarp();
+      for (int c = 0; Cfg::kScaleSlab && c < chunks; ++c) {
+        const int col = (chalf * chunks + c) * 32;
+        const int nv = (glu ? out0 : tn * BN) + col + lane;  // value channel of this lane
+        const uint32_t off = (uint32_t)((glu ? 2 * c : c) * 32 + lane) * 4;
+        float wv = 0.0f, bv = 0.0f;
+        if (nv < n_value_limit) {
+          wv = __ldg(p.s_w + nv);
+          if (p.bias != nullptr) bv = __ldg(p.bias + nv);
+        }
+        asm volatile("st.shared.f32 [%0], %1;" ::"r"(my_sw + off), "f"(wv) : "memory");
+        asm volatile("st.shared.f32 [%0], %1;" ::"r"(my_bias + off), "f"(bv) : "memory");
+        if (glu) {
+          const int ng = p.N / 2 + out0 + col + lane;  // gate channel
+          float wg = 0.0f, bg = 0.0f;
+          if (ng < p.N) {
+            wg = __ldg(p.s_w + ng);
+            if (p.bias != nullptr) bg = __ldg(p.bias + ng);
+          }
+          asm volatile("st.shared.f32 [%0], %1;" ::"r"(my_sw + off + 128), "f"(wg) : "memory");
+          asm volatile("st.shared.f32 [%0], %1;" ::"r"(my_bias + off + 128), "f"(bg) : "memory");
+        }
+      }
       const float sx = (p.s_x_kind == AQT_SCALE_ROW) ? (row_ok ? __ldg(p.s_x + m) : 0.0f) : __ldg(p.s_x);
+      __syncwarp();
+
+      if (!mbar_wait(smem_u32(&tmem_full_bar[buf]), aph, &abort_flag, t_start)) break;
+      tc_fence_after();
       const uint32_t lane_addr = tmem_base + buf * BN + ((uint32_t)(quad * 32) << 16);
-      const int out0 = tn * out_cols_tile;  // first output column of the tile
+      bool ok = true;
 
       for (int c = 0; c < chunks; ++c) {
         const int col = (chalf * chunks + c) * 32;  // column offset inside the tile's output
+        const int oc = out0 + col;                  // first global output column of this chunk
+        const uint32_t sb = store_count % SBUFS;
+        const uint32_t sbuf = my_stage + sb * kStageBufBytes;
         float a[32];
         uint32_t acc[32];
         if (!glu) {
-          const int n0 = tn * BN + col;
           tmem_ld_32x32(lane_addr + col, acc);
           tmem_ld_wait();
-          if (p.acc_debug != nullptr && row_ok) {
+          if (DEBUG) {
+            if (p.acc_debug != nullptr && row_ok) {
+              const int n0 = tn * BN + col;
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (n0 + j < p.N) p.acc_debug[(int64_t)m * p.N + n0 + j] = (int32_t)acc[j];
+              for (int j = 0; j < 32; ++j)
+                if (n0 + j < p.N) p.acc_debug[(int64_t)m * p.N + n0 + j] = (int32_t)acc[j];
+            }
           }
-          dequant32(acc, sx, p.s_w, p.bias, n0, p.N, a);
+          if (Cfg::kScaleSlab) dequant32<SMALL>(acc, sx, my_sw + c * 128, my_bias + c * 128, a);
+          else dequant32_gmem<SMALL>(acc, sx, p.s_w, p.bias, tn * BN + col, p.N, a);
           if (p.act == AQT_ACT_SWISH) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) a[j] = a[j] * sigmoid_f(a[j]);
           }
         } else {
-          const int nv = out0 + col;            // value channel
-          const int ng = p.N / 2 + out0 + col;  // gate channel
           float g[32];
           tmem_ld_32x32(lane_addr + col, acc);
           tmem_ld_wait();
-          if (p.acc_debug != nullptr && row_ok) {
+          if (DEBUG) {
+            if (p.acc_debug != nullptr && row_ok) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (nv + j < p.N / 2) p.acc_debug[(int64_t)m * p.N + nv + j] = (int32_t)acc[j];
+              for (int j = 0; j < 32; ++j)
+                if (oc + j < p.N / 2) p.acc_debug[(int64_t)m * p.N + oc + j] = (int32_t)acc[j];
+            }
           }
-          dequant32(acc, sx, p.s_w, p.bias, nv, p.N / 2, a);
+          if (Cfg::kScaleSlab) dequant32<SMALL>(acc, sx, my_sw + c * 256, my_bias + c * 256, a);
+          else dequant32_gmem<SMALL>(acc, sx, p.s_w, p.bias, oc, p.N / 2, a);
           tmem_ld_32x32(lane_addr + HALF + col, acc);
           tmem_ld_wait();
-          if (p.acc_debug != nullptr && row_ok) {
+          if (DEBUG) {
+            if (p.acc_debug != nullptr && row_ok) {
+              const int ng = p.N / 2 + oc;
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (ng + j < p.N) p.acc_debug[(int64_t)m * p.N + ng + j] = (int32_t)acc[j];
+              for (int j = 0; j < 32; ++j)
+                if (ng + j < p.N) p.acc_debug[(int64_t)m * p.N + ng + j] = (int32_t)acc[j];
+            }
           }
-          dequant32(acc, sx, p.s_w, p.bias, ng, p.N, g);
+          if (Cfg::kScaleSlab) dequant32<SMALL>(acc, sx, my_sw + c * 256 + 128, my_bias + c * 256 + 128, g);
+          else dequant32_gmem<SMALL>(acc, sx, p.s_w, p.bias, p.N / 2 + oc, p.N, g);
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
             a[j] = a[j] * sigmoid_f(g[j]);
             if (p.act == AQT_ACT_GLU_SWISH) a[j] = a[j] * sigmoid_f(a[j]);
           }
         }
-        const int oc = out0 + col;  // first global output column of this chunk
-        if (p.residual != nullptr && row_ok) {
-          const float* rrow = p.residual + (int64_t)m * p.ldr;
+
+        if (has_res) {
+          // Buffers alternate: the residual of this chunk was requested one chunk ago into `sb`.
+          // Request the next chunk's residual into the other buffer once the store that last
+          // used it has been read out, then wait for this chunk's tile.
+          if (lane == 0) {
+            tma_store_wait_read<0>();
+            // next chunk of this warp: next in this tile, or the first of its next tile
+            int ntile = tile, nc = c + 1;
+            if (nc == chunks) { nc = 0; ntile = tile + gridDim.x; }
+            if (ntile < total_tiles) {
+              const int ntm = ntile / p.tiles_n, ntn = ntile - ntm * p.tiles_n;
+              const int noc = ntn * out_cols_tile + (chalf * chunks + nc) * 32, nr = ntm * kBM + quad * 32;
+              const uint32_t nb = (store_count + 1) % SBUFS;
+              const uint32_t bar = smem_u32(&res_bar[ew][nb]);
+              mbar_arrive_expect_tx(bar, kStageBufBytes);
+              // a box that would start outside the tensor is redirected to its origin (never read)
+              tma_load_2d(my_stage + nb * kStageBufBytes, &tm_r, noc < p.n_out ? noc : 0, nr < p.M ? nr : 0, bar);
+            }
+          }
+          __syncwarp();
+          if (!mbar_wait(smem_u32(&res_bar[ew][sb]), (store_count / SBUFS) & 1, &abort_flag, t_start)) { ok = false; break; }
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
-            const float4 r = ld4_guard(rrow, oc + 4 * j, p.n_out, 0.0f);
-            a[4 * j + 0] = __fmaf_rn(p.residual_scale, a[4 * j + 0], r.x);
-            a[4 * j + 1] = __fmaf_rn(p.residual_scale, a[4 * j + 1], r.y);
-            a[4 * j + 2] = __fmaf_rn(p.residual_scale, a[4 * j + 2], r.z);
-            a[4 * j + 3] = __fmaf_rn(p.residual_scale, a[4 * j + 3], r.w);
+            const uint32_t src = sbuf + lane * 128 + ((j ^ (lane & 7)) << 4);
+            float r0, r1, r2, r3;
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r0), "=f"(r1), "=f"(r2), "=f"(r3) : "r"(src) : "memory");
+            a[4 * j + 0] = __fmaf_rn(p.residual_scale, a[4 * j + 0], r0);
+            a[4 * j + 1] = __fmaf_rn(p.residual_scale, a[4 * j + 1], r1);
+            a[4 * j + 2] = __fmaf_rn(p.residual_scale, a[4 * j + 2], r2);
+            a[4 * j + 3] = __fmaf_rn(p.residual_scale, a[4 * j + 3], r3);
           }
+        } else {
+          // staging buffer free once the bulk store that last used it has been read out
+          if (lane == 0) tma_store_wait_read<SBUFS - 1>();
+          __syncwarp();
         }
-        // staging buffer free once the bulk store that last used it has read it
-        const uint32_t sbuf = my_stage + (store_count % kStageBufsPerWarp) * kStageBufBytes;
-        if (lane == 0) tma_store_wait_read<kStageBufsPerWarp - 1>();
-        __syncwarp();
         // row `lane` of the 32 x 32 box; 16-byte chunk j sits at (j ^ (row & 7)) under the 128-byte swizzle
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -413,6 +550,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         }
         ++store_count;
       }
+      if (!ok) break;
       // this warp has read its part of the accumulator buffer
       tc_fence_before();
       __syncwarp();
@@ -458,9 +596,9 @@ static EncodeTiledFn get_encode_tiled() {
 }
 
 // 2-D row-major tensor [rows, cols] with `pitch_bytes` between rows; box [box_rows, box_cols];
-// 128-byte swizzle (box_cols * elem_bytes must be 128).
-static int make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const void* base, uint64_t rows,
-                       uint64_t cols, uint64_t pitch_bytes, uint32_t box_rows, uint32_t box_cols) {
+// 128-byte swizzle (box_cols * element size must be 128 bytes).
+static int make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, const void* base, uint64_t rows, uint64_t cols,
+                       uint64_t pitch_bytes, uint32_t box_rows, uint32_t box_cols) {
   EncodeTiledFn enc = get_encode_tiled();
   if (enc == nullptr) {
     if (debug_enabled()) fprintf(stderr, "[aqt] driver entry point for tensor map encoding not found\n");
@@ -470,7 +608,6 @@ static int make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes,
   cuuint64_t strides[1] = {pitch_bytes};
   cuuint32_t box[2] = {box_cols, box_rows};
   cuuint32_t estr[2] = {1, 1};
-  (void)elem_bytes;
   CUresult r = enc(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS && debug_enabled())
@@ -496,7 +633,7 @@ static int pick_bn(int64_t M, int64_t N, bool glu, int sms) {
   const int cands[3] = {256, 128, 64};
   for (int i = 0; i < 3; ++i) {
     const int bn = cands[i];
-    if (glu && bn == 64) continue;  // GLU output box needs at least 32 columns per half-tile warp pair
+    if (glu && bn == 64) continue;  // a GLU tile needs 32 value + 32 gate columns per epilogue warp pair
     const int64_t tiles = tiles_m * ceil_div(N, bn);
     const int64_t rounds = ceil_div(tiles, sms);
     // per-tile cost: proportional to BN, plus a fixed per-tile overhead worth ~24 columns
@@ -509,50 +646,65 @@ static int pick_bn(int64_t M, int64_t N, bool glu, int sms) {
   return best_bn;
 }
 
-template <int BN>
-static int launch_qgemm_bn(const int8_t* a, const int8_t* b, float* y, int64_t ldy, const GemmParams& p0, cudaStream_t st) {
-  using Cfg = GemmCfg<BN>;
+template <int BN, int STAGES, int EW, bool SMALL, bool DEBUG>
+static int launch_qgemm_inst(const int8_t* a, const int8_t* b, float* y, int64_t ldy, const GemmParams& p0, cudaStream_t st) {
+  using Cfg = GemmCfg<BN, STAGES, EW>;
   GemmParams p = p0;
   p.tiles_m = (int)ceil_div(p.M, kBM);
   p.tiles_n = (int)ceil_div(p.N, BN);
   p.k_blocks = (int)ceil_div(p.K, kBK);
-  CUtensorMap tm_a, tm_b, tm_y;
-  int rc = make_map_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a, (uint64_t)p.M, (uint64_t)p.K, (uint64_t)p.K, kBM, kBK);
+  CUtensorMap tm_a, tm_b, tm_y, tm_r;
+  int rc = make_map_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, a, (uint64_t)p.M, (uint64_t)p.K, (uint64_t)p.K, kBM, kBK);
   if (rc != AQT_OK) return rc;
-  rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, b, (uint64_t)p.N, (uint64_t)p.K, (uint64_t)p.K, BN / 2, kBK);
+  rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, b, (uint64_t)p.N, (uint64_t)p.K, (uint64_t)p.K, BN / 2, kBK);
   if (rc != AQT_OK) return rc;
-  rc = make_map_2d(&tm_y, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, y, (uint64_t)p.M, (uint64_t)p.n_out, (uint64_t)ldy * 4,
-                   kStoreBoxRows, kStoreBoxCols);
+  rc = make_map_2d(&tm_y, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, y, (uint64_t)p.M, (uint64_t)p.n_out, (uint64_t)ldy * 4, kStoreBoxRows,
+                   kStoreBoxCols);
   if (rc != AQT_OK) return rc;
+  if (p.residual != nullptr) {
+    rc = make_map_2d(&tm_r, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, p.residual, (uint64_t)p.M, (uint64_t)p.n_out, (uint64_t)p.ldr * 4,
+                     kStoreBoxRows, kStoreBoxCols);
+    if (rc != AQT_OK) return rc;
+  } else {
+    tm_r = tm_y;  // never dereferenced
+  }
+  auto kernel = qgemm_i8_kernel<BN, STAGES, EW, SMALL, DEBUG>;
   static bool attr_set = false;
   if (!attr_set) {
-    if (debug_enabled()) {
-      cudaFuncAttributes fa;
-      int dev = 0, optin = 0;
-      cudaGetDevice(&dev);
-      cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-      cudaError_t e = cudaFuncGetAttributes(&fa, qgemm_i8_kernel<BN>);
-      fprintf(stderr, "[aqt] qgemm<%d>: get-attr %s static smem %zu regs %d max dyn %d; device opt-in max %d; asking %d\n", BN,
-              cudaGetErrorString(e), fa.sharedSizeBytes, fa.numRegs, fa.maxDynamicSharedSizeBytes, optin, Cfg::kSmemBytes);
-    }
-    AQT_RETURN_IF_CUDA(cudaFuncSetAttribute(qgemm_i8_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
+    AQT_RETURN_IF_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
     attr_set = true;
   }
   const int sms = sm_count();
   if (sms <= 0) return AQT_ERR_CUDA;
   const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
   const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-  qgemm_i8_kernel<BN><<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tm_a, tm_b, tm_y, p);
+  kernel<<<grid, Cfg::kThreads, Cfg::kSmemBytes, st>>>(tm_a, tm_b, tm_y, tm_r, p);
   return AQT_LAUNCH_STATUS();
+}
+
+template <int BN, int STAGES, int EW>
+static int launch_qgemm_cfg(const int8_t* a, const int8_t* b, float* y, int64_t ldy, const GemmParams& p, cudaStream_t st) {
+  if (p.acc_debug != nullptr) return launch_qgemm_inst<BN, STAGES, EW, false, true>(a, b, y, ldy, p, st);
+  if (p.small_acc) return launch_qgemm_inst<BN, STAGES, EW, true, false>(a, b, y, ldy, p, st);
+  return launch_qgemm_inst<BN, STAGES, EW, false, false>(a, b, y, ldy, p, st);
 }
 
 // a: int8 [M, K] codes; b: int8 [N, K] codes (both dense, 16-byte aligned, K % 16 == 0).
 static int launch_qgemm(const int8_t* a, const int8_t* b, float* y, int64_t ldy, const GemmParams& p, cudaStream_t st) {
   const bool glu = (p.act == AQT_ACT_GLU) || (p.act == AQT_ACT_GLU_SWISH);
-  const int bn = pick_bn(p.M, p.N, glu, sm_count() > 0 ? sm_count() : 148);
-  if (bn == 256) return launch_qgemm_bn<256>(a, b, y, ldy, p, st);
-  if (bn == 128) return launch_qgemm_bn<128>(a, b, y, ldy, p, st);
-  return launch_qgemm_bn<64>(a, b, y, ldy, p, st);
+  int bn = pick_bn(p.M, p.N, glu, sm_count() > 0 ? sm_count() : 148);
+  // tuning aid: AQT_BN=64|128|256 in the environment overrides the tile-width heuristic
+  static const char* force = getenv("AQT_BN");
+  if (force != nullptr) {
+    const int v = atoi(force);
+    if ((v == 64 && !glu) || v == 128 || v == 256) bn = v;
+  }
+  // Deep K: operand loads bound the tile, so the ring gets the shared memory and four warps run
+  // the (short) epilogue.  Shallow K: the epilogue bounds the tile and gets eight warps.
+  const bool deep_k = p.K >= 2048 && !glu;
+  if (bn == 256) return deep_k ? launch_qgemm_cfg<256, 4, 4>(a, b, y, ldy, p, st) : launch_qgemm_cfg<256, 3, 8>(a, b, y, ldy, p, st);
+  if (bn == 128) return deep_k ? launch_qgemm_cfg<128, 6, 4>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 4, 8>(a, b, y, ldy, p, st);
+  return deep_k ? launch_qgemm_cfg<64, 8, 4>(a, b, y, ldy, p, st) : launch_qgemm_cfg<64, 5, 8>(a, b, y, ldy, p, st);
 }
 
 }  // namespace aqt
