@@ -69,8 +69,8 @@ int qmatmul_i8a(const int8_t* a_codes, const float* s_x, int s_x_kind, const voi
   p.K = (int)K;
   p.n_out = is_glu(act) ? (int)(N / 2) : (int)N;
   p.tiles_m = p.tiles_n = p.k_blocks = 0;
-  // |acc| <= K * qmax_a * qmax_w (codes never reach -qmax - 1, Section 2.2's symmetric range)
-  p.small_acc = (K * (int64_t)qmax_of(bits_a) * qmax_of(bits_w) < (1ll << 22)) ? 1 : 0;
+  // |acc| <= K * 2^(bits_a - 1) * 2^(bits_w - 1) for any codes the containers can hold
+  p.small_acc = (K * (int64_t)(qmax_of(bits_a) + 1) * (qmax_of(bits_w) + 1) <= (1ll << 22)) ? 1 : 0;
   return launch_qgemm(a_codes, b_codes, y, ldy, p, st);
 }
 
