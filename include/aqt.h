@@ -150,6 +150,36 @@ int aqt_linear_fwd_host(const float* x, int x_on_host, const void* wq, const flo
                         int64_t M, int64_t N, int64_t K, int bits_a, int bits_w, int a_scale_kind, int rounding,
                         int act, float* y, int y_on_host, void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * aqt_qmatmul_w4_noalloc -- aqt_qmatmul for int8 activations and 4-bit weights that needs no
+ * workspace from the caller.  (The paper has no counterpart; this is a packaging variant of the
+ * call above.)
+ *
+ * Who it is for: callers that cannot obtain device scratch memory at all -- code running where
+ * cudaMalloc is forbidden or unavailable (inside a stream capture, in a plugin whose host owns
+ * every allocation, under a fixed memory budget with no allocator hook).  The sign-extended copy
+ * of the weights, which aqt_qmatmul places in `workspace`, is placed here in an array that is
+ * part of the library image itself: AQT_NOALLOC_MAX_WEIGHT_BYTES bytes of device memory that
+ * every GPU holding the library keeps until the process exits.
+ *
+ * Arguments, layouts, limits and results are those of aqt_qmatmul with bits_a = 8, bits_w = 4,
+ * acc_debug = NULL and no workspace.  Additional rules:
+ *  - N * K must not exceed AQT_NOALLOC_MAX_WEIGHT_BYTES; larger weights return
+ *    AQT_ERR_UNSUPPORTED and nothing is enqueued.
+ *  - The first call on each device looks up the array's device address (one runtime query, no
+ *    allocation) with that device current; make that first call outside any stream capture.
+ *  - The call allocates nothing and calls no allocating routine.
+ *  - All calls on a device share the one array, and it keeps the previous call's bytes.  Each
+ *    call rewrites the N * K bytes it uses before reading them, so nothing needs clearing; but two
+ *    calls that overlap on the GPU (different streams, no ordering between them) race on it and
+ *    produce garbage.  Order them on one stream or with events.
+ */
+#define AQT_NOALLOC_MAX_WEIGHT_BYTES (4u << 20)
+int aqt_qmatmul_w4_noalloc(const int8_t* xq, const float* s_x, int s_x_kind, const uint8_t* wq_packed,
+                           const float* s_w, const float* bias, const float* residual, int64_t ldr,
+                           float residual_scale, int64_t M, int64_t N, int64_t K, int act, float* y,
+                           int64_t ldy, void* stream);
+
 /* Scratch bytes needed by `op` (AQT_OP_*) at these sizes; 0 if none.  Host-only, no CUDA call. */
 size_t aqt_workspace_bytes(int op, int64_t M, int64_t N, int64_t K, int bits_a, int bits_w);
 

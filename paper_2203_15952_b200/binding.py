@@ -23,7 +23,8 @@ ACT_NONE, ACT_SWISH, ACT_GLU, ACT_GLU_SWISH = 0, 1, 2, 3
 OP_QMATMUL, OP_LINEAR_FWD = 1, 2
 
 EXPORTS = ("aqt_version", "aqt_status_string", "aqt_quantize", "aqt_pack_int4", "aqt_unpack_int4", "aqt_qmatmul",
-           "aqt_linear_fwd", "aqt_linear_fwd_host", "aqt_workspace_bytes", "aqt_device_status")
+           "aqt_linear_fwd", "aqt_linear_fwd_host", "aqt_workspace_bytes", "aqt_device_status", "aqt_qmatmul_w4_noalloc")
+NOALLOC_MAX_WEIGHT_BYTES = 4 << 20
 
 
 class AqtError(RuntimeError):
@@ -190,6 +191,22 @@ def aqt_qmatmul(xq: torch.Tensor, s_x: torch.Tensor, wq: torch.Tensor, s_w: torc
         _i64(residual.stride(0) if residual is not None else 0), ctypes.c_float(residual_scale), _i64(M), _i64(N), _i64(K),
         int(bits_a), int(bits_w), int(act), _ptr(y), _i64(y.stride(0)), _ptr(acc_debug), _ptr(workspace),
         ctypes.c_size_t(0 if workspace is None else workspace.numel()), _stream(stream)))
+    return y
+
+
+def aqt_qmatmul_w4_noalloc(xq: torch.Tensor, s_x: torch.Tensor, wq_packed: torch.Tensor, s_w: torch.Tensor,
+                           bias: Optional[torch.Tensor] = None, residual: Optional[torch.Tensor] = None,
+                           residual_scale: float = 1.0, *, K: int, act: int = ACT_NONE, s_x_kind: int = SCALE_ROW,
+                           y: torch.Tensor, stream=None) -> torch.Tensor:
+    """aqt_qmatmul for int8 activations and packed 4-bit weights with no workspace: for callers that
+    cannot allocate device memory.  The scratch is a fixed array inside the library (N*K must not
+    exceed NOALLOC_MAX_WEIGHT_BYTES); calls on one device share it, so calls that overlap on the
+    GPU race.  The output tensor `y` must be supplied by the caller: this wrapper allocates nothing."""
+    M, N = xq.shape[0], wq_packed.shape[0]
+    _check("aqt_qmatmul_w4_noalloc", lib().aqt_qmatmul_w4_noalloc(
+        _ptr(xq), _ptr(s_x), int(s_x_kind), _ptr(wq_packed), _ptr(s_w), _ptr(bias), _ptr(residual),
+        _i64(residual.stride(0) if residual is not None else 0), ctypes.c_float(residual_scale), _i64(M), _i64(N), _i64(K),
+        int(act), _ptr(y), _i64(y.stride(0)), _stream(stream)))
     return y
 
 

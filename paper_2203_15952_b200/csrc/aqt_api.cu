@@ -238,6 +238,59 @@ int aqt_linear_fwd_host(const float* x, int x_on_host, const void* wq, const flo
   return AQT_OK;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Allocation-free variant: the scratch lives in the library image.
+
+// Sign-extended weight codes of the call in flight.  This name is only a host-side handle in
+// host code; its device address comes from cudaGetSymbolAddress (noalloc_scratch_address).
+static __device__ __align__(256) uint8_t g_noalloc_weight_scratch[AQT_NOALLOC_MAX_WEIGHT_BYTES];
+
+// Device address of the scratch array on the current device, looked up once per device.
+static int noalloc_scratch_address(uint8_t** out) {
+  constexpr int kMaxDevices = 64;
+  static uint8_t* cached[kMaxDevices] = {nullptr};
+  int dev = 0;
+  AQT_RETURN_IF_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return AQT_ERR_UNSUPPORTED;
+  if (cached[dev] == nullptr) {
+    void* ptr = nullptr;
+    AQT_RETURN_IF_CUDA(cudaGetSymbolAddress(&ptr, g_noalloc_weight_scratch));
+    if (ptr == nullptr) return AQT_ERR_CUDA;
+    cached[dev] = reinterpret_cast<uint8_t*>(ptr);
+  }
+  *out = cached[dev];
+  return AQT_OK;
+}
+
+int aqt_qmatmul_w4_noalloc(const int8_t* xq, const float* s_x, int s_x_kind, const uint8_t* wq_packed, const float* s_w,
+                           const float* bias, const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N,
+                           int64_t K, int act, float* y, int64_t ldy, void* stream) {
+  int rc = validate_matmul_shape(M, N, K, 8, 4, act, s_x_kind);
+  if (rc != AQT_OK) return rc;
+  if (M == 0 || N == 0) return AQT_OK;
+  if ((uint64_t)N * (uint64_t)K > (uint64_t)AQT_NOALLOC_MAX_WEIGHT_BYTES) {
+    if (debug_enabled())
+      fprintf(stderr, "[aqt] aqt_qmatmul_w4_noalloc: N*K = %lld exceeds the built-in scratch of %u bytes\n", (long long)(N * K),
+              AQT_NOALLOC_MAX_WEIGHT_BYTES);
+    return AQT_ERR_UNSUPPORTED;
+  }
+  const int64_t n_out = is_glu(act) ? N / 2 : N;
+  if (xq == nullptr || s_x == nullptr || wq_packed == nullptr || s_w == nullptr || y == nullptr) return AQT_ERR_BADARG;
+  if (ldy < n_out || (residual != nullptr && ldr < n_out)) return AQT_ERR_BADARG;
+  if (!is_aligned(xq, 16) || !is_aligned(wq_packed, 16) || !is_aligned(y, 16) || !is_aligned(s_w, 16) || !is_aligned(s_x, 4) ||
+      (bias != nullptr && !is_aligned(bias, 16)) || (residual != nullptr && !is_aligned(residual, 16)))
+    return AQT_ERR_ALIGN;
+  if (ldy % 4 != 0 || (residual != nullptr && ldr % 4 != 0)) return AQT_ERR_ALIGN;
+  rc = check_device();
+  if (rc != AQT_OK) return rc;
+  uint8_t* scratch = nullptr;
+  rc = noalloc_scratch_address(&scratch);
+  if (rc != AQT_OK) return rc;
+  // qmatmul_i8a unpacks the weights into `scratch` (all N*K bytes it later reads) and runs the GEMM.
+  return qmatmul_i8a(xq, s_x, s_x_kind, wq_packed, s_w, bias, residual, ldr, residual_scale, M, N, K, 8, 4, act, y, ldy, nullptr,
+                     scratch, reinterpret_cast<cudaStream_t>(stream));
+}
+
 int aqt_device_status(void* stream, int* status_out) {
   if (status_out == nullptr) return AQT_ERR_BADARG;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
