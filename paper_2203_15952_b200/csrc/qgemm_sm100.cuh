@@ -8,7 +8,7 @@
 //                 into a ring of shared-memory stages, 128-byte swizzled, K-major
 //   warp 1        MMA issuer: one thread issues four K=32 MMAs per k-block into one of two TMEM
 //                 accumulator buffers and commits the stage back to the producer
-//   warps 2..9    epilogue: TMEM -> registers -> de-quantize / bias / activation / residual ->
+//   warps 2..     epilogue (4, 8 or 16 warps): TMEM -> registers -> de-quantize / bias / activation / residual ->
 //                 swizzled shared staging -> TMA store; overlaps the next tile's MMAs.  The
 //                 residual tile is fetched by TMA into the same staging buffer beforehand.
 // Every wait on an mbarrier is bounded by a wall-clock limit; on expiry the CTA records
@@ -24,17 +24,16 @@ namespace aqt {
 constexpr int kBM = 128;         // tile rows = TMEM lanes
 constexpr int kBK = 128;         // bytes (= int8 elements) of K per pipeline stage: one swizzle row
 constexpr int kMmaK = 32;        // K of one tcgen05.mma kind::i8
-constexpr int kStageBufsPerWarp = 2;  // a warp fills one output staging buffer while the other is being stored
 constexpr int kStoreBoxRows = 32;
 constexpr int kStoreBoxCols = 32;                                  // fp32: 128 bytes = one swizzle row
 constexpr int kStageBufBytes = kStoreBoxRows * kStoreBoxCols * 4;  // 4 KB
-constexpr int kScaleSlabFloats = 2 * 32 * 4;                       // per-warp s_w and bias slices: up to 4 chunks of 32
 constexpr uint64_t kWaitLimitNs = 2000000000ull;                   // 2 s
 
-// BN: tile width.  STAGES: depth of the operand ring.  EW: epilogue warps, 4 (one per TMEM lane
-// quadrant) or 8 (two per quadrant, each taking half of the tile's columns).  Shallow-K shapes are
-// bound by the epilogue and take EW = 8; deep-K shapes are bound by operand loads and give the
-// shared memory of four staging warps to the ring.
+// BN: tile width.  STAGES: depth of the operand ring.  EW: epilogue warps, 4, 8 or 16 (one, two or
+// four per TMEM lane quadrant, each taking an equal share of the tile's columns).  Shallow-K
+// shapes are bound by the epilogue (special-function and issue throughput, long dependent chains)
+// and take 8 or 16 warps; deep-K shapes are bound by operand loads and give the shared memory of
+// the extra staging buffers to the ring.
 template <int BN, int STAGES, int EW>
 struct GemmCfg {
   static constexpr int kThreads = 32 * (2 + EW);
@@ -42,11 +41,15 @@ struct GemmCfg {
   static constexpr int kBBytes = BN * kBK;
   static constexpr int kStages = STAGES;
   static constexpr int kTmemCols = 2 * BN;  // two accumulator buffers; a power of two >= 32
-  static constexpr int kEpiBytes = EW * kStageBufsPerWarp * kStageBufBytes;
-  // With EW == 8 each warp keeps its s_w / bias slices in shared memory; with EW == 4 the scales
-  // are read through L1 instead (the epilogue is a small part of a deep-K tile).
-  static constexpr bool kScaleSlab = (EW == 8);
-  static constexpr int kScaleBytes = kScaleSlab ? EW * kScaleSlabFloats * 4 : 0;
+  // Output staging buffers per warp: two let a warp fill one while the bulk store of the other is
+  // still being read; with sixteen warps each warp stores once per tile and one is enough.
+  static constexpr int kStageBufs = (EW == 16) ? 1 : 2;
+  static constexpr int kEpiBytes = EW * kStageBufs * kStageBufBytes;
+  // With EW >= 8 each warp keeps the s_w / bias slices of its columns in shared memory; with
+  // EW == 4 the scales are read through L1 instead (the epilogue is a small part of a deep-K tile).
+  static constexpr bool kScaleSlab = (EW >= 8);
+  static constexpr int kSlabFloats = BN / (EW / 4);  // per warp and per array (s_w, bias)
+  static constexpr int kScaleBytes = kScaleSlab ? EW * 2 * kSlabFloats * 4 : 0;
   static constexpr int kSmemBytes = STAGES * (kABytes + kBBytes) + kEpiBytes + kScaleBytes + 1024;  // + alignment slack
   static_assert(kSmemBytes + 512 <= 232448, "pipeline + staging must fit the 227 KB a CTA can opt into");
 };
@@ -195,29 +198,25 @@ __host__ __device__ constexpr uint32_t idesc_i8(int bn) {
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
-  asm("ex2.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
 __device__ __forceinline__ float rcp_approx(float x) {
   float y;
-  asm("rcp.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
 
-// sigmoid(z) = 1 / (1 + e^-z).  e^-z = 2^t with t = -z log2(e) formed in two pieces (the rounded
-// product and its exact remainder) so that the exponent's rounding error does not grow with |z|;
-// the special-function unit supplies 2^t and the reciprocal.  Relative error about 4e-7.
-// z is clamped at -87 so that e^-z stays finite (sigmoid is below 2e-38 there).
+// sigmoid(z) = 1 / (1 + e^-z) with e^-z = 2^(-z log2 e): one multiply, the special-function
+// unit's 2^t, one add, its reciprocal.  Five instructions with the caller's final multiply, two of
+// them on the special-function unit, which is the unit that bounds the Swish epilogue.
+// Error: |t| 7e-8 from the rounded product, 2^-22 from 2^t, 2^-23 from the reciprocal; relative to
+// the pre-activation |z| the activation a = z sigmoid(z) is within 3e-7 everywhere (the relative
+// error of a itself passes 1e-6 only below z = -9, where |a| < 1e-3 |z|).  Large |t| saturates
+// cleanly: 2^t = +inf gives sigmoid 0, 2^t = 0 gives sigmoid 1.
 __device__ __forceinline__ float sigmoid_f(float z) {
-  const float kHi = -1.4426950216293335f;     // RN(-log2 e)
-  const float kLo = -1.9259629911266175e-8f;  // -log2 e - kHi
-  const float zc = fmaxf(z, -87.0f);
-  const float t = __fmul_rn(zc, kHi);
-  float r = __fmaf_rn(zc, kHi, -t);
-  r = __fmaf_rn(zc, kLo, r);
-  const float e = ex2_approx(t);
-  const float en = __fmaf_rn(e, r * 0.69314718f, e);  // 2^(t + r) ~ 2^t (1 + r ln 2)
-  return rcp_approx(1.0f + en);
+  const float e = ex2_approx(z * -1.4426950408889634f);
+  return rcp_approx(1.0f + e);
 }
 
 // int32 accumulator -> float, round-to-nearest-even (exact below 2^24).  With SMALL the caller
@@ -280,7 +279,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_r, const GemmParams p) {
   using Cfg = GemmCfg<BN, STAGES, EW>;
   constexpr int HALF = BN / 2;
-  constexpr int SBUFS = kStageBufsPerWarp;
+  constexpr int SBUFS = Cfg::kStageBufs;
 
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full_bar[STAGES];
@@ -383,10 +382,10 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     // ------------------------------------------------------------------ epilogue warps
     const int ew = warp - 2;
     const int quad = warp & 3;  // TMEM lane quadrant this warp may read
-    const int chalf = ew >> 2;  // which half of the tile's output columns (always 0 with four warps)
+    const int chalf = ew >> 2;  // which share of the tile's output columns (0 .. EW/4 - 1)
     const uint32_t my_stage = smem_epi + ew * SBUFS * kStageBufBytes;
-    const uint32_t my_sw = smem_scale + ew * kScaleSlabFloats * 4;   // s_w slices of this warp's chunks
-    const uint32_t my_bias = my_sw + (kScaleSlabFloats / 2) * 4;     // bias slices
+    const uint32_t my_sw = smem_scale + ew * 2 * Cfg::kSlabFloats * 4;  // s_w slices of this warp's chunks
+    const uint32_t my_bias = my_sw + Cfg::kSlabFloats * 4;              // bias slices
     const int out_cols_tile = glu ? HALF : BN;      // output columns per tile
     const int chunks = out_cols_tile / 32 / (EW / 4);  // 32-column chunks per epilogue warp and tile
     const bool has_res = p.residual != nullptr;
@@ -448,9 +447,16 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         const uint32_t sbuf = my_stage + sb * kStageBufBytes;
         float a[32];
         uint32_t acc[32];
+        const bool last_chunk = (c == chunks - 1);
         if (!glu) {
           tmem_ld_32x32(lane_addr + col, acc);
           tmem_ld_wait();
+          if (last_chunk) {
+            // accumulator buffer read out by this warp: hand it back before the arithmetic
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[buf]));
+          }
           if (DEBUG) {
             if (p.acc_debug != nullptr && row_ok) {
               const int n0 = tn * BN + col;
@@ -466,18 +472,8 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             for (int j = 0; j < 32; ++j) a[j] = a[j] * sigmoid_f(a[j]);
           }
         } else {
+          // gates first: g = sigmoid(z_gate); then the values are scaled by it
           float g[32];
-          tmem_ld_32x32(lane_addr + col, acc);
-          tmem_ld_wait();
-          if (DEBUG) {
-            if (p.acc_debug != nullptr && row_ok) {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (oc + j < p.N / 2) p.acc_debug[(int64_t)m * p.N + oc + j] = (int32_t)acc[j];
-            }
-          }
-          if (Cfg::kScaleSlab) dequant32<SMALL>(acc, sx, my_sw + c * 256, my_bias + c * 256, a);
-          else dequant32_gmem<SMALL>(acc, sx, p.s_w, p.bias, oc, p.N / 2, a);
           tmem_ld_32x32(lane_addr + HALF + col, acc);
           tmem_ld_wait();
           if (DEBUG) {
@@ -491,32 +487,52 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           if (Cfg::kScaleSlab) dequant32<SMALL>(acc, sx, my_sw + c * 256 + 128, my_bias + c * 256 + 128, g);
           else dequant32_gmem<SMALL>(acc, sx, p.s_w, p.bias, p.N / 2 + oc, p.N, g);
 #pragma unroll
+          for (int j = 0; j < 32; ++j) g[j] = sigmoid_f(g[j]);
+          tmem_ld_32x32(lane_addr + col, acc);
+          tmem_ld_wait();
+          if (last_chunk) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[buf]));
+          }
+          if (DEBUG) {
+            if (p.acc_debug != nullptr && row_ok) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (oc + j < p.N / 2) p.acc_debug[(int64_t)m * p.N + oc + j] = (int32_t)acc[j];
+            }
+          }
+          if (Cfg::kScaleSlab) dequant32<SMALL>(acc, sx, my_sw + c * 256, my_bias + c * 256, a);
+          else dequant32_gmem<SMALL>(acc, sx, p.s_w, p.bias, oc, p.N / 2, a);
+#pragma unroll
           for (int j = 0; j < 32; ++j) {
-            a[j] = a[j] * sigmoid_f(g[j]);
+            a[j] = a[j] * g[j];
             if (p.act == AQT_ACT_GLU_SWISH) a[j] = a[j] * sigmoid_f(a[j]);
           }
         }
 
         if (has_res) {
-          // Buffers alternate: the residual of this chunk was requested one chunk ago into `sb`.
-          // Request the next chunk's residual into the other buffer once the store that last
-          // used it has been read out, then wait for this chunk's tile.
-          if (lane == 0) {
-            tma_store_wait_read<0>();
-            // next chunk of this warp: next in this tile, or the first of its next tile
-            int ntile = tile, nc = c + 1;
-            if (nc == chunks) { nc = 0; ntile = tile + gridDim.x; }
-            if (ntile < total_tiles) {
-              const int ntm = ntile / p.tiles_n, ntn = ntile - ntm * p.tiles_n;
-              const int noc = ntn * out_cols_tile + (chalf * chunks + nc) * 32, nr = ntm * kBM + quad * 32;
-              const uint32_t nb = (store_count + 1) % SBUFS;
-              const uint32_t bar = smem_u32(&res_bar[ew][nb]);
-              mbar_arrive_expect_tx(bar, kStageBufBytes);
-              // a box that would start outside the tensor is redirected to its origin (never read)
-              tma_load_2d(my_stage + nb * kStageBufBytes, &tm_r, noc < p.n_out ? noc : 0, nr < p.M ? nr : 0, bar);
+          if (SBUFS == 2) {
+            // Buffers alternate: the residual of this chunk was requested one chunk ago into `sb`.
+            // Request the next chunk's residual into the other buffer once the store that last
+            // used it has been read out, then wait for this chunk's tile.
+            if (lane == 0) {
+              tma_store_wait_read<0>();
+              // next chunk of this warp: next in this tile, or the first of its next tile
+              int ntile = tile, nc = c + 1;
+              if (nc == chunks) { nc = 0; ntile = tile + gridDim.x; }
+              if (ntile < total_tiles) {
+                const int ntm = ntile / p.tiles_n, ntn = ntile - ntm * p.tiles_n;
+                const int noc = ntn * out_cols_tile + (chalf * chunks + nc) * 32, nr = ntm * kBM + quad * 32;
+                const uint32_t nb = (store_count + 1) % SBUFS;
+                const uint32_t bar = smem_u32(&res_bar[ew][nb]);
+                mbar_arrive_expect_tx(bar, kStageBufBytes);
+                // a box that would start outside the tensor is redirected to its origin (never read)
+                tma_load_2d(my_stage + nb * kStageBufBytes, &tm_r, noc < p.n_out ? noc : 0, nr < p.M ? nr : 0, bar);
+              }
             }
+            __syncwarp();
           }
-          __syncwarp();
           if (!mbar_wait(smem_u32(&res_bar[ew][sb]), (store_count / SBUFS) & 1, &abort_flag, t_start)) { ok = false; break; }
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
@@ -528,6 +544,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             a[4 * j + 2] = __fmaf_rn(p.residual_scale, a[4 * j + 2], r2);
             a[4 * j + 3] = __fmaf_rn(p.residual_scale, a[4 * j + 3], r3);
           }
+          __syncwarp();  // every lane has read its residual row before the buffer is overwritten
         } else {
           // staging buffer free once the bulk store that last used it has been read out
           if (lane == 0) tma_store_wait_read<SBUFS - 1>();
@@ -547,14 +564,24 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           // boxes that start inside the output are clipped at its edges by the copy engine
           if (oc < p.n_out && tm * kBM + quad * 32 < p.M) tma_store_2d(&tm_y, sbuf, oc, tm * kBM + quad * 32);
           tma_store_commit();
+          if (has_res && SBUFS == 1) {
+            // single buffer: the next chunk's residual can only be requested once this store has
+            // read the buffer out (the warp is otherwise idle until its next chunk)
+            tma_store_wait_read<0>();
+            int ntile = tile, nc = c + 1;
+            if (nc == chunks) { nc = 0; ntile = tile + gridDim.x; }
+            if (ntile < total_tiles) {
+              const int ntm = ntile / p.tiles_n, ntn = ntile - ntm * p.tiles_n;
+              const int noc = ntn * out_cols_tile + (chalf * chunks + nc) * 32, nr = ntm * kBM + quad * 32;
+              const uint32_t bar = smem_u32(&res_bar[ew][0]);
+              mbar_arrive_expect_tx(bar, kStageBufBytes);
+              tma_load_2d(my_stage, &tm_r, noc < p.n_out ? noc : 0, nr < p.M ? nr : 0, bar);
+            }
+          }
         }
         ++store_count;
       }
       if (!ok) break;
-      // this warp has read its part of the accumulator buffer
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[buf]));
     }
     if (lane == 0) tma_store_wait_all();
   }
@@ -676,6 +703,10 @@ static int launch_qgemm_inst(const int8_t* a, const int8_t* b, float* y, int64_t
   }
   const int sms = sm_count();
   if (sms <= 0) return AQT_ERR_CUDA;
+  {
+    const bool glu = (p.act == AQT_ACT_GLU) || (p.act == AQT_ACT_GLU_SWISH);
+    if ((glu ? BN / 2 : BN) / 32 / (EW / 4) < 1) return AQT_ERR_UNSUPPORTED;  // a warp without columns would never release TMEM
+  }
   const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
   const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
   kernel<<<grid, Cfg::kThreads, Cfg::kSmemBytes, st>>>(tm_a, tm_b, tm_y, tm_r, p);
@@ -702,8 +733,11 @@ static int launch_qgemm(const int8_t* a, const int8_t* b, float* y, int64_t ldy,
   // Deep K: operand loads bound the tile, so the ring gets the shared memory and four warps run
   // the (short) epilogue.  Shallow K: the epilogue bounds the tile and gets eight warps.
   const bool deep_k = p.K >= 2048 && !glu;
-  if (bn == 256) return deep_k ? launch_qgemm_cfg<256, 4, 4>(a, b, y, ldy, p, st) : launch_qgemm_cfg<256, 3, 8>(a, b, y, ldy, p, st);
-  if (bn == 128) return deep_k ? launch_qgemm_cfg<128, 6, 4>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 4, 8>(a, b, y, ldy, p, st);
+  if (bn == 256) return deep_k ? launch_qgemm_cfg<256, 4, 4>(a, b, y, ldy, p, st) : launch_qgemm_cfg<256, 3, 16>(a, b, y, ldy, p, st);
+  // every epilogue warp needs at least one 32-column chunk: a GLU tile of width 128 has only
+  // 64 output columns, i.e. two chunks per lane quadrant
+  if (bn == 128 && glu) return launch_qgemm_cfg<128, 4, 8>(a, b, y, ldy, p, st);
+  if (bn == 128) return deep_k ? launch_qgemm_cfg<128, 6, 4>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 4, 16>(a, b, y, ldy, p, st);
   return deep_k ? launch_qgemm_cfg<64, 8, 4>(a, b, y, ldy, p, st) : launch_qgemm_cfg<64, 5, 8>(a, b, y, ldy, p, st);
 }
 
