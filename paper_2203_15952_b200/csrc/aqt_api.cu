@@ -48,11 +48,18 @@ int validate_matmul_shape(int64_t M, int64_t N, int64_t K, int bits_a, int bits_
 int qmatmul_i8a(const int8_t* a_codes, const float* s_x, int s_x_kind, const void* wq, const float* s_w, const float* bias,
                 const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K, int bits_a, int bits_w,
                 int act, float* y, int64_t ldy, int32_t* acc_debug, uint8_t* ws, cudaStream_t st) {
-  const int8_t* b_codes = reinterpret_cast<const int8_t*>(wq);
+  // 4-bit weights: the weight-stationary kernel (K <= 512) sign-extends them itself in shared
+  // memory after TMA staging; deeper K takes a one-off sign-extended copy in the workspace.
+  const void* b_codes = wq;
+  bool b_packed = false;
   if (bits_w == 4) {
-    int rc = launch_unpack_int4(reinterpret_cast<const uint8_t*>(wq), N * K / 2, reinterpret_cast<int8_t*>(ws), st);
-    if (rc != AQT_OK) return rc;
-    b_codes = reinterpret_cast<const int8_t*>(ws);
+    if (qgemm_uses_ws(N, K)) {
+      b_packed = true;
+    } else {
+      int rc = launch_unpack_int4(reinterpret_cast<const uint8_t*>(wq), N * K / 2, reinterpret_cast<int8_t*>(ws), st);
+      if (rc != AQT_OK) return rc;
+      b_codes = ws;
+    }
   }
   GemmParams p;
   p.s_x = s_x;
@@ -71,7 +78,7 @@ int qmatmul_i8a(const int8_t* a_codes, const float* s_x, int s_x_kind, const voi
   p.tiles_m = p.tiles_n = p.k_blocks = 0;
   // |acc| <= K * 2^(bits_a - 1) * 2^(bits_w - 1) for any codes the containers can hold
   p.small_acc = (K * (int64_t)(qmax_of(bits_a) + 1) * (qmax_of(bits_w) + 1) <= (1ll << 22)) ? 1 : 0;
-  return launch_qgemm(a_codes, b_codes, y, ldy, p, st);
+  return launch_qgemm(a_codes, b_codes, b_packed, y, ldy, p, st);
 }
 
 }  // namespace

@@ -18,6 +18,7 @@
 #include <cuda.h>
 
 #include "aqt_common.cuh"
+#include "pack.cuh"
 
 namespace aqt {
 
@@ -34,24 +35,32 @@ constexpr uint64_t kWaitLimitNs = 2000000000ull;                   // 2 s
 // shapes are bound by the epilogue (special-function and issue throughput, long dependent chains)
 // and take 8 or 16 warps; deep-K shapes are bound by operand loads and give the shared memory of
 // the extra staging buffers to the ring.
-template <int BN, int STAGES, int EW>
+// WS ("weight stationary", K <= 512): a CTA keeps one n-tile of the weights resident in shared
+// memory for its whole life and streams only activation k-blocks through the ring, which halves
+// the L2 -> shared-memory traffic and lets the ring hold more than one tile of A.
+constexpr int kWsMaxKBlocks = 4;  // K <= 512
+template <int BN, int STAGES, int EW, bool WS>
 struct GemmCfg {
   static constexpr int kThreads = 32 * (2 + EW);
   static constexpr int kABytes = kBM * kBK;
   static constexpr int kBBytes = BN * kBK;
+  static constexpr int kStageBytes = WS ? kABytes : kABytes + kBBytes;
+  static constexpr int kResidentBytes = WS ? kWsMaxKBlocks * kBBytes : 0;
   static constexpr int kStages = STAGES;
   static constexpr int kTmemCols = 2 * BN;  // two accumulator buffers; a power of two >= 32
   // Output staging buffers per warp: two let a warp fill one while the bulk store of the other is
   // still being read; with sixteen warps each warp stores once per tile and one is enough.
   static constexpr int kStageBufs = (EW == 16) ? 1 : 2;
   static constexpr int kEpiBytes = EW * kStageBufs * kStageBufBytes;
-  // With EW >= 8 each warp keeps the s_w / bias slices of its columns in shared memory; with
-  // EW == 4 the scales are read through L1 instead (the epilogue is a small part of a deep-K tile).
-  static constexpr bool kScaleSlab = (EW >= 8);
-  static constexpr int kSlabFloats = BN / (EW / 4);  // per warp and per array (s_w, bias)
-  static constexpr int kScaleBytes = kScaleSlab ? EW * 2 * kSlabFloats * 4 : 0;
-  static constexpr int kSmemBytes = STAGES * (kABytes + kBBytes) + kEpiBytes + kScaleBytes + 1024;  // + alignment slack
-  static_assert(kSmemBytes + 512 <= 232448, "pipeline + staging must fit the 227 KB a CTA can opt into");
+  // Scales and biases of the tile's columns in shared memory: one slab per CTA when the n-tile is
+  // fixed (WS), one per warp (its own columns) with EW >= 8 otherwise; with EW == 4 they are read
+  // through L1 instead (the epilogue is a small part of a deep-K tile).
+  static constexpr bool kScaleSlab = WS || (EW >= 8);
+  static constexpr int kSlabFloats = WS ? BN : BN / (EW / 4);  // per array (s_w, bias)
+  static constexpr int kScaleBytes = !kScaleSlab ? 0 : (WS ? 2 * BN * 4 : EW * 2 * kSlabFloats * 4);
+  static constexpr int kSmemBytes = STAGES * kStageBytes + kResidentBytes + kEpiBytes + kScaleBytes + 1024;  // + alignment slack
+  static_assert(kSmemBytes + 512 <= 232448, "ring + resident weights + staging must fit the 227 KB a CTA can opt into");
+  static_assert(!WS || kWsMaxKBlocks * BN * 64 <= kEpiBytes, "packed weights are staged in the epilogue buffers");
 };
 
 struct GemmParams {
@@ -273,13 +282,32 @@ __device__ __forceinline__ void dequant32_gmem(const uint32_t (&acc)[32], float 
 // ------------------------------------------------------------------------------------------------
 // The kernel
 
-template <int BN, int STAGES, int EW, bool SMALL, bool DEBUG>
+// i-th tile of this CTA.  Standard order: tiles are numbered n-fastest and dealt round-robin.
+// Weight-stationary order: the CTA owns n-tile (blockIdx % tiles_n) and takes every g-th m-tile,
+// g being the number of CTAs that own the same n-tile.
+template <bool WS>
+__device__ __forceinline__ bool tile_at(const GemmParams& p, int i, int& tm, int& tn) {
+  if (WS) {
+    tn = blockIdx.x % p.tiles_n;
+    const int r = blockIdx.x / p.tiles_n;
+    const int g = ((int)gridDim.x - 1 - tn) / p.tiles_n + 1;
+    tm = r + i * g;
+    return tm < p.tiles_m;
+  }
+  const int tile = blockIdx.x + i * gridDim.x;
+  tm = tile / p.tiles_n;
+  tn = tile - tm * p.tiles_n;
+  return tile < p.tiles_m * p.tiles_n;
+}
+
+template <int BN, int STAGES, int EW, bool WS, bool BPACK, bool SMALL, bool DEBUG>
 __global__ void __launch_bounds__(32 * (2 + EW), 1)
 qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                 const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_r, const GemmParams p) {
-  using Cfg = GemmCfg<BN, STAGES, EW>;
+  using Cfg = GemmCfg<BN, STAGES, EW, WS>;
   constexpr int HALF = BN / 2;
   constexpr int SBUFS = Cfg::kStageBufs;
+  static_assert(!BPACK || WS, "packed weights are unpacked into the resident slab");
 
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full_bar[STAGES];
@@ -287,20 +315,21 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   __shared__ uint64_t tmem_full_bar[2];
   __shared__ uint64_t tmem_empty_bar[2];
   __shared__ uint64_t res_bar[EW][SBUFS];  // residual tile landed in a warp's staging buffer
+  __shared__ uint64_t b_loaded_bar;        // WS: the CTA's weight slab (or its packed form) has landed
+  __shared__ uint64_t b_ready_bar;         // WS + BPACK: every epilogue warp has unpacked its share
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms need 1024-byte alignment
-  const uint32_t smem_a = smem_base;
-  const uint32_t smem_b = smem_base + STAGES * Cfg::kABytes;
-  const uint32_t smem_epi = smem_b + STAGES * Cfg::kBBytes;
+  const uint32_t smem_ring = smem_base;
+  const uint32_t smem_res_b = smem_ring + STAGES * Cfg::kStageBytes;  // WS: resident weights, one 128-byte k-block after another
+  const uint32_t smem_epi = smem_res_b + Cfg::kResidentBytes;
   const uint32_t smem_scale = smem_epi + Cfg::kEpiBytes;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const uint64_t t_start = global_timer_ns();
   const bool glu = (p.act == AQT_ACT_GLU) || (p.act == AQT_ACT_GLU_SWISH);
-  const int total_tiles = p.tiles_m * p.tiles_n;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -318,12 +347,35 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     }
     for (int w = 0; w < EW; ++w)
       for (int b = 0; b < SBUFS; ++b) mbar_init(smem_u32(&res_bar[w][b]), 1);
+    mbar_init(smem_u32(&b_loaded_bar), 1);
+    mbar_init(smem_u32(&b_ready_bar), EW);
     fence_barrier_init();
     fence_proxy_async_smem();
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(&tmem_base_slot), Cfg::kTmemCols);
     tmem_relinquish();
+  }
+  if (WS) {
+    // scales and biases of the CTA's n-tile, once: values first, then (GLU) gates
+    const int tn = blockIdx.x % p.tiles_n;
+    for (int t = threadIdx.x; t < BN; t += blockDim.x) {
+      int n, limit;
+      if (glu) {
+        n = (t < HALF) ? tn * HALF + t : p.N / 2 + tn * HALF + (t - HALF);
+        limit = (t < HALF) ? p.N / 2 : p.N;
+      } else {
+        n = tn * BN + t;
+        limit = p.N;
+      }
+      float wv = 0.0f, bv = 0.0f;
+      if (n < limit) {
+        wv = __ldg(p.s_w + n);
+        if (p.bias != nullptr) bv = __ldg(p.bias + n);
+      }
+      asm volatile("st.shared.f32 [%0], %1;" ::"r"(smem_scale + t * 4), "f"(wv) : "memory");
+      asm volatile("st.shared.f32 [%0], %1;" ::"r"(smem_scale + (BN + t) * 4), "f"(bv) : "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
@@ -335,8 +387,29 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
+      if (WS) {
+        // the CTA's weight slab, once: int8 codes straight into the resident slab, or the packed
+        // nibbles into the (still unused) epilogue staging area for the warps to unpack
+        const int tn = blockIdx.x % p.tiles_n;
+        const int row0 = glu ? tn * HALF : tn * BN;
+        const int row1 = glu ? p.N / 2 + tn * HALF : tn * BN + HALF;
+        const uint32_t bar = smem_u32(&b_loaded_bar);
+        if (BPACK) {
+          mbar_arrive_expect_tx(bar, (uint32_t)p.k_blocks * BN * 64);
+          for (int kb = 0; kb < p.k_blocks; ++kb) {
+            tma_load_2d(smem_epi + kb * BN * 64, &tm_b, kb * 64, row0, bar);
+            tma_load_2d(smem_epi + kb * BN * 64 + HALF * 64, &tm_b, kb * 64, row1, bar);
+          }
+        } else {
+          mbar_arrive_expect_tx(bar, (uint32_t)p.k_blocks * Cfg::kBBytes);
+          for (int kb = 0; kb < p.k_blocks; ++kb) {
+            tma_load_2d(smem_res_b + kb * Cfg::kBBytes, &tm_b, kb * kBK, row0, bar);
+            tma_load_2d(smem_res_b + kb * Cfg::kBBytes + HALF * kBK, &tm_b, kb * kBK, row1, bar);
+          }
+        }
+      }
+      int tm, tn;
+      for (int i = 0; ok && tile_at<WS>(p, i, tm, tn); ++i) {
         // B rows of the two half-tiles: adjacent output channels, or (value, gate) halves for GLU
         const int row0 = glu ? tn * HALF : tn * BN;
         const int row1 = glu ? p.N / 2 + tn * HALF : tn * BN + HALF;
@@ -344,10 +417,13 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
           if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1, &abort_flag, t_start)) { ok = false; break; }
           const uint32_t bar = smem_u32(&full_bar[s]);
-          mbar_arrive_expect_tx(bar, Cfg::kABytes + Cfg::kBBytes);
-          tma_load_2d(smem_a + s * Cfg::kABytes, &tm_a, kb * kBK, tm * kBM, bar);
-          tma_load_2d(smem_b + s * Cfg::kBBytes, &tm_b, kb * kBK, row0, bar);
-          tma_load_2d(smem_b + s * Cfg::kBBytes + HALF * kBK, &tm_b, kb * kBK, row1, bar);
+          const uint32_t stage = smem_ring + s * Cfg::kStageBytes;
+          mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
+          tma_load_2d(stage, &tm_a, kb * kBK, tm * kBM, bar);
+          if (!WS) {
+            tma_load_2d(stage + Cfg::kABytes, &tm_b, kb * kBK, row0, bar);
+            tma_load_2d(stage + Cfg::kABytes + HALF * kBK, &tm_b, kb * kBK, row1, bar);
+          }
         }
       }
     }
@@ -357,7 +433,9 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       constexpr uint32_t idesc = idesc_i8(BN);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+      if (WS) ok = mbar_wait(smem_u32(BPACK ? &b_ready_bar : &b_loaded_bar), 0, &abort_flag, t_start);
+      int tm, tn;
+      for (int i = 0; ok && tile_at<WS>(p, i, tm, tn); ++i, ++tcount) {
         const uint32_t buf = tcount & 1, aph = (tcount >> 1) & 1;
         if (!mbar_wait(smem_u32(&tmem_empty_bar[buf]), aph ^ 1, &abort_flag, t_start)) break;
         tc_fence_after();
@@ -366,8 +444,9 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
           if (!mbar_wait(smem_u32(&full_bar[s]), ph, &abort_flag, t_start)) { ok = false; break; }
           tc_fence_after();
-          const uint64_t a_desc = smem_desc_k_major_sw128(smem_a + s * Cfg::kABytes);
-          const uint64_t b_desc = smem_desc_k_major_sw128(smem_b + s * Cfg::kBBytes);
+          const uint32_t stage = smem_ring + s * Cfg::kStageBytes;
+          const uint64_t a_desc = smem_desc_k_major_sw128(stage);
+          const uint64_t b_desc = smem_desc_k_major_sw128(WS ? smem_res_b + kb * Cfg::kBBytes : stage + Cfg::kABytes);
 #pragma unroll
           for (int kk = 0; kk < kBK / kMmaK; ++kk) {
             // advancing K inside the 128-byte swizzle row: +32 bytes = +2 in the 16-byte address field
@@ -384,52 +463,91 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     const int quad = warp & 3;  // TMEM lane quadrant this warp may read
     const int chalf = ew >> 2;  // which share of the tile's output columns (0 .. EW/4 - 1)
     const uint32_t my_stage = smem_epi + ew * SBUFS * kStageBufBytes;
-    const uint32_t my_sw = smem_scale + ew * 2 * Cfg::kSlabFloats * 4;  // s_w slices of this warp's chunks
-    const uint32_t my_bias = my_sw + Cfg::kSlabFloats * 4;              // bias slices
-    const int out_cols_tile = glu ? HALF : BN;      // output columns per tile
+    const int out_cols_tile = glu ? HALF : BN;         // output columns per tile
     const int chunks = out_cols_tile / 32 / (EW / 4);  // 32-column chunks per epilogue warp and tile
     const bool has_res = p.residual != nullptr;
     const int n_value_limit = glu ? p.N / 2 : p.N;
-    uint32_t tcount = 0, store_count = 0;
+    // where the scales of this warp's chunk c start: per-CTA slab (WS) or per-warp slab
+    const uint32_t slab_sw = WS ? smem_scale + (uint32_t)(chalf * chunks * 32) * 4 : smem_scale + ew * 2 * Cfg::kSlabFloats * 4;
+    const uint32_t slab_bias = WS ? slab_sw + BN * 4 : slab_sw + Cfg::kSlabFloats * 4;
+    const uint32_t slab_chunk_stride = (WS || !glu) ? 128 : 256;  // bytes between consecutive chunks of this warp
+    const uint32_t slab_gate_off = WS ? HALF * 4 : 128;           // gate columns relative to the value columns
+    uint32_t store_count = 0;
+    bool ok = true;
 
+    if (WS && BPACK) {
+      // Sign-extend the CTA's packed weights into the resident slab, in the layout a swizzled
+      // TMA load of int8 codes would have produced: row r of a k-block is 128 bytes, its 16-byte
+      // chunk j sits at position j ^ (r & 7).  Exact (integers), done once per CTA.
+      ok = mbar_wait(smem_u32(&b_loaded_bar), 0, &abort_flag, t_start);
+      if (ok) {
+        const int pieces = p.k_blocks * BN * 4;  // 16 packed bytes -> 32 codes each
+        for (int q = (ew * 32 + lane); q < pieces; q += EW * 32) {
+          const int kb = q / (BN * 4), rem = q - kb * (BN * 4);
+          const int r = rem >> 2, piece = rem & 3;
+          uint32_t w0, w1, w2, w3;
+          asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                       : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3)
+                       : "r"(smem_epi + kb * BN * 64 + r * 64 + piece * 16)
+                       : "memory");
+          uint32_t o[8];
+          unpack_word(w0, o[0], o[1]);
+          unpack_word(w1, o[2], o[3]);
+          unpack_word(w2, o[4], o[5]);
+          unpack_word(w3, o[6], o[7]);
+          const uint32_t row_base = smem_res_b + kb * Cfg::kBBytes + r * 128;
+          const uint32_t d0 = row_base + (((2 * piece) ^ (r & 7)) << 4);
+          const uint32_t d1 = row_base + (((2 * piece + 1) ^ (r & 7)) << 4);
+          asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(d0), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+          asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(d1), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+        }
+        fence_proxy_async_smem();  // the tensor core reads the slab through the async proxy
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&b_ready_bar));
+        // nobody may overwrite the packed bytes (they sit in the staging buffers) before all have read them
+        ok = mbar_wait(smem_u32(&b_ready_bar), 0, &abort_flag, t_start);
+      }
+    }
+
+    int tm, tn;
     // residual prefetch for the very first chunk of this warp
-    if (has_res && lane == 0 && (int)blockIdx.x < total_tiles) {
-      const int tm0 = blockIdx.x / p.tiles_n, tn0 = blockIdx.x - tm0 * p.tiles_n;
-      const int oc0 = tn0 * out_cols_tile + chalf * chunks * 32, r0 = tm0 * kBM + quad * 32;
+    if (ok && has_res && lane == 0 && tile_at<WS>(p, 0, tm, tn)) {
+      const int oc0 = tn * out_cols_tile + chalf * chunks * 32, r0 = tm * kBM + quad * 32;
       const uint32_t bar = smem_u32(&res_bar[ew][0]);
       mbar_arrive_expect_tx(bar, kStageBufBytes);
       tma_load_2d(my_stage, &tm_r, oc0 < p.n_out ? oc0 : 0, r0 < p.M ? r0 : 0, bar);
     }
 
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tcount) {
-      const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
-      const uint32_t buf = tcount & 1, aph = (tcount >> 1) & 1;
+    for (int i = 0; ok && tile_at<WS>(p, i, tm, tn); ++i) {
+      const uint32_t buf = i & 1, aph = (i >> 1) & 1;
       const int out0 = tn * out_cols_tile;  // first output column of the tile
       const int m = tm * kBM + quad * 32 + lane;
       const bool row_ok = m < p.M;
 
-      // this warp's s_w / bias slices for the tile -> shared memory (before the accumulator is ready)
-      __syncwarp();
-      for (int c = 0; Cfg::kScaleSlab && c < chunks; ++c) {
-        const int col = (chalf * chunks + c) * 32;
-        const int nv = (glu ? out0 : tn * BN) + col + lane;  // value channel of this lane
-        const uint32_t off = (uint32_t)((glu ? 2 * c : c) * 32 + lane) * 4;
-        float wv = 0.0f, bv = 0.0f;
-        if (nv < n_value_limit) {
-          wv = __ldg(p.s_w + nv);
-          if (p.bias != nullptr) bv = __ldg(p.bias + nv);
-        }
-        asm volatile("st.shared.f32 [%0], %1;" ::"r"(my_sw + off), "f"(wv) : "memory");
-        asm volatile("st.shared.f32 [%0], %1;" ::"r"(my_bias + off), "f"(bv) : "memory");
-        if (glu) {
-          const int ng = p.N / 2 + out0 + col + lane;  // gate channel
-          float wg = 0.0f, bg = 0.0f;
-          if (ng < p.N) {
-            wg = __ldg(p.s_w + ng);
-            if (p.bias != nullptr) bg = __ldg(p.bias + ng);
+      if (!WS && Cfg::kScaleSlab) {
+        // this warp's s_w / bias slices for the tile -> shared memory (before the accumulator is ready)
+        __syncwarp();
+        for (int c = 0; c < chunks; ++c) {
+          const int col = (chalf * chunks + c) * 32;
+          const int nv = (glu ? out0 : tn * BN) + col + lane;  // value channel of this lane
+          const uint32_t off = c * slab_chunk_stride + lane * 4;
+          float wv = 0.0f, bv = 0.0f;
+          if (nv < n_value_limit) {
+            wv = __ldg(p.s_w + nv);
+            if (p.bias != nullptr) bv = __ldg(p.bias + nv);
           }
-          asm volatile("st.shared.f32 [%0], %1;" ::"r"(my_sw + off + 128), "f"(wg) : "memory");
-          asm volatile("st.shared.f32 [%0], %1;" ::"r"(my_bias + off + 128), "f"(bg) : "memory");
+          asm volatile("st.shared.f32 [%0], %1;" ::"r"(slab_sw + off), "f"(wv) : "memory");
+          asm volatile("st.shared.f32 [%0], %1;" ::"r"(slab_bias + off), "f"(bv) : "memory");
+          if (glu) {
+            const int ng = p.N / 2 + out0 + col + lane;  // gate channel
+            float wg = 0.0f, bg = 0.0f;
+            if (ng < p.N) {
+              wg = __ldg(p.s_w + ng);
+              if (p.bias != nullptr) bg = __ldg(p.bias + ng);
+            }
+            asm volatile("st.shared.f32 [%0], %1;" ::"r"(slab_sw + off + slab_gate_off), "f"(wg) : "memory");
+            asm volatile("st.shared.f32 [%0], %1;" ::"r"(slab_bias + off + slab_gate_off), "f"(bg) : "memory");
+          }
         }
       }
       const float sx = (p.s_x_kind == AQT_SCALE_ROW) ? (row_ok ? __ldg(p.s_x + m) : 0.0f) : __ldg(p.s_x);
@@ -438,13 +556,13 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       if (!mbar_wait(smem_u32(&tmem_full_bar[buf]), aph, &abort_flag, t_start)) break;
       tc_fence_after();
       const uint32_t lane_addr = tmem_base + buf * BN + ((uint32_t)(quad * 32) << 16);
-      bool ok = true;
 
       for (int c = 0; c < chunks; ++c) {
         const int col = (chalf * chunks + c) * 32;  // column offset inside the tile's output
         const int oc = out0 + col;                  // first global output column of this chunk
         const uint32_t sb = store_count % SBUFS;
         const uint32_t sbuf = my_stage + sb * kStageBufBytes;
+        const uint32_t c_sw = slab_sw + c * slab_chunk_stride, c_bias = slab_bias + c * slab_chunk_stride;
         float a[32];
         uint32_t acc[32];
         const bool last_chunk = (c == chunks - 1);
@@ -465,7 +583,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 if (n0 + j < p.N) p.acc_debug[(int64_t)m * p.N + n0 + j] = (int32_t)acc[j];
             }
           }
-          if (Cfg::kScaleSlab) dequant32<SMALL>(acc, sx, my_sw + c * 128, my_bias + c * 128, a);
+          if (Cfg::kScaleSlab) dequant32<SMALL>(acc, sx, c_sw, c_bias, a);
           else dequant32_gmem<SMALL>(acc, sx, p.s_w, p.bias, tn * BN + col, p.N, a);
           if (p.act == AQT_ACT_SWISH) {
 #pragma unroll
@@ -484,7 +602,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 if (ng + j < p.N) p.acc_debug[(int64_t)m * p.N + ng + j] = (int32_t)acc[j];
             }
           }
-          if (Cfg::kScaleSlab) dequant32<SMALL>(acc, sx, my_sw + c * 256 + 128, my_bias + c * 256 + 128, g);
+          if (Cfg::kScaleSlab) dequant32<SMALL>(acc, sx, c_sw + slab_gate_off, c_bias + slab_gate_off, g);
           else dequant32_gmem<SMALL>(acc, sx, p.s_w, p.bias, p.N / 2 + oc, p.N, g);
 #pragma unroll
           for (int j = 0; j < 32; ++j) g[j] = sigmoid_f(g[j]);
@@ -502,7 +620,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 if (oc + j < p.N / 2) p.acc_debug[(int64_t)m * p.N + oc + j] = (int32_t)acc[j];
             }
           }
-          if (Cfg::kScaleSlab) dequant32<SMALL>(acc, sx, my_sw + c * 256, my_bias + c * 256, a);
+          if (Cfg::kScaleSlab) dequant32<SMALL>(acc, sx, c_sw, c_bias, a);
           else dequant32_gmem<SMALL>(acc, sx, p.s_w, p.bias, oc, p.N / 2, a);
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
@@ -511,6 +629,15 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           }
         }
 
+        // the chunk this warp handles after this one (for the residual prefetch)
+        int ntm = tm, ntn = tn, nc = c + 1;
+        bool have_next = true;
+        if (nc == chunks) {
+          nc = 0;
+          have_next = tile_at<WS>(p, i + 1, ntm, ntn);
+        }
+        const int noc = ntn * out_cols_tile + (chalf * chunks + nc) * 32, nr = ntm * kBM + quad * 32;
+
         if (has_res) {
           if (SBUFS == 2) {
             // Buffers alternate: the residual of this chunk was requested one chunk ago into `sb`.
@@ -518,12 +645,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             // used it has been read out, then wait for this chunk's tile.
             if (lane == 0) {
               tma_store_wait_read<0>();
-              // next chunk of this warp: next in this tile, or the first of its next tile
-              int ntile = tile, nc = c + 1;
-              if (nc == chunks) { nc = 0; ntile = tile + gridDim.x; }
-              if (ntile < total_tiles) {
-                const int ntm = ntile / p.tiles_n, ntn = ntile - ntm * p.tiles_n;
-                const int noc = ntn * out_cols_tile + (chalf * chunks + nc) * 32, nr = ntm * kBM + quad * 32;
+              if (have_next) {
                 const uint32_t nb = (store_count + 1) % SBUFS;
                 const uint32_t bar = smem_u32(&res_bar[ew][nb]);
                 mbar_arrive_expect_tx(bar, kStageBufBytes);
@@ -568,11 +690,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             // single buffer: the next chunk's residual can only be requested once this store has
             // read the buffer out (the warp is otherwise idle until its next chunk)
             tma_store_wait_read<0>();
-            int ntile = tile, nc = c + 1;
-            if (nc == chunks) { nc = 0; ntile = tile + gridDim.x; }
-            if (ntile < total_tiles) {
-              const int ntm = ntile / p.tiles_n, ntn = ntile - ntm * p.tiles_n;
-              const int noc = ntn * out_cols_tile + (chalf * chunks + nc) * 32, nr = ntm * kBM + quad * 32;
+            if (have_next) {
               const uint32_t bar = smem_u32(&res_bar[ew][0]);
               mbar_arrive_expect_tx(bar, kStageBufBytes);
               tma_load_2d(my_stage, &tm_r, noc < p.n_out ? noc : 0, nr < p.M ? nr : 0, bar);
@@ -623,9 +741,9 @@ static EncodeTiledFn get_encode_tiled() {
 }
 
 // 2-D row-major tensor [rows, cols] with `pitch_bytes` between rows; box [box_rows, box_cols];
-// 128-byte swizzle (box_cols * element size must be 128 bytes).
+// 128-byte swizzle (box_cols * element size must then be 128 bytes) or none.
 static int make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, const void* base, uint64_t rows, uint64_t cols,
-                       uint64_t pitch_bytes, uint32_t box_rows, uint32_t box_cols) {
+                       uint64_t pitch_bytes, uint32_t box_rows, uint32_t box_cols, bool swizzle128 = true) {
   EncodeTiledFn enc = get_encode_tiled();
   if (enc == nullptr) {
     if (debug_enabled()) fprintf(stderr, "[aqt] driver entry point for tensor map encoding not found\n");
@@ -636,7 +754,8 @@ static int make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, const void* bas
   cuuint32_t box[2] = {box_cols, box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = enc(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                   swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS && debug_enabled())
     fprintf(stderr, "[aqt] tensor map encode failed: CUresult %d (rows %llu cols %llu pitch %llu box %u x %u base %p)\n", (int)r,
             (unsigned long long)rows, (unsigned long long)cols, (unsigned long long)pitch_bytes, box_rows, box_cols, base);
@@ -673,17 +792,29 @@ static int pick_bn(int64_t M, int64_t N, bool glu, int sms) {
   return best_bn;
 }
 
-template <int BN, int STAGES, int EW, bool SMALL, bool DEBUG>
-static int launch_qgemm_inst(const int8_t* a, const int8_t* b, float* y, int64_t ldy, const GemmParams& p0, cudaStream_t st) {
-  using Cfg = GemmCfg<BN, STAGES, EW>;
+// b: weight codes as the kernel reads them -- int8 [N, K], or (BPACK) packed nibbles [N, K/2].
+template <int BN, int STAGES, int EW, bool WS, bool BPACK, bool SMALL, bool DEBUG>
+static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t ldy, const GemmParams& p0, cudaStream_t st) {
+  using Cfg = GemmCfg<BN, STAGES, EW, WS>;
   GemmParams p = p0;
   p.tiles_m = (int)ceil_div(p.M, kBM);
   p.tiles_n = (int)ceil_div(p.N, BN);
   p.k_blocks = (int)ceil_div(p.K, kBK);
+  const int sms = sm_count();
+  if (sms <= 0) return AQT_ERR_CUDA;
+  {
+    const bool glu = (p.act == AQT_ACT_GLU) || (p.act == AQT_ACT_GLU_SWISH);
+    if ((glu ? BN / 2 : BN) / 32 / (EW / 4) < 1) return AQT_ERR_UNSUPPORTED;  // a warp without columns would never release TMEM
+    if (WS && (p.k_blocks > kWsMaxKBlocks || p.tiles_n > sms)) return AQT_ERR_UNSUPPORTED;
+  }
   CUtensorMap tm_a, tm_b, tm_y, tm_r;
   int rc = make_map_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, a, (uint64_t)p.M, (uint64_t)p.K, (uint64_t)p.K, kBM, kBK);
   if (rc != AQT_OK) return rc;
-  rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, b, (uint64_t)p.N, (uint64_t)p.K, (uint64_t)p.K, BN / 2, kBK);
+  if (BPACK) {
+    rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, b, (uint64_t)p.N, (uint64_t)p.K / 2, (uint64_t)p.K / 2, BN / 2, 64, false);
+  } else {
+    rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, b, (uint64_t)p.N, (uint64_t)p.K, (uint64_t)p.K, BN / 2, kBK);
+  }
   if (rc != AQT_OK) return rc;
   rc = make_map_2d(&tm_y, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, y, (uint64_t)p.M, (uint64_t)p.n_out, (uint64_t)ldy * 4, kStoreBoxRows,
                    kStoreBoxCols);
@@ -695,34 +826,44 @@ static int launch_qgemm_inst(const int8_t* a, const int8_t* b, float* y, int64_t
   } else {
     tm_r = tm_y;  // never dereferenced
   }
-  auto kernel = qgemm_i8_kernel<BN, STAGES, EW, SMALL, DEBUG>;
+  auto kernel = qgemm_i8_kernel<BN, STAGES, EW, WS, BPACK, SMALL, DEBUG>;
   static bool attr_set = false;
   if (!attr_set) {
     AQT_RETURN_IF_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
     attr_set = true;
   }
-  const int sms = sm_count();
-  if (sms <= 0) return AQT_ERR_CUDA;
-  {
-    const bool glu = (p.act == AQT_ACT_GLU) || (p.act == AQT_ACT_GLU_SWISH);
-    if ((glu ? BN / 2 : BN) / 32 / (EW / 4) < 1) return AQT_ERR_UNSUPPORTED;  // a warp without columns would never release TMEM
-  }
   const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
-  const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+  unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+  if (WS && (int)grid < p.tiles_n) grid = (unsigned)p.tiles_n;  // every n-tile needs an owner
   kernel<<<grid, Cfg::kThreads, Cfg::kSmemBytes, st>>>(tm_a, tm_b, tm_y, tm_r, p);
   return AQT_LAUNCH_STATUS();
 }
 
-template <int BN, int STAGES, int EW>
-static int launch_qgemm_cfg(const int8_t* a, const int8_t* b, float* y, int64_t ldy, const GemmParams& p, cudaStream_t st) {
-  if (p.acc_debug != nullptr) return launch_qgemm_inst<BN, STAGES, EW, false, true>(a, b, y, ldy, p, st);
-  if (p.small_acc) return launch_qgemm_inst<BN, STAGES, EW, true, false>(a, b, y, ldy, p, st);
-  return launch_qgemm_inst<BN, STAGES, EW, false, false>(a, b, y, ldy, p, st);
+template <int BN, int STAGES, int EW, bool WS, bool BPACK>
+static int launch_qgemm_cfg(const int8_t* a, const void* b, float* y, int64_t ldy, const GemmParams& p, cudaStream_t st) {
+  if (p.acc_debug != nullptr) return launch_qgemm_inst<BN, STAGES, EW, WS, BPACK, false, true>(a, b, y, ldy, p, st);
+  if (p.small_acc) return launch_qgemm_inst<BN, STAGES, EW, WS, BPACK, true, false>(a, b, y, ldy, p, st);
+  return launch_qgemm_inst<BN, STAGES, EW, WS, BPACK, false, false>(a, b, y, ldy, p, st);
 }
 
-// a: int8 [M, K] codes; b: int8 [N, K] codes (both dense, 16-byte aligned, K % 16 == 0).
-static int launch_qgemm(const int8_t* a, const int8_t* b, float* y, int64_t ldy, const GemmParams& p, cudaStream_t st) {
+// True if the weight-stationary kernel takes this shape (and can therefore unpack 4-bit weights itself).
+static bool qgemm_uses_ws(int64_t N, int64_t K) {
+  static const char* off = getenv("AQT_NO_WS");  // tuning aid: force the streaming kernel
+  if (off != nullptr) return false;
+  const int sms = sm_count() > 0 ? sm_count() : 148;
+  return ceil_div(K, kBK) <= kWsMaxKBlocks && ceil_div(N, 128) <= sms;
+}
+
+// a: int8 [M, K] codes.  b: int8 [N, K] codes, or -- only if b_packed and qgemm_uses_ws(N, K) --
+// packed nibbles [N, K/2].  All dense, 16-byte aligned.
+static int launch_qgemm(const int8_t* a, const void* b, bool b_packed, float* y, int64_t ldy, const GemmParams& p, cudaStream_t st) {
   const bool glu = (p.act == AQT_ACT_GLU) || (p.act == AQT_ACT_GLU_SWISH);
+  if (qgemm_uses_ws(p.N, p.K)) {
+    // tile width 128; a GLU tile has 64 output columns, i.e. two chunks per lane quadrant
+    if (glu) return b_packed ? launch_qgemm_cfg<128, 6, 8, true, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 6, 8, true, false>(a, b, y, ldy, p, st);
+    return b_packed ? launch_qgemm_cfg<128, 6, 16, true, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 6, 16, true, false>(a, b, y, ldy, p, st);
+  }
+  if (b_packed) return AQT_ERR_UNSUPPORTED;
   int bn = pick_bn(p.M, p.N, glu, sm_count() > 0 ? sm_count() : 148);
   // tuning aid: AQT_BN=64|128|256 in the environment overrides the tile-width heuristic
   static const char* force = getenv("AQT_BN");
@@ -731,14 +872,14 @@ static int launch_qgemm(const int8_t* a, const int8_t* b, float* y, int64_t ldy,
     if ((v == 64 && !glu) || v == 128 || v == 256) bn = v;
   }
   // Deep K: operand loads bound the tile, so the ring gets the shared memory and four warps run
-  // the (short) epilogue.  Shallow K: the epilogue bounds the tile and gets eight warps.
+  // the (short) epilogue.  Shallow K: the epilogue bounds the tile and gets more warps.
   const bool deep_k = p.K >= 2048 && !glu;
-  if (bn == 256) return deep_k ? launch_qgemm_cfg<256, 4, 4>(a, b, y, ldy, p, st) : launch_qgemm_cfg<256, 3, 16>(a, b, y, ldy, p, st);
+  if (bn == 256) return deep_k ? launch_qgemm_cfg<256, 4, 4, false, false>(a, b, y, ldy, p, st) : launch_qgemm_cfg<256, 3, 16, false, false>(a, b, y, ldy, p, st);
   // every epilogue warp needs at least one 32-column chunk: a GLU tile of width 128 has only
   // 64 output columns, i.e. two chunks per lane quadrant
-  if (bn == 128 && glu) return launch_qgemm_cfg<128, 4, 8>(a, b, y, ldy, p, st);
-  if (bn == 128) return deep_k ? launch_qgemm_cfg<128, 6, 4>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 4, 16>(a, b, y, ldy, p, st);
-  return deep_k ? launch_qgemm_cfg<64, 8, 4>(a, b, y, ldy, p, st) : launch_qgemm_cfg<64, 5, 8>(a, b, y, ldy, p, st);
+  if (bn == 128 && glu) return launch_qgemm_cfg<128, 4, 8, false, false>(a, b, y, ldy, p, st);
+  if (bn == 128) return deep_k ? launch_qgemm_cfg<128, 6, 4, false, false>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 4, 16, false, false>(a, b, y, ldy, p, st);
+  return deep_k ? launch_qgemm_cfg<64, 8, 4, false, false>(a, b, y, ldy, p, st) : launch_qgemm_cfg<64, 5, 8, false, false>(a, b, y, ldy, p, st);
 }
 
 }  // namespace aqt
