@@ -213,15 +213,19 @@ def run_ours(args):
     names = ["quantize(x) 12800x512", "qmatmul 512->2048 swish", "quantize(u) 12800x2048", "qmatmul 2048->512"]
 
     # pre-marshalled C-ABI calls (one set per rotating buffer) so that Python stays ahead of the GPU
-    calls = []
-    for r in range(R):
-        calls.append((
-            aqt.bind_quantize(xs[r], specs[0].bits_a, aqt.AXIS_ROW, aqt.ROUND_NEAREST_EVEN, False, q1, s1),
-            aqt.bind_qmatmul(q1, s1, layers[0].wq, layers[0].s_w, None, None, 1.0, specs[0].K, 8, specs[0].bits_w, specs[0].act,
-                             aqt.SCALE_ROW, u, ws),
-            aqt.bind_quantize(u, specs[1].bits_a, aqt.AXIS_ROW, aqt.ROUND_NEAREST_EVEN, False, q2, s2),
-            aqt.bind_qmatmul(q2, s2, layers[1].wq, layers[1].s_w, None, None, 1.0, specs[1].K, 8, specs[1].bits_w, specs[1].act,
-                             aqt.SCALE_ROW, ys[r], ws)))
+    def make_calls(st):
+        out = []
+        for r in range(R):
+            out.append((
+                aqt.bind_quantize(xs[r], specs[0].bits_a, aqt.AXIS_ROW, aqt.ROUND_NEAREST_EVEN, False, q1, s1, st),
+                aqt.bind_qmatmul(q1, s1, layers[0].wq, layers[0].s_w, None, None, 1.0, specs[0].K, 8, specs[0].bits_w,
+                                 specs[0].act, aqt.SCALE_ROW, u, ws, st),
+                aqt.bind_quantize(u, specs[1].bits_a, aqt.AXIS_ROW, aqt.ROUND_NEAREST_EVEN, False, q2, s2, st),
+                aqt.bind_qmatmul(q2, s2, layers[1].wq, layers[1].s_w, None, None, 1.0, specs[1].K, 8, specs[1].bits_w,
+                                 specs[1].act, aqt.SCALE_ROW, ys[r], ws, st)))
+        return out
+
+    calls = make_calls(stream)
 
     def step(i, events=None):
         c = calls[i % R]
@@ -245,20 +249,56 @@ def run_ours(args):
     if aqt.aqt_device_status() != 0:
         raise SystemExit("device status reports a failed wait during warm-up")
 
+    # The same C-ABI calls for R consecutive steps captured in a CUDA graph (launch latency out of
+    # the way).  The timed region replays the graph and, every R + 1 steps, runs one step call by
+    # call with CUDA events around each call: those give the per-kernel durations of the roofline.
+    graph = None
+    if not args.no_graph:
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            gcalls = make_calls(side)
+            for r in range(R):
+                for c in gcalls[r]:
+                    c()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for r in range(R):
+                for c in gcalls[r]:
+                    c()
+        for _ in range(2):
+            graph.replay()
+        barrier()
+
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    n_instr = len([i for i in range(args.steps) if i % (R + 1) == 0]) if graph is not None else args.steps
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(n_instr)]
+    e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
-    for i in range(args.steps):
-        step(i, evs[i])
+    e_begin.record(stream)
+    i, k, replays = 0, 0, 0
+    while i < args.steps:
+        if graph is None:
+            step(i, evs[k]); k += 1; i += 1
+            continue
+        step(i, evs[k]); k += 1; i += 1          # instrumented step
+        if args.steps - i >= R:
+            graph.replay(); replays += 1; i += R  # R steps, one launch
+        else:
+            while i < args.steps:
+                step(i); i += 1
+    e_end.record(stream)
     barrier()
-    total_ms = evs[0][0].elapsed_time(evs[-1][4])
+    total_ms = e_begin.elapsed_time(e_end)
     clocks = sampler.stop() if rank == 0 else None
     status = aqt.aqt_device_status()
+    evs = evs[:k]
 
-    per_call_ms = [statistics.mean(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(args.steps)) for j in range(4)]
+    per_call_ms = [statistics.mean(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(len(evs))) for j in range(4)]
     t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -324,7 +364,9 @@ def run_ours(args):
             "clocks": clocks, "device_status": status,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 4 * M * s0.K, "d2h_bytes_per_step": 4 * M * s1_.N,
                     "ms_per_step": float(te.item()) / args.steps},
-            "gpu_launches": args.steps * 6, "sum_call_ms_per_step": sum(per_call_ms),
+            "gpu_launches": args.steps * 5, "sum_call_ms_per_step": sum(per_call_ms),
+            "launch_mode": ("cuda graph of %d steps x %d replays + %d call-by-call steps with per-call events" % (R, replays, len(evs)))
+            if graph is not None else "call by call",
             "roofline": roofline}
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline()
@@ -339,6 +381,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch every step call by call (no CUDA graph replay)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

@@ -10,12 +10,30 @@ namespace aqt {
 constexpr int kQuantThreads = 256;
 constexpr int kQuantMaxVec = 4;  // float4 loads held in registers per thread (16 elements)
 
-// Pack four codes into the output word: int8 container (4 bytes) or nibbles (2 bytes).
+// Pack four codes (sign-extended ints) into the output word: int8 container (4 bytes) or nibbles
+// (2 bytes).  Byte permutes take the low byte of each code.
 __device__ __forceinline__ uint32_t pack4_i8(int a, int b, int c, int d) {
-  return (uint32_t)(a & 0xFF) | ((uint32_t)(b & 0xFF) << 8) | ((uint32_t)(c & 0xFF) << 16) | ((uint32_t)(d & 0xFF) << 24);
+  const uint32_t lo = __byte_perm((uint32_t)a, (uint32_t)b, 0x0040);  // a.b0, b.b0
+  const uint32_t hi = __byte_perm((uint32_t)c, (uint32_t)d, 0x0040);  // c.b0, d.b0
+  return __byte_perm(lo, hi, 0x5410);
 }
 __device__ __forceinline__ uint32_t pack4_i4(int a, int b, int c, int d) {
-  return (uint32_t)(a & 0xF) | ((uint32_t)(b & 0xF) << 4) | ((uint32_t)(c & 0xF) << 8) | ((uint32_t)(d & 0xF) << 12);
+  const uint32_t x = pack4_i8(a, b, c, d) & 0x0F0F0F0Fu;
+  const uint32_t y = x | (x >> 4);         // byte 0 = n0 | n1 << 4, byte 2 = n2 | n3 << 4
+  return __byte_perm(y, 0u, 0x4420) & 0xFFFFu;
+}
+
+// Four elements of a row whose scale constants are known, fast path of quantize_elem: the
+// correctly rounded quotient by one multiply and two FMAs, then one conversion.  No clip: with
+// abs-max scaling |x / s| <= qmax (1 + 2^-23), which every rounding rule maps inside +-qmax; the
+// clip only matters for the subnormal scales that never take this path.
+template <int ROUNDING>
+__device__ __forceinline__ int quantize_fast(float x, float s, float r) {
+  const float q0 = __fmul_rn(x, r);
+  const float e = __fmaf_rn(-q0, s, x);
+  const float v = __fmaf_rn(e, r, q0);
+  if (ROUNDING == AQT_ROUND_HALF_UP_FLOOR) return __float2int_rd(__fadd_rn(v, 0.5f));
+  return __float2int_rn(v);
 }
 
 // Per-row quantizer, row held in registers.  G threads cooperate on one row (G a power of two,
@@ -65,10 +83,18 @@ __global__ void __launch_bounds__(kQuantThreads) quantize_rows_reg_kernel(
   for (int i = 0; i < kQuantMaxVec; ++i) {
     const int idx = t + i * G;
     if (idx < nvec) {
-      const int a = quantize_elem<ROUNDING>(v[i].x, c, qmax);
-      const int b = quantize_elem<ROUNDING>(v[i].y, c, qmax);
-      const int cc = quantize_elem<ROUNDING>(v[i].z, c, qmax);
-      const int d = quantize_elem<ROUNDING>(v[i].w, c, qmax);
+      int a, b, cc, d;
+      if (c.fast) {  // uniform over the row
+        a = quantize_fast<ROUNDING>(v[i].x, c.s, c.r);
+        b = quantize_fast<ROUNDING>(v[i].y, c.s, c.r);
+        cc = quantize_fast<ROUNDING>(v[i].z, c.s, c.r);
+        d = quantize_fast<ROUNDING>(v[i].w, c.s, c.r);
+      } else {
+        a = quantize_elem<ROUNDING>(v[i].x, c, qmax);
+        b = quantize_elem<ROUNDING>(v[i].y, c, qmax);
+        cc = quantize_elem<ROUNDING>(v[i].z, c, qmax);
+        d = quantize_elem<ROUNDING>(v[i].w, c, qmax);
+      }
       // one output word per float4: 2 bytes of nibbles or 4 bytes of int8 codes
       if (PACK) {
         reinterpret_cast<uint16_t*>(q_out)[row * (int64_t)nvec + idx] = (uint16_t)pack4_i4(a, b, cc, d);
