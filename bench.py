@@ -368,10 +368,51 @@ def run_ours(args):
             "launch_mode": ("cuda graph of %d steps x %d replays + %d call-by-call steps with per-call events" % (R, replays, len(evs)))
             if graph is not None else "call by call",
             "roofline": roofline}
+    if world == 1 and not args.no_encoder:
+        line["encoder"] = encoder_frames_per_s(dev)
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline()
     print(json.dumps(line), flush=True)
     return 0
+
+
+def encoder_frames_per_s(dev, steps: int = 5):
+    """Second half of the metric: frames/s of the 17-block Conformer-encoder linear stack
+    (d = 512, ff = 2048, batch 64 x 400 frames, FFN weights int4, attention / pointwise weights int8,
+    int8 per-row activations, fp32 residual adds fused into the epilogues).  170 aqt_linear_fwd calls
+    per step, replayed from a CUDA graph.  Weights are N(0, 1/fan_in) drawn on the GPU (seeded)."""
+    import torch
+    from paper_2203_15952_b200 import inputs as gen
+    from paper_2203_15952_b200.encoder import EncoderStack, QuantLinear
+    w = gen.WORKLOADS[4]
+    specs = gen.workload_layers(w)
+    g = torch.Generator(device=dev).manual_seed(4)
+    blocks = []
+    for _ in range(w.blocks):
+        blocks.append([QuantLinear.from_float(s, torch.randn((s.N, s.K), generator=g, device=dev) * (s.K ** -0.5)) for s in specs])
+    stack = EncoderStack(w.M, w.d, w.ff, blocks, dev)
+    x = torch.randn((w.M, w.d), generator=g, device=dev)
+    stream = torch.cuda.current_stream()
+    side = torch.cuda.Stream()
+    side.wait_stream(stream)
+    with torch.cuda.stream(side):
+        stack.forward(x)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        stack.forward(x)
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        graph.replay()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    return {"workload": w.name, "frames_per_s": w.M / (ms * 1e-3), "ms_per_step": ms, "tops": stack.ops / (ms * 1e-3) / 1e12,
+            "steps": steps, "linears_per_step": len(specs) * w.blocks, "launch_mode": "cuda graph"}
 
 
 def main():
@@ -381,6 +422,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-encoder", action="store_true", help="skip the 17-block encoder-stack frames/s leg")
     ap.add_argument("--no-graph", action="store_true", help="launch every step call by call (no CUDA graph replay)")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -11,6 +11,11 @@
 //   warps 2..     epilogue (4, 8 or 16 warps): TMEM -> registers -> de-quantize / bias / activation / residual ->
 //                 swizzled shared staging -> TMA store; overlaps the next tile's MMAs.  The
 //                 residual tile is fetched by TMA into the same staging buffer beforehand.
+// CTA pairs (K > 512, M > 128): two CTAs of a cluster share one 256-row tile.  Each loads its own
+// 128 rows of A and half of the tile's weight rows; the pair's leader issues
+// tcgen05.mma.cta_group::2 (M = 256), which reads both CTAs' shared memory and writes each CTA's
+// rows into that CTA's TMEM.  Per CTA this halves the weight bytes per MMA clock (operand loads and
+// shared-memory reads), which is what bounds the deep-K shapes.  No load is multicast.
 // Every wait on an mbarrier is bounded by a wall-clock limit; on expiry the CTA records
 // AQT_ERR_TIMEOUT in the device status word, leaves its loops, frees its TMEM and returns.
 #pragma once
@@ -39,11 +44,12 @@ constexpr uint64_t kWaitLimitNs = 2000000000ull;                   // 2 s
 // memory for its whole life and streams only activation k-blocks through the ring, which halves
 // the L2 -> shared-memory traffic and lets the ring hold more than one tile of A.
 constexpr int kWsMaxKBlocks = 4;  // K <= 512
-template <int BN, int STAGES, int EW, bool WS>
+template <int BN, int STAGES, int EW, bool WS, bool CTA2 = false>
 struct GemmCfg {
+  static_assert(!(WS && CTA2), "the weight-stationary kernel runs one CTA per tile");
   static constexpr int kThreads = 32 * (2 + EW);
   static constexpr int kABytes = kBM * kBK;
-  static constexpr int kBBytes = BN * kBK;
+  static constexpr int kBBytes = (CTA2 ? BN / 2 : BN) * kBK;  // a CTA of a pair holds half of the tile's weight rows
   static constexpr int kStageBytes = WS ? kABytes : kABytes + kBBytes;
   static constexpr int kResidentBytes = WS ? kWsMaxKBlocks * kBBytes : 0;
   static constexpr int kStages = STAGES;
@@ -136,6 +142,29 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* m, 
       "l"(reinterpret_cast<uint64_t>(m)), "r"(c0), "r"(c1), "r"(bar)
       : "memory");
 }
+// The same for a CTA of a pair: completion is counted on the barrier at the same shared-memory
+// offset in the pair's leader (rank bit of the address cleared).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* m, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(m)), "r"(c0), "r"(c1), "r"(bar & 0xFEFFFFFFu)
+      : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Arrive on the mbarrier at this shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar, uint32_t rank) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(bar), "r"(rank));
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, uint32_t src, int c0, int c1) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(
                    reinterpret_cast<uint64_t>(m)),
@@ -157,6 +186,30 @@ __device__ __forceinline__ void tmem_relinquish() {
 }
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// Pair form: arrive on the barrier at this offset in both CTAs once the pair's MMAs have completed.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+               "h"((uint16_t)3)
+               : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B^T, 256 x N x 32: each CTA supplies 128 rows of A and N/2 rows of B.
+__device__ __forceinline__ void tc_mma_i8_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
 }
 // Arrive on an mbarrier once all MMAs issued so far by this thread have completed.
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -198,8 +251,8 @@ __device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t saddr) {
   return d;
 }
 // Instruction descriptor: D int32, A and B signed 8-bit, both K-major, M = 128, N = BN.
-__host__ __device__ constexpr uint32_t idesc_i8(int bn) {
-  return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+__host__ __device__ constexpr uint32_t idesc_i8(int bn, int m = kBM) {
+  return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -285,8 +338,15 @@ __device__ __forceinline__ void dequant32_gmem(const uint32_t (&acc)[32], float 
 // i-th tile of this CTA.  Standard order: tiles are numbered n-fastest and dealt round-robin.
 // Weight-stationary order: the CTA owns n-tile (blockIdx % tiles_n) and takes every g-th m-tile,
 // g being the number of CTAs that own the same n-tile.
-template <bool WS>
+// CTA pairs: both CTAs of a pair walk the pair's tiles; tm counts 256-row tiles.
+template <bool WS, bool CTA2 = false>
 __device__ __forceinline__ bool tile_at(const GemmParams& p, int i, int& tm, int& tn) {
+  if (CTA2) {
+    const int tile = (blockIdx.x >> 1) + i * (gridDim.x >> 1);
+    tm = tile / p.tiles_n;
+    tn = tile - tm * p.tiles_n;
+    return tile < p.tiles_m * p.tiles_n;
+  }
   if (WS) {
     tn = blockIdx.x % p.tiles_n;
     const int r = blockIdx.x / p.tiles_n;
@@ -300,14 +360,17 @@ __device__ __forceinline__ bool tile_at(const GemmParams& p, int i, int& tm, int
   return tile < p.tiles_m * p.tiles_n;
 }
 
-template <int BN, int STAGES, int EW, bool WS, bool BPACK, bool SMALL, bool DEBUG>
+template <int BN, int STAGES, int EW, bool WS, bool BPACK, bool SMALL, bool DEBUG, bool CTA2 = false>
 __global__ void __launch_bounds__(32 * (2 + EW), 1)
 qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                 const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_r, const GemmParams p) {
-  using Cfg = GemmCfg<BN, STAGES, EW, WS>;
+  using Cfg = GemmCfg<BN, STAGES, EW, WS, CTA2>;
   constexpr int HALF = BN / 2;
   constexpr int SBUFS = Cfg::kStageBufs;
+  constexpr int TILE_M = CTA2 ? 2 * kBM : kBM;  // rows of a tile (of the pair's tile)
   static_assert(!BPACK || WS, "packed weights are unpacked into the resident slab");
+  const uint32_t pair_rank = CTA2 ? cluster_ctarank() : 0u;  // 0 = leader: issues the MMAs, owns the barriers the pair shares
+  const int row_in_tile = (int)pair_rank * kBM;               // this CTA's first row inside the tile
 
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full_bar[STAGES];
@@ -343,7 +406,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&tmem_full_bar[b]), 1);
-      mbar_init(smem_u32(&tmem_empty_bar[b]), EW);
+      mbar_init(smem_u32(&tmem_empty_bar[b]), CTA2 ? 2 * EW : EW);  // pair: both CTAs' epilogue warps release the leader's MMA
     }
     for (int w = 0; w < EW; ++w)
       for (int b = 0; b < SBUFS; ++b) mbar_init(smem_u32(&res_bar[w][b]), 1);
@@ -353,8 +416,13 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     fence_proxy_async_smem();
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(&tmem_base_slot), Cfg::kTmemCols);
-    tmem_relinquish();
+    if (CTA2) {
+      tmem_alloc_pair(smem_u32(&tmem_base_slot), Cfg::kTmemCols);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(smem_u32(&tmem_base_slot), Cfg::kTmemCols);
+      tmem_relinquish();
+    }
   }
   if (WS) {
     // scales and biases of the CTA's n-tile, once: values first, then (GLU) gates
@@ -379,6 +447,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   }
   tc_fence_before();
   __syncthreads();
+  if (CTA2) cluster_sync_all();  // the peer's barriers are initialised before anything is signalled on them
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
 
@@ -409,7 +478,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         }
       }
       int tm, tn;
-      for (int i = 0; ok && tile_at<WS>(p, i, tm, tn); ++i) {
+      for (int i = 0; ok && tile_at<WS, CTA2>(p, i, tm, tn); ++i) {
         // B rows of the two half-tiles: adjacent output channels, or (value, gate) halves for GLU
         const int row0 = glu ? tn * HALF : tn * BN;
         const int row1 = glu ? p.N / 2 + tn * HALF : tn * BN + HALF;
@@ -418,6 +487,14 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1, &abort_flag, t_start)) { ok = false; break; }
           const uint32_t bar = smem_u32(&full_bar[s]);
           const uint32_t stage = smem_ring + s * Cfg::kStageBytes;
+          if (CTA2) {
+            // The leader's barrier counts both CTAs' bytes; each CTA loads its 128 rows of A and
+            // its half of the weight rows (leader: first half / values, peer: second half / gates).
+            if (pair_rank == 0) mbar_arrive_expect_tx(bar, 2 * Cfg::kStageBytes);
+            tma_load_2d_pair(stage, &tm_a, kb * kBK, tm * TILE_M + row_in_tile, bar);
+            tma_load_2d_pair(stage + Cfg::kABytes, &tm_b, kb * kBK, pair_rank == 0 ? row0 : row1, bar);
+            continue;
+          }
           mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
           tma_load_2d(stage, &tm_a, kb * kBK, tm * kBM, bar);
           if (!WS) {
@@ -429,13 +506,13 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = idesc_i8(BN);
+    if (lane == 0 && pair_rank == 0) {
+      constexpr uint32_t idesc = idesc_i8(BN, TILE_M);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       if (WS) ok = mbar_wait(smem_u32(BPACK ? &b_ready_bar : &b_loaded_bar), 0, &abort_flag, t_start);
       int tm, tn;
-      for (int i = 0; ok && tile_at<WS>(p, i, tm, tn); ++i, ++tcount) {
+      for (int i = 0; ok && tile_at<WS, CTA2>(p, i, tm, tn); ++i, ++tcount) {
         const uint32_t buf = tcount & 1, aph = (tcount >> 1) & 1;
         if (!mbar_wait(smem_u32(&tmem_empty_bar[buf]), aph ^ 1, &abort_flag, t_start)) break;
         tc_fence_after();
@@ -450,11 +527,17 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 #pragma unroll
           for (int kk = 0; kk < kBK / kMmaK; ++kk) {
             // advancing K inside the 128-byte swizzle row: +32 bytes = +2 in the 16-byte address field
-            tc_mma_i8(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+            if (CTA2) tc_mma_i8_pair(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+            else tc_mma_i8(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
           }
-          tc_commit(smem_u32(&empty_bar[s]));  // stage reusable once these MMAs have read it
+          // stage reusable (in both CTAs of a pair) once these MMAs have read it
+          if (CTA2) tc_commit_pair(smem_u32(&empty_bar[s]));
+          else tc_commit(smem_u32(&empty_bar[s]));
         }
-        if (ok) tc_commit(smem_u32(&tmem_full_bar[buf]));  // accumulator complete
+        if (ok) {  // accumulator complete (in both CTAs' TMEM)
+          if (CTA2) tc_commit_pair(smem_u32(&tmem_full_bar[buf]));
+          else tc_commit(smem_u32(&tmem_full_bar[buf]));
+        }
       }
     }
   } else {
@@ -511,17 +594,18 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 
     int tm, tn;
     // residual prefetch for the very first chunk of this warp
-    if (ok && has_res && lane == 0 && tile_at<WS>(p, 0, tm, tn)) {
-      const int oc0 = tn * out_cols_tile + chalf * chunks * 32, r0 = tm * kBM + quad * 32;
+    if (ok && has_res && lane == 0 && tile_at<WS, CTA2>(p, 0, tm, tn)) {
+      const int oc0 = tn * out_cols_tile + chalf * chunks * 32, r0 = tm * TILE_M + row_in_tile + quad * 32;
       const uint32_t bar = smem_u32(&res_bar[ew][0]);
       mbar_arrive_expect_tx(bar, kStageBufBytes);
       tma_load_2d(my_stage, &tm_r, oc0 < p.n_out ? oc0 : 0, r0 < p.M ? r0 : 0, bar);
     }
 
-    for (int i = 0; ok && tile_at<WS>(p, i, tm, tn); ++i) {
+    for (int i = 0; ok && tile_at<WS, CTA2>(p, i, tm, tn); ++i) {
       const uint32_t buf = i & 1, aph = (i >> 1) & 1;
       const int out0 = tn * out_cols_tile;  // first output column of the tile
-      const int m = tm * kBM + quad * 32 + lane;
+      const int row0_warp = tm * TILE_M + row_in_tile + quad * 32;  // first output row of this warp
+      const int m = row0_warp + lane;
       const bool row_ok = m < p.M;
 
       if (!WS && Cfg::kScaleSlab) {
@@ -573,7 +657,10 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             // accumulator buffer read out by this warp: hand it back before the arithmetic
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[buf]));
+            if (lane == 0) {
+              if (CTA2) mbar_arrive_cluster(smem_u32(&tmem_empty_bar[buf]), 0);
+              else mbar_arrive(smem_u32(&tmem_empty_bar[buf]));
+            }
           }
           if (DEBUG) {
             if (p.acc_debug != nullptr && row_ok) {
@@ -611,7 +698,10 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           if (last_chunk) {
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[buf]));
+            if (lane == 0) {
+              if (CTA2) mbar_arrive_cluster(smem_u32(&tmem_empty_bar[buf]), 0);
+              else mbar_arrive(smem_u32(&tmem_empty_bar[buf]));
+            }
           }
           if (DEBUG) {
             if (p.acc_debug != nullptr && row_ok) {
@@ -634,9 +724,9 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         bool have_next = true;
         if (nc == chunks) {
           nc = 0;
-          have_next = tile_at<WS>(p, i + 1, ntm, ntn);
+          have_next = tile_at<WS, CTA2>(p, i + 1, ntm, ntn);
         }
-        const int noc = ntn * out_cols_tile + (chalf * chunks + nc) * 32, nr = ntm * kBM + quad * 32;
+        const int noc = ntn * out_cols_tile + (chalf * chunks + nc) * 32, nr = ntm * TILE_M + row_in_tile + quad * 32;
 
         if (has_res) {
           if (SBUFS == 2) {
@@ -684,7 +774,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         __syncwarp();
         if (lane == 0) {
           // boxes that start inside the output are clipped at its edges by the copy engine
-          if (oc < p.n_out && tm * kBM + quad * 32 < p.M) tma_store_2d(&tm_y, sbuf, oc, tm * kBM + quad * 32);
+          if (oc < p.n_out && row0_warp < p.M) tma_store_2d(&tm_y, sbuf, oc, row0_warp);
           tma_store_commit();
           if (has_res && SBUFS == 1) {
             // single buffer: the next chunk's residual can only be requested once this store has
@@ -714,10 +804,12 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     }
   }
   __syncthreads();
+  if (CTA2) cluster_sync_all();  // neither CTA leaves (or frees TMEM) while its peer may still signal it or use its memory
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, Cfg::kTmemCols);
+    if (CTA2) tmem_dealloc_pair(tmem_base, Cfg::kTmemCols);
+    else tmem_dealloc(tmem_base, Cfg::kTmemCols);
   }
 }
 
@@ -793,11 +885,11 @@ static int pick_bn(int64_t M, int64_t N, bool glu, int sms) {
 }
 
 // b: weight codes as the kernel reads them -- int8 [N, K], or (BPACK) packed nibbles [N, K/2].
-template <int BN, int STAGES, int EW, bool WS, bool BPACK, bool SMALL, bool DEBUG>
+template <int BN, int STAGES, int EW, bool WS, bool BPACK, bool SMALL, bool DEBUG, bool CTA2 = false>
 static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t ldy, const GemmParams& p0, cudaStream_t st) {
-  using Cfg = GemmCfg<BN, STAGES, EW, WS>;
+  using Cfg = GemmCfg<BN, STAGES, EW, WS, CTA2>;
   GemmParams p = p0;
-  p.tiles_m = (int)ceil_div(p.M, kBM);
+  p.tiles_m = (int)ceil_div(p.M, CTA2 ? 2 * kBM : kBM);
   p.tiles_n = (int)ceil_div(p.N, BN);
   p.k_blocks = (int)ceil_div(p.K, kBK);
   const int sms = sm_count();
@@ -826,7 +918,7 @@ static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t l
   } else {
     tm_r = tm_y;  // never dereferenced
   }
-  auto kernel = qgemm_i8_kernel<BN, STAGES, EW, WS, BPACK, SMALL, DEBUG>;
+  auto kernel = qgemm_i8_kernel<BN, STAGES, EW, WS, BPACK, SMALL, DEBUG, CTA2>;
   static bool attr_set = false;
   if (!attr_set) {
     AQT_RETURN_IF_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
@@ -835,15 +927,34 @@ static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t l
   const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
   unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
   if (WS && (int)grid < p.tiles_n) grid = (unsigned)p.tiles_n;  // every n-tile needs an owner
+  if (CTA2) {
+    // one cluster of two CTAs per tile in flight
+    const int64_t pairs = sms / 2;
+    grid = 2u * (unsigned)(tiles < pairs ? tiles : pairs);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(Cfg::kThreads, 1, 1);
+    cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    AQT_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, kernel, tm_a, tm_b, tm_y, tm_r, p));
+    return AQT_LAUNCH_STATUS();
+  }
   kernel<<<grid, Cfg::kThreads, Cfg::kSmemBytes, st>>>(tm_a, tm_b, tm_y, tm_r, p);
   return AQT_LAUNCH_STATUS();
 }
 
-template <int BN, int STAGES, int EW, bool WS, bool BPACK>
+template <int BN, int STAGES, int EW, bool WS, bool BPACK, bool CTA2 = false>
 static int launch_qgemm_cfg(const int8_t* a, const void* b, float* y, int64_t ldy, const GemmParams& p, cudaStream_t st) {
-  if (p.acc_debug != nullptr) return launch_qgemm_inst<BN, STAGES, EW, WS, BPACK, false, true>(a, b, y, ldy, p, st);
-  if (p.small_acc) return launch_qgemm_inst<BN, STAGES, EW, WS, BPACK, true, false>(a, b, y, ldy, p, st);
-  return launch_qgemm_inst<BN, STAGES, EW, WS, BPACK, false, false>(a, b, y, ldy, p, st);
+  if (p.acc_debug != nullptr) return launch_qgemm_inst<BN, STAGES, EW, WS, BPACK, false, true, CTA2>(a, b, y, ldy, p, st);
+  if (p.small_acc) return launch_qgemm_inst<BN, STAGES, EW, WS, BPACK, true, false, CTA2>(a, b, y, ldy, p, st);
+  return launch_qgemm_inst<BN, STAGES, EW, WS, BPACK, false, false, CTA2>(a, b, y, ldy, p, st);
 }
 
 // True if the weight-stationary kernel takes this shape (and can therefore unpack 4-bit weights itself).
@@ -864,6 +975,23 @@ static int launch_qgemm(const int8_t* a, const void* b, bool b_packed, float* y,
     return b_packed ? launch_qgemm_cfg<128, 6, 16, true, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 6, 16, true, false>(a, b, y, ldy, p, st);
   }
   if (b_packed) return AQT_ERR_UNSUPPORTED;
+  const bool deep_k = p.K >= 2048 && !glu;
+  static const char* no_pairs = getenv("AQT_NO_PAIRS");  // tuning aid: one CTA per tile
+  // Pairs pay off only for deep K and many tiles per pair (measured: +4 % at 65 536 x 1024 x 4096,
+  // slower than single CTAs at M = 12 800 .. 25 600); everything else takes one CTA per tile.
+  const bool pairs_ok = deep_k && ceil_div(p.M, 2 * kBM) * ceil_div(p.N, 256) >= 4 * ((sm_count() > 0 ? sm_count() : 148) / 2);
+  if (no_pairs == nullptr && (pairs_ok || getenv("AQT_FORCE_PAIRS") != nullptr) && p.M > kBM) {
+    // CTA pairs on 256-row tiles; width by the number of rounds over the pairs
+    const int pairs = (sm_count() > 0 ? sm_count() : 148) / 2;
+    const int64_t tiles_m2 = ceil_div(p.M, 2 * kBM);
+    const double cost256 = (double)ceil_div(tiles_m2 * ceil_div(p.N, 256), pairs) * (256 + 24);
+    const double cost128 = (double)ceil_div(tiles_m2 * ceil_div(p.N, 128), pairs) * (128 + 24);
+    int bn2 = cost256 <= cost128 ? 256 : 128;
+    static const char* force2 = getenv("AQT_BN");
+    if (force2 != nullptr && (atoi(force2) == 128 || atoi(force2) == 256)) bn2 = atoi(force2);
+    if (bn2 == 256) return deep_k ? launch_qgemm_cfg<256, 6, 4, false, false, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<256, 4, 8, false, false, true>(a, b, y, ldy, p, st);
+    return deep_k ? launch_qgemm_cfg<128, 8, 4, false, false, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 6, 8, false, false, true>(a, b, y, ldy, p, st);
+  }
   int bn = pick_bn(p.M, p.N, glu, sm_count() > 0 ? sm_count() : 148);
   // tuning aid: AQT_BN=64|128|256 in the environment overrides the tile-width heuristic
   static const char* force = getenv("AQT_BN");
@@ -873,7 +1001,6 @@ static int launch_qgemm(const int8_t* a, const void* b, bool b_packed, float* y,
   }
   // Deep K: operand loads bound the tile, so the ring gets the shared memory and four warps run
   // the (short) epilogue.  Shallow K: the epilogue bounds the tile and gets more warps.
-  const bool deep_k = p.K >= 2048 && !glu;
   if (bn == 256) return deep_k ? launch_qgemm_cfg<256, 4, 4, false, false>(a, b, y, ldy, p, st) : launch_qgemm_cfg<256, 3, 16, false, false>(a, b, y, ldy, p, st);
   // every epilogue warp needs at least one 32-column chunk: a GLU tile of width 128 has only
   // 64 output columns, i.e. two chunks per lane quadrant

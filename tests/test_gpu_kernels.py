@@ -135,10 +135,11 @@ def _run_qmatmul(M, N, K, bits_a, bits_w, act, with_bias, with_res, s_x_kind=aqt
     else:
         assert np.isfinite(y).all()
         # float tolerance: 1e-6 relative to the larger of the result and the terms it is formed from
-        z = orc.epilogue_f64(acc_ref, s_x, s_x_kind, s_w, bias, None, 0.0, aqt.ACT_NONE)
-        mag = np.abs(y64)
-        zmag = np.abs(z[:, :n_out]) if z.shape[1] != n_out else np.abs(z)
-        mag = np.maximum(mag, zmag)
+        # (the de-quantized sum acc * s_x * s_w and the bias, which may cancel; the residual)
+        z = orc.epilogue_f64(acc_ref, s_x, s_x_kind, s_w, None, None, 0.0, aqt.ACT_NONE)
+        mag = np.maximum(np.abs(y64), np.abs(z[:, :n_out]))
+        if bias is not None:
+            mag = np.maximum(mag, np.abs(bias[:n_out])[None, :])
         if res is not None:
             mag = np.maximum(mag, np.abs(res))
         assert np.all(np.abs(y - y64) <= 1e-6 * mag + 1e-30), float(np.max(np.abs(y - y64) / (mag + 1e-30)))
@@ -174,6 +175,41 @@ def test_qmatmul_many_tiles_persistent_loop():
     """More tiles than SMs, so every CTA walks several tiles and both accumulator buffers."""
     _run_qmatmul(128 * 40, 2048, 512, 8, 8, aqt.ACT_SWISH, False, False)
     _run_qmatmul(128 * 37 + 5, 512, 2048, 8, 8, aqt.ACT_NONE, False, True)
+
+
+def test_qmatmul_cta_pairs_forced(monkeypatch):
+    """The two-CTA (cta_group::2) form of the streaming kernel, forced on for shapes that would
+    normally take one CTA per tile: ragged M (the second CTA's rows partly or wholly outside),
+    ragged N, GLU halves split across the pair, residual, several tiles per pair."""
+    monkeypatch.setenv("AQT_FORCE_PAIRS", "1")
+    _run_qmatmul(130, 200, 2048, 8, 8, aqt.ACT_NONE, True, True, extremes=True)
+    _run_qmatmul(256, 512, 1024, 8, 4, aqt.ACT_GLU_SWISH, True, True)
+    _run_qmatmul(700, 384, 640, 8, 8, aqt.ACT_SWISH, True, False)
+    _run_qmatmul(256 * 80 + 37, 256, 2048, 8, 8, aqt.ACT_NONE, False, True)
+    _run_qmatmul(512, 1024, 4096, 4, 4, aqt.ACT_NONE, False, False, s_x_kind=aqt.SCALE_TENSOR)
+
+
+def test_qmatmul_cta_pairs_large_deep_k_sampled_rows():
+    """A shape that takes CTA pairs by itself (deep K, many tiles per pair): 19 200 x 1024 x 2048.
+    Accumulators and outputs are compared with the oracle on sampled rows."""
+    M, N, K = 19200, 1024, 2048
+    rng = np.random.default_rng(7)
+    xq = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    wq = rng.integers(-7, 8, (N, K)).astype(np.int8)
+    s_x = rng.uniform(1e-3, 5e-2, M).astype(np.float32)
+    s_w = rng.uniform(1e-4, 5e-3, N).astype(np.float32)
+    res = rng.standard_normal((M, N)).astype(np.float32)
+    acc_d = torch.empty((M, N), dtype=torch.int32, device=DEV)
+    y = aqt.aqt_qmatmul(_dev(xq), _dev(s_x), _dev(orc.pack_int4(wq)), _dev(s_w), None, _dev(res), 0.5, K=K, bits_a=8, bits_w=4,
+                        acc_debug=acc_d)
+    y2 = aqt.aqt_qmatmul(_dev(xq), _dev(s_x), _dev(orc.pack_int4(wq)), _dev(s_w), None, _dev(res), 0.5, K=K, bits_a=8, bits_w=4)
+    _status_ok()
+    rows = sorted(set([0, 127, 128, 255, 256, M - 257, M - 129, M - 1]) | set(rng.integers(0, M, 40).tolist()))
+    acc_ref = orc.int_matmul(xq[rows], wq)
+    assert np.array_equal(acc_d.cpu().numpy()[rows].astype(np.int64), acc_ref)
+    y_ref = orc.epilogue_f32(acc_ref, s_x[rows], orc.SCALE_ROW, s_w, None, res[rows], 0.5, orc.ACT_NONE)
+    assert np.array_equal(y.cpu().numpy()[rows].view(np.uint32), y_ref.view(np.uint32))
+    assert torch.equal(y.view(torch.int32), y2.view(torch.int32))
 
 
 # ----------------------------------------------------------------------------- whole layer

@@ -56,8 +56,10 @@ def _check_layer(spec, cpu_w, x_rows, y_rows, residual_rows=None, rs=1.0, a_scal
         assert np.array_equal(y_rows.view(np.uint32), y_ref.view(np.uint32)), spec.name
     else:
         y64 = orc.epilogue_f64(acc, sx, kind, sw, bias, residual_rows, rs, spec.act)
-        z = np.abs(orc.epilogue_f64(acc, sx, kind, sw, bias, None, 0.0, orc.ACT_NONE))
+        z = np.abs(orc.epilogue_f64(acc, sx, kind, sw, None, None, 0.0, orc.ACT_NONE))   # de-quantized sum, before the bias
         mag = np.maximum(np.abs(y64), z[:, :y64.shape[1]])
+        if bias is not None:
+            mag = np.maximum(mag, np.abs(bias[:y64.shape[1]])[None, :])
         if residual_rows is not None:
             mag = np.maximum(mag, np.abs(residual_rows))
         err = np.abs(y_rows - y64)
