@@ -975,11 +975,17 @@ static int launch_qgemm(const int8_t* a, const void* b, bool b_packed, float* y,
     return b_packed ? launch_qgemm_cfg<128, 6, 16, true, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 6, 16, true, false>(a, b, y, ldy, p, st);
   }
   if (b_packed) return AQT_ERR_UNSUPPORTED;
-  const bool deep_k = p.K >= 2048 && !glu;
+  // "Deep" configuration (four-warp epilogue, longest ring): pays off when K is deep AND every
+  // CTA walks many tiles; with few tiles per CTA the exposed epilogue of the last tile costs more
+  // than the extra ring stages gain (measured at M = 12 800 .. 25 600).
+  const int sms_ = sm_count() > 0 ? sm_count() : 148;
+  bool deep_k = p.K >= 2048 && !glu && ceil_div(p.M, kBM) * ceil_div(p.N, 256) >= 4 * sms_;
+  static const char* deep_env = getenv("AQT_DEEP");  // tuning aid: 0 / 1 overrides the deep-K choice
+  if (deep_env != nullptr && !glu) deep_k = atoi(deep_env) != 0;
   static const char* no_pairs = getenv("AQT_NO_PAIRS");  // tuning aid: one CTA per tile
   // Pairs pay off only for deep K and many tiles per pair (measured: +4 % at 65 536 x 1024 x 4096,
   // slower than single CTAs at M = 12 800 .. 25 600); everything else takes one CTA per tile.
-  const bool pairs_ok = deep_k && ceil_div(p.M, 2 * kBM) * ceil_div(p.N, 256) >= 4 * ((sm_count() > 0 ? sm_count() : 148) / 2);
+  const bool pairs_ok = deep_k;
   if (no_pairs == nullptr && (pairs_ok || getenv("AQT_FORCE_PAIRS") != nullptr) && p.M > kBM) {
     // CTA pairs on 256-row tiles; width by the number of rounds over the pairs
     const int pairs = (sm_count() > 0 ? sm_count() : 148) / 2;
