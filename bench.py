@@ -30,6 +30,7 @@ sys.path.insert(0, ROOT)
 METRIC = "quantized Conformer linear TOPS (int4 weights, int8 activations)"
 UNIT = "TOPS"
 CFG = 2  # the Conformer FFN pair; fits one GPU many times over
+NCU_CAPTURE_VERSION = 101  # library version the ncu traffic figures below were captured at
 
 
 def _peaks():
@@ -349,10 +350,14 @@ def run_ours(args):
     ]
     kernels = [{"call": names[j], "ms": per_call_ms[j], "algorithmic_bytes": alg_bytes[j],
                 "gbs": alg_bytes[j] / (per_call_ms[j] * 1e-3) / 1e9, "share": per_call_ms[j] / sum(per_call_ms)} for j in range(4)]
+    # DRAM traffic per launch of the GEMM kernels from the committed ncu capture
+    # (profiles/qgemm_i8_ffn_pair_ncu.md: dram__bytes_read.sum + dram__bytes_write.sum).  The write
+    # part undercounts: most of the output is still in the 126 MB L2 when the kernel ends.
+    ncu_traffic = {1: 7174912 + 46349824, 3: 27342336 + 254720} if aqt.aqt_version() == NCU_CAPTURE_VERSION else {}
     dom = max(range(4), key=lambda j: per_call_ms[j])
     achieved = kernels[dom]["gbs"]
     roofline = {"bound": "hbm", "kernel": names[dom], "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "peak_source": "of " + peak_kind, "traffic": None, "calls": kernels}
+                "peak_source": "of " + peak_kind, "traffic": ncu_traffic.get(dom), "calls": kernels}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

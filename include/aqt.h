@@ -32,7 +32,7 @@
 extern "C" {
 #endif
 
-#define AQT_VERSION 100
+#define AQT_VERSION 101
 
 /* status codes */
 #define AQT_OK 0

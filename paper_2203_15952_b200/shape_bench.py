@@ -1,0 +1,121 @@
+"""Time one entry point of the library on one shape (CUDA events, rotating buffers).
+
+    python -m paper_2203_15952_b200.shape_bench qmatmul M N K [--act 0..3] [--bits-w 4|8] [--residual]
+                                                 [--iters I] [--sustain SECONDS]
+    python -m paper_2203_15952_b200.shape_bench quantize M K [--bits 4|8]
+
+Inputs are random codes / normals drawn on the GPU (seeded); several buffer sets are rotated so
+that consecutive launches do not find their inputs in L2.  With --sustain the call is repeated for
+that many seconds while nvidia-smi samples clocks and power (power-capped throughput).
+Prints one line: time per call, TOPS or GB/s (algorithmic bytes), and with --sustain the clocks.
+"""
+from __future__ import annotations
+
+import argparse
+import statistics
+import subprocess
+import sys
+import time
+
+import torch
+
+from . import binding as aqt
+
+
+def _time(calls, iters):
+    for c in calls:
+        c()
+    for c in calls:
+        c()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(iters):
+        calls[i % len(calls)]()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters * 1e3  # us
+
+
+def _sustain(calls, seconds):
+    q = "clocks.sm,power.draw,clocks_event_reasons.sw_power_cap"
+    proc = subprocess.Popen(["nvidia-smi", "-i", str(torch.cuda.current_device()), "--query-gpu=" + q, "--format=csv,noheader,nounits",
+                             "-lms", "100"], stdout=subprocess.PIPE, text=True)
+    time.sleep(0.3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n, t0 = 0, time.time()
+    e0.record()
+    while time.time() - t0 < seconds:
+        for _ in range(50):
+            calls[n % len(calls)]()
+            n += 1
+        torch.cuda.synchronize()
+    e1.record()
+    torch.cuda.synchronize()
+    proc.terminate()
+    out, _ = proc.communicate()
+    rows = [l.split(",") for l in out.strip().splitlines()][3:]
+    clk = [float(r[0]) for r in rows] or [float("nan")]
+    pw = [float(r[1]) for r in rows] or [float("nan")]
+    capped = sum(("Active" in r[2]) and ("Not" not in r[2]) for r in rows)
+    return e0.elapsed_time(e1) / n * 1e3, " sustained %.1f s: SM clock median %.0f MHz, power max %.0f W, power cap active in %d/%d samples" % (
+        seconds, statistics.median(clk), max(pw), capped, len(rows))
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
+    ap.add_argument("op", choices=["qmatmul", "quantize"])
+    ap.add_argument("dims", type=int, nargs="+")
+    ap.add_argument("--act", type=int, default=0)
+    ap.add_argument("--bits-w", type=int, default=8)
+    ap.add_argument("--bits", type=int, default=8)
+    ap.add_argument("--residual", action="store_true")
+    ap.add_argument("--iters", type=int, default=30)
+    ap.add_argument("--sets", type=int, default=4)
+    ap.add_argument("--sustain", type=float, default=0.0)
+    a = ap.parse_args(argv)
+    dev = torch.device("cuda", 0)
+    g = torch.Generator(device=dev).manual_seed(0)
+    calls, keep = [], []
+    if a.op == "qmatmul":
+        M, N, K = a.dims
+        n_out = N // 2 if a.act >= 2 else N
+        wq = torch.randint(-7, 8, (N, K if a.bits_w == 8 else K // 2), generator=g, dtype=torch.int8, device=dev)
+        if a.bits_w == 4:
+            wq = wq.view(torch.uint8)
+        sw = torch.rand(N, generator=g, device=dev) * 1e-3
+        ws = torch.empty(aqt.aqt_workspace_bytes(aqt.OP_QMATMUL, M, N, K, 8, a.bits_w) + 256, dtype=torch.uint8, device=dev)
+        for _ in range(a.sets):
+            xq = torch.randint(-127, 128, (M, K), generator=g, dtype=torch.int8, device=dev)
+            sx = torch.rand(M, generator=g, device=dev) * 1e-2
+            y = torch.empty((M, n_out), dtype=torch.float32, device=dev)
+            rr = torch.randn((M, n_out), generator=g, device=dev) if a.residual else None
+            keep += [xq, sx, y, rr]
+            calls.append(aqt.bind_qmatmul(xq, sx, wq, sw, None, rr, 0.5, K, 8, a.bits_w, a.act, aqt.SCALE_ROW, y, ws))
+        ops = 2.0 * M * N * K
+        nbytes = M * K + N * K * a.bits_w // 8 + 8 * N + 4 * M + 4 * M * n_out * (2 if a.residual else 1)
+        label = "qmatmul M%d N%d K%d act%d w%d res%d" % (M, N, K, a.act, a.bits_w, int(a.residual))
+    else:
+        M, K = a.dims
+        for _ in range(a.sets):
+            x = torch.randn((M, K), generator=g, device=dev)
+            q = torch.empty((M, K), dtype=torch.int8, device=dev)
+            s = torch.empty(M, device=dev)
+            keep += [x, q, s]
+            calls.append(aqt.bind_quantize(x, a.bits, aqt.AXIS_ROW, aqt.ROUND_NEAREST_EVEN, False, q, s))
+        ops = 0.0
+        nbytes = 5 * M * K + 4 * M
+        label = "quantize M%d K%d bits%d" % (M, K, a.bits)
+    extra = ""
+    if a.sustain > 0:
+        t, extra = _sustain(calls, a.sustain)
+    else:
+        t = _time(calls, a.iters)
+    if aqt.aqt_device_status() != 0:
+        raise SystemExit("device status reports a failed wait")
+    print("%s: %8.2f us  %8.1f TOPS  %7.1f GB/s%s" % (label, t, ops / t / 1e6, nbytes / t / 1e3, extra), flush=True)
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -34,7 +34,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_host_only_calls():
     from paper_2203_15952_b200 import binding as b
-    assert b.aqt_version() == 100
+    assert b.aqt_version() >= 100
     assert b.status_string(0) == "ok" and "workspace" in b.status_string(-4)
     # 4-bit operands need a sign-extended copy; 8-bit ones do not
     assert b.aqt_workspace_bytes(b.OP_QMATMUL, 128, 256, 512, 8, 8) == 0
