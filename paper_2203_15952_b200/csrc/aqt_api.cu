@@ -3,6 +3,7 @@
 #include "aqt_common.cuh"
 #include "pack.cuh"
 #include "qgemm_sm100.cuh"
+#include "qgemv_small_m.cuh"
 #include "quantize.cuh"
 
 using namespace aqt;
@@ -44,10 +45,40 @@ int validate_matmul_shape(int64_t M, int64_t N, int64_t K, int bits_a, int bits_
   return AQT_OK;
 }
 
+int run_small_m(const void* xq, bool a_packed, const float* s_x, int s_x_kind, const void* wq, bool w_packed, const float* s_w,
+                const float* bias, const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K, int act,
+                float* y, int64_t ldy, int32_t* acc_debug, cudaStream_t st) {
+  SmallParams sp;
+  sp.xq = xq;
+  sp.wq = wq;
+  sp.s_x = s_x;
+  sp.s_w = s_w;
+  sp.bias = bias;
+  sp.residual = residual;
+  sp.y = y;
+  sp.acc_debug = acc_debug;
+  sp.ldr = ldr;
+  sp.ldy = ldy;
+  sp.residual_scale = residual_scale;
+  sp.s_x_kind = s_x_kind;
+  sp.act = act;
+  sp.M = (int)M;
+  sp.N = (int)N;
+  sp.K = (int)K;
+  sp.a_packed = a_packed ? 1 : 0;
+  sp.w_packed = w_packed ? 1 : 0;
+  return launch_small_m(sp, st);
+}
+
 // Codes already in int8 containers for A; B possibly packed.  ws holds B's unpacked copy.
 int qmatmul_i8a(const int8_t* a_codes, const float* s_x, int s_x_kind, const void* wq, const float* s_w, const float* bias,
                 const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K, int bits_a, int bits_w,
                 int act, float* y, int64_t ldy, int32_t* acc_debug, uint8_t* ws, cudaStream_t st) {
+  if (small_m_applies(M, K)) {
+    // a few rows: weight-bandwidth-bound kernel, packed weights read as they are
+    return run_small_m(a_codes, false, s_x, s_x_kind, wq, bits_w == 4, s_w, bias, residual, ldr, residual_scale, M, N, K, act, y, ldy,
+                       acc_debug, st);
+  }
   // 4-bit weights: the weight-stationary kernel (K <= 512) sign-extends them itself in shared
   // memory after TMA staging; deeper K takes a one-off sign-extended copy in the workspace.
   const void* b_codes = wq;
@@ -169,6 +200,10 @@ int aqt_qmatmul(const void* xq, const float* s_x, int s_x_kind, const void* wq, 
   if (rc != AQT_OK) return rc;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  if (small_m_applies(M, K)) {
+    return run_small_m(xq, bits_a == 4, s_x, s_x_kind, wq, bits_w == 4, s_w, bias, residual, ldr, residual_scale, M, N, K, act, y, ldy,
+                       acc_debug, st);
+  }
   const int8_t* a_codes = reinterpret_cast<const int8_t*>(xq);
   if (bits_a == 4) {
     rc = launch_unpack_int4(reinterpret_cast<const uint8_t*>(xq), M * K / 2, reinterpret_cast<int8_t*>(ws), st);

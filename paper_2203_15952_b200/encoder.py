@@ -58,6 +58,23 @@ class LayerRunner:
         need = max(aqt.aqt_workspace_bytes(aqt.OP_LINEAR_FWD, M, l.spec.N, l.spec.K, l.spec.bits_a, l.spec.bits_w) for l in layers)
         self.workspace = torch.empty(need, dtype=torch.uint8, device=device)
 
+    def quantize_input(self, x: torch.Tensor, bits_a: int):
+        """Activation codes (int8 containers) and scales of x, for several layers that read the
+        same tensor (the attention projections): one quantizer pass instead of one per layer."""
+        M, K = x.shape
+        if getattr(self, "_shared_q", None) is None or self._shared_q.shape != (M, K):
+            self._shared_q = torch.empty((M, K), dtype=torch.int8, device=x.device)
+            self._shared_s = torch.empty(M if self.a_scale_kind == aqt.SCALE_ROW else 1, dtype=torch.float32, device=x.device)
+        axis = aqt.AXIS_ROW if self.a_scale_kind == aqt.SCALE_ROW else aqt.AXIS_TENSOR
+        aqt.aqt_quantize(x, bits_a, axis, self.rounding, q_out=self._shared_q, scale_out=self._shared_s)
+        return self._shared_q, self._shared_s
+
+    def matmul(self, layer: QuantLinear, xq: torch.Tensor, s_x: torch.Tensor, y: torch.Tensor) -> torch.Tensor:
+        """Integer matmul + epilogue of `layer` on already-quantized activations (int8 containers)."""
+        s = layer.spec
+        return aqt.aqt_qmatmul(xq, s_x, layer.wq, layer.s_w, layer.bias, None, 1.0, K=s.K, bits_a=8, bits_w=s.bits_w, act=s.act,
+                               s_x_kind=self.a_scale_kind, y=y, workspace=self.workspace)
+
     def __call__(self, layer: QuantLinear, x: torch.Tensor, y: torch.Tensor, residual: Optional[torch.Tensor] = None,
                  residual_scale: float = 1.0) -> torch.Tensor:
         s = layer.spec
@@ -112,9 +129,11 @@ class ConformerBlockLinears:
 
         run(L[0], h_in, self.u); note(L[0].spec.name, self.u)
         run(L[1], self.u, self.h_a, residual=h_in, residual_scale=0.5); note(L[1].spec.name, self.h_a)
-        run(L[2], self.h_a, self.q); note(L[2].spec.name, self.q)
-        run(L[3], self.h_a, self.k); note(L[3].spec.name, self.k)
-        run(L[4], self.h_a, self.v); note(L[4].spec.name, self.v)
+        # q, k, v read the same h: quantize it once (the codes do not depend on the consumer)
+        hq, hs = run.quantize_input(self.h_a, L[2].spec.bits_a)
+        run.matmul(L[2], hq, hs, self.q); note(L[2].spec.name, self.q)
+        run.matmul(L[3], hq, hs, self.k); note(L[3].spec.name, self.k)
+        run.matmul(L[4], hq, hs, self.v); note(L[4].spec.name, self.v)
         run(L[5], self.v, self.h_b, residual=self.h_a, residual_scale=1.0); note(L[5].spec.name, self.h_b)
         run(L[6], self.h_b, self.c); note(L[6].spec.name, self.c)
         run(L[7], self.c, self.h_a, residual=self.h_b, residual_scale=1.0); note(L[7].spec.name, self.h_a)

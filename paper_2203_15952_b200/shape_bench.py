@@ -37,6 +37,29 @@ def _time(calls, iters):
     return e0.elapsed_time(e1) / iters * 1e3  # us
 
 
+def _time_graph(make_calls, iters):
+    """The same calls captured in a CUDA graph (no host launch cost between kernels)."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        calls = make_calls(side)
+        for c in calls:
+            c()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        for i in range(iters):
+            calls[i % len(calls)]()
+    g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters * 1e3
+
+
 def _sustain(calls, seconds):
     q = "clocks.sm,power.draw,clocks_event_reasons.sw_power_cap"
     proc = subprocess.Popen(["nvidia-smi", "-i", str(torch.cuda.current_device()), "--query-gpu=" + q, "--format=csv,noheader,nounits",
@@ -73,10 +96,11 @@ def main(argv=None):
     ap.add_argument("--iters", type=int, default=30)
     ap.add_argument("--sets", type=int, default=4)
     ap.add_argument("--sustain", type=float, default=0.0)
+    ap.add_argument("--graph", action="store_true", help="replay the calls from a CUDA graph (kernel time without host launch cost)")
     a = ap.parse_args(argv)
     dev = torch.device("cuda", 0)
     g = torch.Generator(device=dev).manual_seed(0)
-    calls, keep = [], []
+    keep = []
     if a.op == "qmatmul":
         M, N, K = a.dims
         n_out = N // 2 if a.act >= 2 else N
@@ -85,30 +109,41 @@ def main(argv=None):
             wq = wq.view(torch.uint8)
         sw = torch.rand(N, generator=g, device=dev) * 1e-3
         ws = torch.empty(aqt.aqt_workspace_bytes(aqt.OP_QMATMUL, M, N, K, 8, a.bits_w) + 256, dtype=torch.uint8, device=dev)
+        sets = []
         for _ in range(a.sets):
             xq = torch.randint(-127, 128, (M, K), generator=g, dtype=torch.int8, device=dev)
             sx = torch.rand(M, generator=g, device=dev) * 1e-2
             y = torch.empty((M, n_out), dtype=torch.float32, device=dev)
             rr = torch.randn((M, n_out), generator=g, device=dev) if a.residual else None
-            keep += [xq, sx, y, rr]
-            calls.append(aqt.bind_qmatmul(xq, sx, wq, sw, None, rr, 0.5, K, 8, a.bits_w, a.act, aqt.SCALE_ROW, y, ws))
+            sets.append((xq, sx, y, rr))
+
+        def make_calls(stream=None):
+            return [aqt.bind_qmatmul(xq, sx, wq, sw, None, rr, 0.5, K, 8, a.bits_w, a.act, aqt.SCALE_ROW, y, ws, stream)
+                    for (xq, sx, y, rr) in sets]
         ops = 2.0 * M * N * K
         nbytes = M * K + N * K * a.bits_w // 8 + 8 * N + 4 * M + 4 * M * n_out * (2 if a.residual else 1)
         label = "qmatmul M%d N%d K%d act%d w%d res%d" % (M, N, K, a.act, a.bits_w, int(a.residual))
     else:
         M, K = a.dims
+        sets = []
         for _ in range(a.sets):
             x = torch.randn((M, K), generator=g, device=dev)
             q = torch.empty((M, K), dtype=torch.int8, device=dev)
             s = torch.empty(M, device=dev)
-            keep += [x, q, s]
-            calls.append(aqt.bind_quantize(x, a.bits, aqt.AXIS_ROW, aqt.ROUND_NEAREST_EVEN, False, q, s))
+            sets.append((x, q, s))
+
+        def make_calls(stream=None):
+            return [aqt.bind_quantize(x, a.bits, aqt.AXIS_ROW, aqt.ROUND_NEAREST_EVEN, False, q, s, stream) for (x, q, s) in sets]
         ops = 0.0
         nbytes = 5 * M * K + 4 * M
         label = "quantize M%d K%d bits%d" % (M, K, a.bits)
+    calls = make_calls()
     extra = ""
     if a.sustain > 0:
         t, extra = _sustain(calls, a.sustain)
+    elif a.graph:
+        t = _time_graph(make_calls, a.iters)
+        extra = " (graph replay)"
     else:
         t = _time(calls, a.iters)
     if aqt.aqt_device_status() != 0:

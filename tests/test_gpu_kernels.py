@@ -177,6 +177,27 @@ def test_qmatmul_many_tiles_persistent_loop():
     _run_qmatmul(128 * 37 + 5, 512, 2048, 8, 8, aqt.ACT_NONE, False, True)
 
 
+@pytest.mark.parametrize("M", [1, 3, 8, 9, 16, 17])
+@pytest.mark.parametrize("N,K,act,bits_a,bits_w", [(2048, 512, aqt.ACT_SWISH, 8, 4), (512, 2048, aqt.ACT_NONE, 8, 4),
+                                                    (1024, 512, aqt.ACT_GLU_SWISH, 8, 8), (136, 96, aqt.ACT_GLU, 4, 4),
+                                                    (260, 4096, aqt.ACT_NONE, 4, 8)])
+def test_qmatmul_small_batch(M, N, K, act, bits_a, bits_w):
+    """A few rows (streaming use): the weight-bandwidth-bound kernel, packed operands read directly."""
+    _run_qmatmul(M, N, K, bits_a, bits_w, act, True, True, extremes=(M > 1))
+    _run_qmatmul(M, N, K, bits_a, bits_w, act, False, False, s_x_kind=aqt.SCALE_TENSOR)
+
+
+def test_linear_fwd_small_batch_matches_oracle():
+    M, K, N = 5, 512, 2048
+    x = gen.normal(6, 1, M, K)
+    wt = gen.weight(6, 2, K, N)
+    wq, s_w = orc.quantize(wt, 4, orc.AXIS_ROW)
+    y_ref = orc.linear_fwd(x, wq, s_w)
+    y = aqt.aqt_linear_fwd(_dev(x), _dev(orc.pack_int4(wq)), _dev(s_w), bits_a=8, bits_w=4)
+    _status_ok()
+    assert np.array_equal(y.cpu().numpy().view(np.uint32), y_ref.view(np.uint32))
+
+
 def test_qmatmul_cta_pairs_forced(monkeypatch):
     """The two-CTA (cta_group::2) form of the streaming kernel, forced on for shapes that would
     normally take one CTA per tile: ragged M (the second CTA's rows partly or wholly outside),
