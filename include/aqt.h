@@ -190,6 +190,15 @@ size_t aqt_workspace_bytes(int op, int64_t M, int64_t N, int64_t K, int bits_a, 
  */
 int aqt_device_status(void* stream, int* status_out);
 
+/*
+ * aqt_selftest_bounded_wait -- exercises the failure path of the kernels' bounded waits without
+ * hanging anything: one CTA waits, for at most limit_ns (1 .. 10^9), on a barrier that nothing
+ * signals.  The wait gives up, the kernel returns normally, *gave_up_dev (device int) is set to 1
+ * and the device status word to AQT_ERR_TIMEOUT, which the next aqt_device_status() reports and
+ * clears.  (The paper has no counterpart: this is the library's own fault-reporting check.)
+ */
+int aqt_selftest_bounded_wait(uint64_t limit_ns, int* gave_up_dev, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,7 +23,8 @@ ACT_NONE, ACT_SWISH, ACT_GLU, ACT_GLU_SWISH = 0, 1, 2, 3
 OP_QMATMUL, OP_LINEAR_FWD = 1, 2
 
 EXPORTS = ("aqt_version", "aqt_status_string", "aqt_quantize", "aqt_pack_int4", "aqt_unpack_int4", "aqt_qmatmul",
-           "aqt_linear_fwd", "aqt_linear_fwd_host", "aqt_workspace_bytes", "aqt_device_status", "aqt_qmatmul_w4_noalloc")
+           "aqt_linear_fwd", "aqt_linear_fwd_host", "aqt_workspace_bytes", "aqt_device_status", "aqt_qmatmul_w4_noalloc",
+           "aqt_selftest_bounded_wait")
 NOALLOC_MAX_WEIGHT_BYTES = 4 << 20
 
 
@@ -127,6 +128,15 @@ def aqt_device_status(stream=None) -> int:
     out = ctypes.c_int(0)
     _check("aqt_device_status", lib().aqt_device_status(_stream(stream), ctypes.byref(out)))
     return out.value
+
+
+def aqt_selftest_bounded_wait(limit_ns: int = 1_000_000, stream=None) -> bool:
+    """Runs the bounded-wait self-test; True if the wait gave up as it must.  Leaves
+    AQT_ERR_TIMEOUT in the device status word for the next aqt_device_status()."""
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    _check("aqt_selftest_bounded_wait", lib().aqt_selftest_bounded_wait(ctypes.c_uint64(limit_ns), _ptr(flag), _stream(stream)))
+    torch.cuda.synchronize()
+    return bool(flag.item() == 1)
 
 
 def aqt_quantize(x: torch.Tensor, bits: int, axis: int = AXIS_ROW, rounding: int = ROUND_NEAREST_EVEN,

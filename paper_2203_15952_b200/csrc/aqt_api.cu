@@ -333,6 +333,14 @@ int aqt_qmatmul_w4_noalloc(const int8_t* xq, const float* s_x, int s_x_kind, con
                      scratch, reinterpret_cast<cudaStream_t>(stream));
 }
 
+int aqt_selftest_bounded_wait(uint64_t limit_ns, int* gave_up_dev, void* stream) {
+  if (gave_up_dev == nullptr || limit_ns == 0 || limit_ns > 1000000000ull) return AQT_ERR_BADARG;
+  int rc = check_device();
+  if (rc != AQT_OK) return rc;
+  bounded_wait_selftest_kernel<<<1, 64, 0, reinterpret_cast<cudaStream_t>(stream)>>>(limit_ns, gave_up_dev);
+  return AQT_LAUNCH_STATUS();
+}
+
 int aqt_device_status(void* stream, int* status_out) {
   if (status_out == nullptr) return AQT_ERR_BADARG;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);

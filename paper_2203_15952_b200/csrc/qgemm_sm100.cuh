@@ -113,12 +113,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 
 // Bounded wait.  Returns false if the CTA is aborting or the limit passed (and then sets both
 // the CTA's abort flag and the device status word).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint64_t t_start) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint64_t t_start,
+                                          uint64_t limit_ns = kWaitLimitNs) {
   for (uint32_t spin = 1;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((spin & 0xFF) == 0) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t_start > kWaitLimitNs) {
+      if (global_timer_ns() - t_start > limit_ns) {
         *abort_flag = 1;
         atomicExch(&g_device_status, AQT_ERR_TIMEOUT);
         return false;
@@ -811,6 +812,23 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     if (CTA2) tmem_dealloc_pair(tmem_base, Cfg::kTmemCols);
     else tmem_dealloc(tmem_base, Cfg::kTmemCols);
   }
+}
+
+// Self-test of the bounded wait: one CTA waits on an mbarrier that nothing ever arrives on, with
+// a short limit.  The wait must give up, record AQT_ERR_TIMEOUT in the device status word and let
+// the kernel return normally (the context stays usable).
+__global__ void bounded_wait_selftest_kernel(uint64_t limit_ns, int* gave_up) {
+  __shared__ uint64_t never_signalled;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&never_signalled), 1);
+    fence_barrier_init();
+  }
+  __syncthreads();
+  const bool ok = mbar_wait(smem_u32(&never_signalled), 0, &abort_flag, global_timer_ns(), limit_ns);
+  __syncthreads();
+  if (threadIdx.x == 0) *gave_up = ok ? 0 : 1;
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -213,6 +213,72 @@ __global__ void __launch_bounds__(kQuantThreads) quantize_with_scales_kernel(
   }
 }
 
+// Whole-tensor scale for small tensors in one launch: one CTA finds the abs-max, forms the scale
+// and quantizes (the tensor is re-read from L1/L2).  Replaces the four-launch path below where
+// launch latency, not bandwidth, is the cost (e.g. a [64, 256] activation).
+constexpr int kSmallTensorElems = 1 << 16;
+template <int ROUNDING, bool PACK>
+__global__ void __launch_bounds__(1024) quantize_tensor_small_kernel(const float* __restrict__ x, int rows, int cols, int64_t ld,
+                                                                      int qmax, void* __restrict__ q_out,
+                                                                      float* __restrict__ scale_out) {
+  __shared__ float warp_max[32];
+  const int total = rows * cols;
+  // dense, aligned tensors of up to 16 K elements stay in registers: all loads are issued at once
+  const bool in_regs = (ld == cols) && (total % 4 == 0) && (total <= 4 * 4 * 1024) &&
+                       ((reinterpret_cast<uintptr_t>(x) & 15) == 0) && ((reinterpret_cast<uintptr_t>(q_out) & 3) == 0);
+  float4 v[4];
+  float amax = 0.0f;
+  if (in_regs) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int idx = threadIdx.x + i * 1024;
+      v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (idx < total / 4) v[i] = __ldg(reinterpret_cast<const float4*>(x) + idx);
+      amax = fmaxf(amax, fmaxf(fmaxf(fabsf(v[i].x), fabsf(v[i].y)), fmaxf(fabsf(v[i].z), fabsf(v[i].w))));
+    }
+  } else {
+    for (int i = threadIdx.x; i < total; i += blockDim.x) {
+      const int r = i / cols, j = i - r * cols;
+      amax = fmaxf(amax, fabsf(x[(int64_t)r * ld + j]));
+    }
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
+  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = amax;
+  __syncthreads();
+  amax = 0.0f;
+  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) amax = fmaxf(amax, warp_max[w]);
+  const ScaleCtx c = make_scale_ctx(amax, qmax);
+  if (threadIdx.x == 0) scale_out[0] = c.s;
+  if (in_regs) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int idx = threadIdx.x + i * 1024;
+      if (idx < total / 4) {
+        const int a = quantize_elem<ROUNDING>(v[i].x, c, qmax), b = quantize_elem<ROUNDING>(v[i].y, c, qmax);
+        const int cc = quantize_elem<ROUNDING>(v[i].z, c, qmax), d = quantize_elem<ROUNDING>(v[i].w, c, qmax);
+        if (PACK) reinterpret_cast<uint16_t*>(q_out)[idx] = (uint16_t)pack4_i4(a, b, cc, d);
+        else reinterpret_cast<uint32_t*>(q_out)[idx] = pack4_i8(a, b, cc, d);
+      }
+    }
+    return;
+  }
+  const int pairs_per_row = (cols + 1) / 2;
+  for (int i = threadIdx.x; i < rows * pairs_per_row; i += blockDim.x) {
+    const int r = i / pairs_per_row, p = i - r * pairs_per_row;
+    const int j0 = 2 * p, j1 = 2 * p + 1;
+    const int a = quantize_elem<ROUNDING>(x[(int64_t)r * ld + j0], c, qmax);
+    const int b = j1 < cols ? quantize_elem<ROUNDING>(x[(int64_t)r * ld + j1], c, qmax) : 0;
+    if (PACK) {
+      reinterpret_cast<uint8_t*>(q_out)[(int64_t)r * (cols / 2) + p] = (uint8_t)((a & 0xF) | ((b & 0xF) << 4));
+    } else {
+      int8_t* q = reinterpret_cast<int8_t*>(q_out) + (int64_t)r * cols;
+      q[j0] = (int8_t)a;
+      if (j1 < cols) q[j1] = (int8_t)b;
+    }
+  }
+}
+
 template <int ROUNDING, bool PACK>
 static int launch_quantize_rows(const float* x, int64_t rows, int64_t cols, int64_t ld, int qmax, void* q_out,
                                 float* scale_out, cudaStream_t st) {
@@ -243,6 +309,10 @@ static int launch_quantize_axis(const float* x, int64_t rows, int64_t cols, int6
                                 float* scale_out, cudaStream_t st) {
   if (axis == AQT_AXIS_ROW) return launch_quantize_rows<ROUNDING, PACK>(x, rows, cols, ld, qmax, q_out, scale_out, st);
   const bool per_col = axis == AQT_AXIS_COL;
+  if (!per_col && rows * cols <= kSmallTensorElems) {
+    quantize_tensor_small_kernel<ROUNDING, PACK><<<1, 1024, 0, st>>>(x, (int)rows, (int)cols, ld, qmax, q_out, scale_out);
+    return AQT_LAUNCH_STATUS();
+  }
   const int64_t n_scale = per_col ? cols : 1;
   AQT_RETURN_IF_CUDA(cudaMemsetAsync(scale_out, 0, (size_t)n_scale * sizeof(float), st));
   if (per_col) {

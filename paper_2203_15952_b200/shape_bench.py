@@ -3,6 +3,7 @@
     python -m paper_2203_15952_b200.shape_bench qmatmul M N K [--act 0..3] [--bits-w 4|8] [--residual]
                                                  [--iters I] [--sustain SECONDS]
     python -m paper_2203_15952_b200.shape_bench quantize M K [--bits 4|8]
+    python -m paper_2203_15952_b200.shape_bench linear M N K [--act ..] [--bits-w ..] [--bits 4|8] [--per-tensor]
 
 Inputs are random codes / normals drawn on the GPU (seeded); several buffer sets are rotated so
 that consecutive launches do not find their inputs in L2.  With --sustain the call is repeated for
@@ -87,12 +88,13 @@ def _sustain(calls, seconds):
 
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("op", choices=["qmatmul", "quantize"])
+    ap.add_argument("op", choices=["qmatmul", "quantize", "linear"])
     ap.add_argument("dims", type=int, nargs="+")
     ap.add_argument("--act", type=int, default=0)
     ap.add_argument("--bits-w", type=int, default=8)
     ap.add_argument("--bits", type=int, default=8)
     ap.add_argument("--residual", action="store_true")
+    ap.add_argument("--per-tensor", action="store_true", help="linear: one activation scale for the whole tensor")
     ap.add_argument("--iters", type=int, default=30)
     ap.add_argument("--sets", type=int, default=4)
     ap.add_argument("--sustain", type=float, default=0.0)
@@ -123,6 +125,24 @@ def main(argv=None):
         ops = 2.0 * M * N * K
         nbytes = M * K + N * K * a.bits_w // 8 + 8 * N + 4 * M + 4 * M * n_out * (2 if a.residual else 1)
         label = "qmatmul M%d N%d K%d act%d w%d res%d" % (M, N, K, a.act, a.bits_w, int(a.residual))
+    elif a.op == "linear":
+        M, N, K = a.dims
+        n_out = N // 2 if a.act >= 2 else N
+        wq = torch.randint(-7, 8, (N, K if a.bits_w == 8 else K // 2), generator=g, dtype=torch.int8, device=dev)
+        if a.bits_w == 4:
+            wq = wq.view(torch.uint8)
+        sw = torch.rand(N, generator=g, device=dev) * 1e-3
+        ws = torch.empty(aqt.aqt_workspace_bytes(aqt.OP_LINEAR_FWD, M, N, K, a.bits, a.bits_w) + 256, dtype=torch.uint8, device=dev)
+        kind = aqt.SCALE_TENSOR if a.per_tensor else aqt.SCALE_ROW
+        sets = [(torch.randn((M, K), generator=g, device=dev), torch.empty((M, n_out), dtype=torch.float32, device=dev))
+                for _ in range(a.sets)]
+
+        def make_calls(stream=None):
+            return [aqt.bind_linear_fwd(x, wq, sw, None, None, 1.0, a.bits, a.bits_w, kind, aqt.ROUND_NEAREST_EVEN, a.act, y, ws, stream)
+                    for (x, y) in sets]
+        ops = 2.0 * M * N * K
+        nbytes = 4 * M * K + N * K * a.bits_w // 8 + 8 * N + 4 * M * n_out
+        label = "linear M%d N%d K%d act%d a%d w%d %s" % (M, N, K, a.act, a.bits, a.bits_w, "per-tensor" if a.per_tensor else "per-row")
     else:
         M, K = a.dims
         sets = []

@@ -268,6 +268,18 @@ def test_linear_fwd_host_buffers():
     assert np.all(np.abs(y - y_ref) <= 1e-6 * np.maximum(np.abs(y_ref), 1e-3) + 1e-30)
 
 
+def test_bounded_wait_gives_up_and_reports_timeout():
+    """A wait on a barrier nothing signals runs out after its limit: the kernel returns, the
+    status word says AQT_ERR_TIMEOUT once, and the context keeps working."""
+    assert aqt.aqt_device_status() == 0
+    assert aqt.aqt_selftest_bounded_wait(2_000_000) is True
+    assert aqt.aqt_device_status() == -6
+    assert aqt.aqt_device_status() == 0                      # cleared by the read
+    x = torch.ones((4, 32), dtype=torch.float32, device=DEV)
+    q, s = aqt.aqt_quantize(x, 8, aqt.AXIS_ROW)              # the context is still usable
+    assert int(q.min()) == 127 and aqt.aqt_device_status() == 0
+
+
 def test_status_codes_on_device():
     x = torch.zeros((128, 128), dtype=torch.int8, device=DEV)
     s = torch.ones(128, dtype=torch.float32, device=DEV)
