@@ -151,7 +151,7 @@ def run_reference(args):
     ops_per_row = sum(2 * s.N * s.K for s in specs)
     t_probe = _oracle_time_rows(w, specs, wts, 128)
     # a step = a row sample sized so that warm-up + steps finish within about two minutes
-    per_step_budget = 100.0 / max(1, args.steps + args.warmup)
+    per_step_budget = args.ref_budget_s / max(1, args.steps + args.warmup)
     rows = int(max(64, min(w.M, 128 * per_step_budget / max(t_probe, 1e-6)))) // 64 * 64
     for i in range(args.warmup):
         _oracle_time_rows(w, specs, wts, rows, offset=i * rows)
@@ -444,6 +444,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ref-budget-s", type=float, default=100.0, help="--impl reference: CPU seconds for warm-up + steps together")
     ap.add_argument("--no-encoder", action="store_true", help="skip the 17-block encoder-stack frames/s leg")
     ap.add_argument("--no-graph", action="store_true", help="launch every step call by call (no CUDA graph replay)")
     args = ap.parse_args()
