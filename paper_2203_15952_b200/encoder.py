@@ -55,7 +55,7 @@ class LayerRunner:
     def __init__(self, M: int, layers: List[QuantLinear], device, a_scale_kind: int = aqt.SCALE_ROW,
                  rounding: int = aqt.ROUND_NEAREST_EVEN):
         self.M, self.device, self.a_scale_kind, self.rounding = M, device, a_scale_kind, rounding
-        need = max(aqt.aqt_workspace_bytes(aqt.OP_LINEAR_FWD, M, l.spec.N, l.spec.K, l.spec.bits_a, l.spec.bits_w) for l in layers)
+        need = max(aqt.aqt_workspace_bytes(aqt.OP_LINEAR_FWD, M, 3 * l.spec.N, l.spec.K, l.spec.bits_a, l.spec.bits_w) for l in layers)
         self.workspace = torch.empty(need, dtype=torch.uint8, device=device)
 
     def quantize_input(self, x: torch.Tensor, bits_a: int):
@@ -110,9 +110,10 @@ class ConformerBlockLinears:
         self.run = LayerRunner(M, layers_for_sizing, device, **kw)
         f32 = dict(dtype=torch.float32, device=device)
         self.u = torch.empty((M, ff), **f32)
-        self.q = torch.empty((M, d), **f32)
-        self.k = torch.empty((M, d), **f32)
-        self.v = torch.empty((M, d), **f32)
+        # q, k, v come out of one GEMM over the concatenated projection weights (N = 3d)
+        self.qkv = torch.empty((M, 3 * d), **f32)
+        self.q, self.k, self.v = self.qkv[:, 0:d], self.qkv[:, d:2 * d], self.qkv[:, 2 * d:3 * d]
+        self._qkv_weights: Dict[int, tuple] = {}
         self.c = torch.empty((M, d), **f32)
         self.h_a = torch.empty((M, d), **f32)
         self.h_b = torch.empty((M, d), **f32)
@@ -129,17 +130,30 @@ class ConformerBlockLinears:
 
         run(L[0], h_in, self.u); note(L[0].spec.name, self.u)
         run(L[1], self.u, self.h_a, residual=h_in, residual_scale=0.5); note(L[1].spec.name, self.h_a)
-        # q, k, v read the same h: quantize it once (the codes do not depend on the consumer)
+        # q, k, v read the same h: quantize it once (the codes do not depend on the consumer) and
+        # run the three projections as one matmul over their concatenated output channels
         hq, hs = run.quantize_input(self.h_a, L[2].spec.bits_a)
-        run.matmul(L[2], hq, hs, self.q); note(L[2].spec.name, self.q)
-        run.matmul(L[3], hq, hs, self.k); note(L[3].spec.name, self.k)
-        run.matmul(L[4], hq, hs, self.v); note(L[4].spec.name, self.v)
+        wq, s_w, bias = self._fused_qkv(L)
+        aqt.aqt_qmatmul(hq, hs, wq, s_w, bias, None, 1.0, K=self.d, bits_a=8, bits_w=L[2].spec.bits_w, act=aqt.ACT_NONE,
+                        s_x_kind=run.a_scale_kind, y=self.qkv, workspace=run.workspace)
+        note(L[2].spec.name, self.q); note(L[3].spec.name, self.k); note(L[4].spec.name, self.v)
         run(L[5], self.v, self.h_b, residual=self.h_a, residual_scale=1.0); note(L[5].spec.name, self.h_b)
         run(L[6], self.h_b, self.c); note(L[6].spec.name, self.c)
         run(L[7], self.c, self.h_a, residual=self.h_b, residual_scale=1.0); note(L[7].spec.name, self.h_a)
         run(L[8], self.h_a, self.u); note(L[8].spec.name, self.u)
         run(L[9], self.u, h_out, residual=self.h_a, residual_scale=0.5); note(L[9].spec.name, h_out)
         return h_out
+
+    def _fused_qkv(self, L: List[QuantLinear]):
+        """Codes, scales and bias of the q, k, v projections stacked along the output channels
+        (built once per block and kept)."""
+        key = id(L[2])
+        if key not in self._qkv_weights:
+            q, k, v = L[2], L[3], L[4]
+            assert q.spec.bits_w == k.spec.bits_w == v.spec.bits_w and q.spec.act == k.spec.act == v.spec.act == aqt.ACT_NONE
+            bias = None if q.bias is None else torch.cat([q.bias, k.bias, v.bias]).contiguous()
+            self._qkv_weights[key] = (torch.cat([q.wq, k.wq, v.wq]).contiguous(), torch.cat([q.s_w, k.s_w, v.s_w]).contiguous(), bias)
+        return self._qkv_weights[key]
 
     def ops(self, layers: List[QuantLinear]) -> int:
         return sum(2 * self.M * l.spec.N * l.spec.K for l in layers)
