@@ -111,7 +111,7 @@ int aqt_unpack_int4(const uint8_t* packed, int64_t rows, int64_t cols, int8_t* q
  * acc_debug NULL, or int32 [M, N] dense: receives the raw accumulators (for parity checks).
  * workspace at least aqt_workspace_bytes(AQT_OP_QMATMUL, ...) bytes, 256-byte aligned; holds the
  *           sign-extended copy of each 4-bit operand.  May be NULL when both operands are 8-bit.
- * Limits: K % 32 == 0; N % 4 == 0 (N % 8 == 0 for GLU); ldy % 4 == 0, ldr % 4 == 0; xq, wq, y,
+ * Limits: K % 16 == 0; N % 4 == 0 (N % 8 == 0 for GLU); ldy % 4 == 0, ldr % 4 == 0; xq, wq, y,
  * residual, s_w, bias 16-byte aligned; M, N, K < 2^31 and M*N < 2^40.  K <= 133 000 keeps every
  * accumulator inside int32.  M == 0 or N == 0 is a no-op.
  */

@@ -40,7 +40,7 @@ int validate_matmul_shape(int64_t M, int64_t N, int64_t K, int bits_a, int bits_
   if (M < 0 || N < 0 || K <= 0) return AQT_ERR_BADARG;
   if (!bits_ok(bits_a) || !bits_ok(bits_w) || !act_ok(act)) return AQT_ERR_BADARG;
   if (s_x_kind != AQT_SCALE_ROW && s_x_kind != AQT_SCALE_TENSOR) return AQT_ERR_BADARG;
-  if (K % 32 != 0 || N % 4 != 0 || (is_glu(act) && N % 8 != 0)) return AQT_ERR_BADARG;
+  if (K % 16 != 0 || N % 4 != 0 || (is_glu(act) && N % 8 != 0)) return AQT_ERR_BADARG;
   if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 31) || M * N >= (1ll << 40)) return AQT_ERR_UNSUPPORTED;
   return AQT_OK;
 }
@@ -84,7 +84,7 @@ int qmatmul_i8a(const int8_t* a_codes, const float* s_x, int s_x_kind, const voi
   const void* b_codes = wq;
   bool b_packed = false;
   if (bits_w == 4) {
-    if (qgemm_uses_ws(N, K)) {
+    if (qgemm_uses_ws(N, K) && K % 32 == 0) {  // the packed rows must keep the 16-byte pitch bulk copies need
       b_packed = true;
     } else {
       int rc = launch_unpack_int4(reinterpret_cast<const uint8_t*>(wq), N * K / 2, reinterpret_cast<int8_t*>(ws), st);

@@ -64,7 +64,7 @@ def test_argument_errors_are_reported_before_any_cuda_call():
         ldy = N if ldy is None else ldy
         return L.aqt_qmatmul(xq, one, kind, one, one, None, None, i64(0), f, i64(M), i64(N), i64(K), ba, bw, act, one,
                              i64(ldy), None, ws, ctypes.c_size_t(wsb), None)
-    assert mm(128, 256, 100, 8, 8, 0) == -1          # K not a multiple of 32
+    assert mm(128, 256, 100, 8, 8, 0) == -1          # K not a multiple of 16
     assert mm(128, 250, 128, 8, 8, 0) == -1          # N not a multiple of 4
     assert mm(128, 260, 128, 8, 8, 2) == -1          # GLU needs N % 8 == 0
     assert mm(128, 256, 128, 3, 8, 0) == -1

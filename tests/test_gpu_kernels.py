@@ -167,6 +167,28 @@ def test_qmatmul_activations(act, M, N, K):
     _run_qmatmul(M, N, K, 8, 4, act, True, True)
 
 
+@pytest.mark.parametrize("M", [4, 200, 1300])
+@pytest.mark.parametrize("N,K,act,bits_a,bits_w", [(576, 144, aqt.ACT_SWISH, 8, 4), (144, 576, aqt.ACT_NONE, 8, 4), (144, 144, aqt.ACT_NONE, 4, 4),
+                                                    (288, 144, aqt.ACT_GLU_SWISH, 8, 8), (144, 1168, aqt.ACT_NONE, 8, 4)])
+def test_qmatmul_conformer_s_widths(M, N, K, act, bits_a, bits_w):
+    """Model width 144 (the paper's Conformer S, Section 3.2): K is a multiple of 16 but not of 32 or
+    128, so the last k-block is partly outside the tensor and packed rows are 72 bytes."""
+    _run_qmatmul(M, N, K, bits_a, bits_w, act, True, True, extremes=True)
+
+
+def test_linear_fwd_conformer_s_width():
+    M, K, N = 333, 144, 576
+    x = gen.normal(8, 1, M, K)
+    wt = gen.weight(8, 2, K, N)
+    wq, s_w = orc.quantize(wt, 4, orc.AXIS_ROW)
+    y_ref = orc.linear_fwd(x, wq, s_w)
+    wq_d, sw_d = aqt.aqt_quantize(_dev(wt), 4, aqt.AXIS_ROW, pack=True)
+    assert np.array_equal(wq_d.cpu().numpy(), orc.pack_int4(wq))
+    y = aqt.aqt_linear_fwd(_dev(x), wq_d, sw_d, bits_a=8, bits_w=4)
+    _status_ok()
+    assert np.array_equal(y.cpu().numpy().view(np.uint32), y_ref.view(np.uint32))
+
+
 def test_qmatmul_per_tensor_scale_and_deep_k():
     _run_qmatmul(256, 256, 4096, 8, 8, aqt.ACT_NONE, True, False, s_x_kind=aqt.SCALE_TENSOR, extremes=True)
 
