@@ -32,7 +32,7 @@
 extern "C" {
 #endif
 
-#define AQT_VERSION 101
+#define AQT_VERSION 102
 
 /* status codes */
 #define AQT_OK 0
@@ -65,6 +65,7 @@ extern "C" {
 /* operations for aqt_workspace_bytes */
 #define AQT_OP_QMATMUL 1
 #define AQT_OP_LINEAR_FWD 2
+#define AQT_OP_QMATMUL_REQUANT 3
 
 int aqt_version(void);
 const char* aqt_status_string(int status);
@@ -119,6 +120,33 @@ int aqt_qmatmul(const void* xq, const float* s_x, int s_x_kind, const void* wq, 
                 const float* bias, const float* residual, int64_t ldr, float residual_scale, int64_t M,
                 int64_t N, int64_t K, int bits_a, int bits_w, int act, float* y, int64_t ldy,
                 int32_t* acc_debug, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * aqt_qmatmul_requant -- aqt_qmatmul whose output rows are quantized for the next layer inside
+ * the same kernel (Section 2.2: every quantized layer quantizes its input dynamically, so the
+ * tensor between two such layers is only ever consumed as codes and row scales; Fig. 2 is
+ * applied to the output rows before they leave the SM, and the fp32 tensor is not written
+ * unless the caller asks for it):
+ *   u            = what aqt_qmatmul would write to y (same arguments, same arithmetic)
+ *   q_out, s_out = aqt_quantize(u, axis = AQT_AXIS_ROW, bits_out, rounding, pack_out)
+ * q_out     bits_out == 8 or pack_out == 0: int8 [M, N_out] dense;  pack_out == 1 (bits_out == 4
+ *           only): uint8 [M, N_out/2] packed.
+ * s_out     fp32 [M].
+ * y         NULL, or fp32 [M, N_out] with row pitch ldy: also receives u (a residual stream, or
+ *           a parity check).  residual != NULL requires y != NULL.
+ * workspace at least aqt_workspace_bytes(AQT_OP_QMATMUL_REQUANT, ...) bytes, 256-byte aligned:
+ *           what aqt_qmatmul needs plus the area through which CTAs exchange row maxima.
+ * Limits: those of aqt_qmatmul, and N_out % 16 == 0 (N_out % 32 == 0 if pack_out).  The fused
+ * kernel takes K <= 512 with act NONE or SWISH; it is launched cooperatively (its CTAs wait on
+ * one another, with the same bounded waits as everything else) on at most one CTA per SM.
+ * Other shapes run the two steps one after the other through y and return
+ * AQT_ERR_UNSUPPORTED if y is NULL.
+ */
+int aqt_qmatmul_requant(const void* xq, const float* s_x, int s_x_kind, const void* wq, const float* s_w,
+                        const float* bias, const float* residual, int64_t ldr, float residual_scale, int64_t M,
+                        int64_t N, int64_t K, int bits_a, int bits_w, int act, int bits_out, int rounding,
+                        int pack_out, void* q_out, float* s_out, float* y, int64_t ldy, void* workspace,
+                        size_t workspace_bytes, void* stream);
 
 /*
  * aqt_linear_fwd -- the whole layer for fp32 activations: aqt_quantize(x, axis = K) with a

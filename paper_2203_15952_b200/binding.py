@@ -20,11 +20,11 @@ AXIS_ROW, AXIS_COL, AXIS_TENSOR = 0, 1, 2
 ROUND_HALF_UP_FLOOR, ROUND_NEAREST_EVEN = 0, 1
 SCALE_ROW, SCALE_TENSOR = 0, 1
 ACT_NONE, ACT_SWISH, ACT_GLU, ACT_GLU_SWISH = 0, 1, 2, 3
-OP_QMATMUL, OP_LINEAR_FWD = 1, 2
+OP_QMATMUL, OP_LINEAR_FWD, OP_QMATMUL_REQUANT = 1, 2, 3
 
 EXPORTS = ("aqt_version", "aqt_status_string", "aqt_quantize", "aqt_pack_int4", "aqt_unpack_int4", "aqt_qmatmul",
            "aqt_linear_fwd", "aqt_linear_fwd_host", "aqt_workspace_bytes", "aqt_device_status", "aqt_qmatmul_w4_noalloc",
-           "aqt_selftest_bounded_wait")
+           "aqt_selftest_bounded_wait", "aqt_qmatmul_requant")
 NOALLOC_MAX_WEIGHT_BYTES = 4 << 20
 
 
@@ -104,6 +104,16 @@ def bind_qmatmul(xq, s_x, wq, s_w, bias, residual, residual_scale, K, bits_a, bi
                 _i64(residual.stride(0) if residual is not None else 0), ctypes.c_float(residual_scale), _i64(M), _i64(N),
                 _i64(K), int(bits_a), int(bits_w), int(act), _ptr(y), _i64(y.stride(0)), _ptr(None), _ptr(workspace),
                 ctypes.c_size_t(0 if workspace is None else workspace.numel()), _stream(stream))
+
+
+def bind_qmatmul_requant(xq, s_x, wq, s_w, bias, residual, residual_scale, K, bits_a, bits_w, act, s_x_kind, bits_out, rounding,
+                         pack_out, q_out, s_out, y, workspace, stream=None):
+    M, N = xq.shape[0], wq.shape[0]
+    return bind("aqt_qmatmul_requant", _ptr(xq), _ptr(s_x), int(s_x_kind), _ptr(wq), _ptr(s_w), _ptr(bias), _ptr(residual),
+                _i64(residual.stride(0) if residual is not None else 0), ctypes.c_float(residual_scale), _i64(M), _i64(N),
+                _i64(K), int(bits_a), int(bits_w), int(act), int(bits_out), int(rounding), int(bool(pack_out)), _ptr(q_out),
+                _ptr(s_out), _ptr(y), _i64(y.stride(0) if y is not None else 0), _ptr(workspace),
+                ctypes.c_size_t(workspace.numel()), _stream(stream))
 
 
 def bind_linear_fwd(x, wq, s_w, bias, residual, residual_scale, bits_a, bits_w, a_scale_kind, rounding, act, y, workspace,
@@ -202,6 +212,34 @@ def aqt_qmatmul(xq: torch.Tensor, s_x: torch.Tensor, wq: torch.Tensor, s_w: torc
         int(bits_a), int(bits_w), int(act), _ptr(y), _i64(y.stride(0)), _ptr(acc_debug), _ptr(workspace),
         ctypes.c_size_t(0 if workspace is None else workspace.numel()), _stream(stream)))
     return y
+
+
+def aqt_qmatmul_requant(xq: torch.Tensor, s_x: torch.Tensor, wq: torch.Tensor, s_w: torch.Tensor,
+                        bias: Optional[torch.Tensor] = None, residual: Optional[torch.Tensor] = None,
+                        residual_scale: float = 1.0, *, K: int, bits_a: int = 8, bits_w: int = 8, act: int = ACT_NONE,
+                        s_x_kind: int = SCALE_ROW, bits_out: int = 8, rounding: int = ROUND_NEAREST_EVEN, pack_out: bool = False,
+                        want_y: bool = False, q_out: Optional[torch.Tensor] = None, s_out: Optional[torch.Tensor] = None,
+                        y: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, stream=None):
+    """aqt_qmatmul whose output rows leave the kernel already quantized for the next layer.
+    Returns (q_out, s_out, y); y is None unless want_y (or a residual / y tensor is given)."""
+    M, N = xq.shape[0], wq.shape[0]
+    n_out = _n_out(N, act)
+    if q_out is None:
+        q_out = torch.empty((M, n_out // 2 if pack_out else n_out), dtype=torch.uint8 if pack_out else torch.int8,
+                            device=xq.device)
+    if s_out is None:
+        s_out = torch.empty((M,), dtype=torch.float32, device=xq.device)
+    if y is None and (want_y or residual is not None):
+        y = torch.empty((M, n_out), dtype=torch.float32, device=xq.device)
+    need = aqt_workspace_bytes(OP_QMATMUL_REQUANT, M, N, K, bits_a, bits_w)
+    workspace = _workspace(need, workspace, xq.device)
+    _check("aqt_qmatmul_requant", lib().aqt_qmatmul_requant(
+        _ptr(xq), _ptr(s_x), int(s_x_kind), _ptr(wq), _ptr(s_w), _ptr(bias), _ptr(residual),
+        _i64(residual.stride(0) if residual is not None else 0), ctypes.c_float(residual_scale), _i64(M), _i64(N), _i64(K),
+        int(bits_a), int(bits_w), int(act), int(bits_out), int(rounding), int(bool(pack_out)), _ptr(q_out), _ptr(s_out),
+        _ptr(y), _i64(y.stride(0) if y is not None else 0), _ptr(workspace),
+        ctypes.c_size_t(0 if workspace is None else workspace.numel()), _stream(stream)))
+    return q_out, s_out, y
 
 
 def aqt_qmatmul_w4_noalloc(xq: torch.Tensor, s_x: torch.Tensor, wq_packed: torch.Tensor, s_w: torch.Tensor,

@@ -3,6 +3,7 @@
 #include "aqt_common.cuh"
 #include "pack.cuh"
 #include "qgemm_sm100.cuh"
+#include "qgemm_requant_sm100.cuh"
 #include "qgemv_small_m.cuh"
 #include "quantize.cuh"
 
@@ -135,6 +136,7 @@ size_t aqt_workspace_bytes(int op, int64_t M, int64_t N, int64_t K, int bits_a, 
   if (M < 0 || N < 0 || K < 0) return 0;
   if (op == AQT_OP_QMATMUL) return ws_qmatmul(M, N, K, bits_a, bits_w);
   if (op == AQT_OP_LINEAR_FWD) return ws_linear(M, N, K, bits_w);
+  if (op == AQT_OP_QMATMUL_REQUANT) return round_up(ws_qmatmul(M, N, K, bits_a, bits_w), 256) + requant_exchange_bytes(M, N);
   return 0;
 }
 
@@ -213,6 +215,86 @@ int aqt_qmatmul(const void* xq, const float* s_x, int s_x_kind, const void* wq, 
   }
   return qmatmul_i8a(a_codes, s_x, s_x_kind, wq, s_w, bias, residual, ldr, residual_scale, M, N, K, bits_a, bits_w, act, y,
                      ldy, acc_debug, ws, st);
+}
+
+int aqt_qmatmul_requant(const void* xq, const float* s_x, int s_x_kind, const void* wq, const float* s_w, const float* bias,
+                        const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K, int bits_a,
+                        int bits_w, int act, int bits_out, int rounding, int pack_out, void* q_out, float* s_out, float* y,
+                        int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = validate_matmul_shape(M, N, K, bits_a, bits_w, act, s_x_kind);
+  if (rc != AQT_OK) return rc;
+  if (!bits_ok(bits_out) || (pack_out != 0 && pack_out != 1) || (pack_out == 1 && bits_out != 4)) return AQT_ERR_BADARG;
+  if (rounding != AQT_ROUND_HALF_UP_FLOOR && rounding != AQT_ROUND_NEAREST_EVEN) return AQT_ERR_BADARG;
+  const int64_t n_out = is_glu(act) ? N / 2 : N;
+  if (n_out % (pack_out ? 32 : 16) != 0) return AQT_ERR_BADARG;  // rows of codes keep a 16-byte pitch
+  if (residual != nullptr && y == nullptr) return AQT_ERR_BADARG;
+  if (M == 0 || N == 0) return AQT_OK;
+  if (xq == nullptr || s_x == nullptr || wq == nullptr || s_w == nullptr || q_out == nullptr || s_out == nullptr) return AQT_ERR_BADARG;
+  if (y != nullptr && (ldy < n_out || ldy % 4 != 0)) return AQT_ERR_BADARG;
+  if (residual != nullptr && (ldr < n_out || ldr % 4 != 0)) return AQT_ERR_BADARG;
+  if (!is_aligned(xq, 16) || !is_aligned(wq, 16) || !is_aligned(q_out, 16) || !is_aligned(s_w, 16) || !is_aligned(s_x, 4) ||
+      !is_aligned(s_out, 4) || (y != nullptr && !is_aligned(y, 16)) || (bias != nullptr && !is_aligned(bias, 16)) ||
+      (residual != nullptr && !is_aligned(residual, 16)))
+    return AQT_ERR_ALIGN;
+  const size_t mm_bytes = round_up(ws_qmatmul(M, N, K, bits_a, bits_w), 256);
+  const size_t need = mm_bytes + requant_exchange_bytes(M, N);
+  if (workspace == nullptr || workspace_bytes < need) return AQT_ERR_WORKSPACE;
+  if (!is_aligned(workspace, 256)) return AQT_ERR_ALIGN;
+  rc = check_device();
+  if (rc != AQT_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+
+  if (!requant_applies(M, N, K, act)) {
+    // Shapes the fused kernel does not take: the two steps one after the other, through y.
+    if (y == nullptr) return AQT_ERR_UNSUPPORTED;
+    rc = aqt_qmatmul(xq, s_x, s_x_kind, wq, s_w, bias, residual, ldr, residual_scale, M, N, K, bits_a, bits_w, act, y, ldy, nullptr,
+                     workspace, mm_bytes, stream);
+    if (rc != AQT_OK) return rc;
+    return aqt_quantize(y, M, n_out, ldy, bits_out, AQT_AXIS_ROW, rounding, pack_out, q_out, s_out, stream);
+  }
+
+  const int8_t* a_codes = reinterpret_cast<const int8_t*>(xq);
+  if (bits_a == 4) {
+    rc = launch_unpack_int4(reinterpret_cast<const uint8_t*>(xq), M * K / 2, reinterpret_cast<int8_t*>(ws), st);
+    if (rc != AQT_OK) return rc;
+    a_codes = reinterpret_cast<const int8_t*>(ws);
+    ws += round_up((size_t)M * (size_t)K, 256);
+  }
+  const void* b_codes = wq;
+  bool b_packed = false;
+  if (bits_w == 4) {
+    if (K % 32 == 0) {
+      b_packed = true;
+    } else {
+      rc = launch_unpack_int4(reinterpret_cast<const uint8_t*>(wq), N * K / 2, reinterpret_cast<int8_t*>(ws), st);
+      if (rc != AQT_OK) return rc;
+      b_codes = ws;
+    }
+  }
+  RequantParams rp;
+  GemmParams& p = rp.g;
+  p.s_x = s_x;
+  p.s_w = s_w;
+  p.bias = bias;
+  p.residual = residual;
+  p.acc_debug = nullptr;
+  p.ldr = ldr;
+  p.residual_scale = residual_scale;
+  p.s_x_kind = s_x_kind;
+  p.act = act;
+  p.M = (int)M;
+  p.N = (int)N;
+  p.K = (int)K;
+  p.n_out = (int)N;
+  p.tiles_m = p.tiles_n = p.k_blocks = 0;
+  p.small_acc = (K * (int64_t)(qmax_of(bits_a) + 1) * (qmax_of(bits_w) + 1) <= (1ll << 22)) ? 1 : 0;
+  rp.s_out = s_out;
+  rp.exchange = nullptr;
+  rp.qmax_out = qmax_of(bits_out);
+  rp.rounding = rounding;
+  rp.pack_out = pack_out;
+  return launch_requant(a_codes, b_codes, b_packed, q_out, y, ldy, rp, reinterpret_cast<uint8_t*>(workspace) + mm_bytes, st);
 }
 
 int aqt_linear_fwd(const float* x, int64_t ldx, const void* wq, const float* s_w, const float* bias, const float* residual,

@@ -851,9 +851,9 @@ static EncodeTiledFn get_encode_tiled() {
 }
 
 // 2-D row-major tensor [rows, cols] with `pitch_bytes` between rows; box [box_rows, box_cols];
-// 128-byte swizzle (box_cols * element size must then be 128 bytes) or none.
+// swizzle_bytes: 128 or 32 (box_cols * element size must then be that many bytes), or 0 for none.
 static int make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, const void* base, uint64_t rows, uint64_t cols,
-                       uint64_t pitch_bytes, uint32_t box_rows, uint32_t box_cols, bool swizzle128 = true) {
+                       uint64_t pitch_bytes, uint32_t box_rows, uint32_t box_cols, int swizzle_bytes = 128) {
   EncodeTiledFn enc = get_encode_tiled();
   if (enc == nullptr) {
     if (debug_enabled()) fprintf(stderr, "[aqt] driver entry point for tensor map encoding not found\n");
@@ -864,7 +864,8 @@ static int make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, const void* bas
   cuuint32_t box[2] = {box_cols, box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = enc(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                   swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (swizzle_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE),
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS && debug_enabled())
     fprintf(stderr, "[aqt] tensor map encode failed: CUresult %d (rows %llu cols %llu pitch %llu box %u x %u base %p)\n", (int)r,
@@ -921,7 +922,7 @@ static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t l
   int rc = make_map_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, a, (uint64_t)p.M, (uint64_t)p.K, (uint64_t)p.K, kBM, kBK);
   if (rc != AQT_OK) return rc;
   if (BPACK) {
-    rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, b, (uint64_t)p.N, (uint64_t)p.K / 2, (uint64_t)p.K / 2, BN / 2, 64, false);
+    rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, b, (uint64_t)p.N, (uint64_t)p.K / 2, (uint64_t)p.K / 2, BN / 2, 64, 0);
   } else {
     rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, b, (uint64_t)p.N, (uint64_t)p.K, (uint64_t)p.K, BN / 2, kBK);
   }

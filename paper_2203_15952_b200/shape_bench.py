@@ -2,6 +2,7 @@
 
     python -m paper_2203_15952_b200.shape_bench qmatmul M N K [--act 0..3] [--bits-w 4|8] [--residual]
                                                  [--iters I] [--sustain SECONDS]
+    python -m paper_2203_15952_b200.shape_bench requant M N K [--act 0|1] [--bits-w 4|8] [--bits 4|8] [--with-y] [--residual]
     python -m paper_2203_15952_b200.shape_bench quantize M K [--bits 4|8]
     python -m paper_2203_15952_b200.shape_bench linear M N K [--act ..] [--bits-w ..] [--bits 4|8] [--per-tensor]
 
@@ -88,12 +89,13 @@ def _sustain(calls, seconds):
 
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("op", choices=["qmatmul", "quantize", "linear"])
+    ap.add_argument("op", choices=["qmatmul", "requant", "quantize", "linear"])
     ap.add_argument("dims", type=int, nargs="+")
     ap.add_argument("--act", type=int, default=0)
     ap.add_argument("--bits-w", type=int, default=8)
     ap.add_argument("--bits", type=int, default=8)
     ap.add_argument("--residual", action="store_true")
+    ap.add_argument("--with-y", action="store_true", help="requant: also write the fp32 output")
     ap.add_argument("--per-tensor", action="store_true", help="linear: one activation scale for the whole tensor")
     ap.add_argument("--iters", type=int, default=30)
     ap.add_argument("--sets", type=int, default=4)
@@ -125,6 +127,33 @@ def main(argv=None):
         ops = 2.0 * M * N * K
         nbytes = M * K + N * K * a.bits_w // 8 + 8 * N + 4 * M + 4 * M * n_out * (2 if a.residual else 1)
         label = "qmatmul M%d N%d K%d act%d w%d res%d" % (M, N, K, a.act, a.bits_w, int(a.residual))
+    elif a.op == "requant":
+        # matmul whose epilogue quantizes the output rows (--bits: width of the output codes)
+        M, N, K = a.dims
+        wq = torch.randint(-7, 8, (N, K if a.bits_w == 8 else K // 2), generator=g, dtype=torch.int8, device=dev)
+        if a.bits_w == 4:
+            wq = wq.view(torch.uint8)
+        sw = torch.rand(N, generator=g, device=dev) * 1e-3
+        ws = torch.empty(aqt.aqt_workspace_bytes(aqt.OP_QMATMUL_REQUANT, M, N, K, 8, a.bits_w) + 256, dtype=torch.uint8, device=dev)
+        pack = a.bits == 4
+        sets = []
+        for _ in range(a.sets):
+            xq = torch.randint(-127, 128, (M, K), generator=g, dtype=torch.int8, device=dev)
+            sx = torch.rand(M, generator=g, device=dev) * 1e-2
+            q = torch.empty((M, N // 2 if pack else N), dtype=torch.uint8 if pack else torch.int8, device=dev)
+            so = torch.empty(M, device=dev)
+            y = torch.empty((M, N), dtype=torch.float32, device=dev) if (a.with_y or a.residual) else None
+            rr = torch.randn((M, N), generator=g, device=dev) if a.residual else None
+            sets.append((xq, sx, q, so, y, rr))
+
+        def make_calls(stream=None):
+            return [aqt.bind_qmatmul_requant(xq, sx, wq, sw, None, rr, 0.5, K, 8, a.bits_w, a.act, aqt.SCALE_ROW, a.bits,
+                                             aqt.ROUND_NEAREST_EVEN, pack, q, so, y, ws, stream)
+                    for (xq, sx, q, so, y, rr) in sets]
+        ops = 2.0 * M * N * K
+        nbytes = (M * K + N * K * a.bits_w // 8 + 8 * N + 8 * M + M * N * a.bits // 8
+                  + 4 * M * N * ((1 if (a.with_y or a.residual) else 0) + (1 if a.residual else 0)))
+        label = "requant M%d N%d K%d act%d w%d out%d y%d res%d" % (M, N, K, a.act, a.bits_w, a.bits, int(a.with_y or a.residual), int(a.residual))
     elif a.op == "linear":
         M, N, K = a.dims
         n_out = N // 2 if a.act >= 2 else N

@@ -1,0 +1,118 @@
+"""Parity of the matmul that quantizes its own output rows (Fig. 2 applied in the epilogue) against
+the CPU oracle, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+from paper_2203_15952_b200 import binding as aqt
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+
+
+def _codes(rng, rows, K, bits):
+    qm = 127 if bits == 8 else 7
+    return rng.integers(-qm, qm + 1, (rows, K)).astype(np.int8)
+
+
+def _run(M, N, K, bits_a, bits_w, act, with_bias, with_res, bits_out, rounding, pack_out, special_rows=False):
+    rng = np.random.default_rng(7 + 1000 * M + N + K + bits_out)
+    xq = _codes(rng, M, K, bits_a)
+    wq = _codes(rng, N, K, bits_w)
+    s_x = rng.uniform(1e-3, 5e-2, M).astype(np.float32)
+    if special_rows:
+        xq[0, :] = 0                       # with no bias: an all-zero output row (scale 0, codes 0)
+        if M > 2:
+            s_x[1] = 1e-37                 # a row whose maximum is far below the fast-division range
+            s_x[2] = 3e33                  # and one far above it
+    s_w = rng.uniform(1e-4, 5e-3, N).astype(np.float32)
+    bias = (rng.standard_normal(N) * 0.1).astype(np.float32) if with_bias else None
+    res = rng.standard_normal((M, N)).astype(np.float32) if with_res else None
+    acc_ref = orc.int_matmul(xq, wq)
+    y_ref = orc.epilogue_f32(acc_ref, s_x, aqt.SCALE_ROW, s_w, bias, res, 0.5, act)
+    y64 = orc.epilogue_f64(acc_ref, s_x, aqt.SCALE_ROW, s_w, bias, res, 0.5, act)
+
+    xq_d = _dev(orc.pack_int4(xq)) if bits_a == 4 else _dev(xq)
+    wq_d = _dev(orc.pack_int4(wq)) if bits_w == 4 else _dev(wq)
+    args = (xq_d, _dev(s_x), wq_d, _dev(s_w), None if bias is None else _dev(bias), None if res is None else _dev(res), 0.5)
+    kw = dict(K=K, bits_a=bits_a, bits_w=bits_w, act=act, bits_out=bits_out, rounding=rounding, pack_out=pack_out)
+    q_shape = (M, N // 2) if pack_out else (M, N)
+    q_d = torch.full(q_shape, 0x55, dtype=torch.uint8 if pack_out else torch.int8, device=DEV)
+    s_d = torch.full((M,), float("nan"), dtype=torch.float32, device=DEV)
+    y_d = torch.full((M, N), float("nan"), dtype=torch.float32, device=DEV)
+    aqt.aqt_qmatmul_requant(*args, **kw, q_out=q_d, s_out=s_d, y=y_d)
+    assert aqt.aqt_device_status() == 0
+    y = y_d.cpu().numpy()
+    q = q_d.cpu().numpy()
+    s = s_d.cpu().numpy()
+
+    # the fp32 output: the same bar as the plain matmul
+    if act == aqt.ACT_NONE:
+        assert np.array_equal(y.view(np.uint32), y_ref.view(np.uint32))
+    else:
+        assert np.isfinite(y).all()
+        z = orc.epilogue_f64(acc_ref, s_x, aqt.SCALE_ROW, s_w, None, None, 0.0, aqt.ACT_NONE)
+        mag = np.maximum(np.abs(y64), np.abs(z))
+        if bias is not None:
+            mag = np.maximum(mag, np.abs(bias)[None, :])
+        if res is not None:
+            mag = np.maximum(mag, np.abs(res))
+        assert np.all(np.abs(y - y64) <= 1e-6 * mag + 1e-30), float(np.max(np.abs(y - y64) / (mag + 1e-30)))
+
+    # codes and scales: the oracle's quantizer on the rows the kernel itself produced, bit for bit
+    q_ref, s_ref = orc.quantize(y, bits_out, orc.AXIS_ROW, rounding)
+    assert np.array_equal(s.view(np.uint32), s_ref.reshape(-1).view(np.uint32)), "scales differ in %d rows" % (s != s_ref.reshape(-1)).sum()
+    q_cmp = orc.pack_int4(q_ref) if pack_out else q_ref
+    assert np.array_equal(q, q_cmp), "codes differ: %d of %d" % ((q != q_cmp).sum(), q.size)
+    if act == aqt.ACT_NONE:
+        q_ref2, s_ref2 = orc.quantize(y_ref, bits_out, orc.AXIS_ROW, rounding)   # nothing of the kernel's in the reference
+        assert np.array_equal(q_ref2, q_ref) and np.array_equal(s_ref2, s_ref)
+
+    # without the fp32 output the codes are the same ones
+    if res is None:
+        q2_d = torch.full(q_shape, 0x55, dtype=q_d.dtype, device=DEV)
+        s2_d = torch.full((M,), float("nan"), dtype=torch.float32, device=DEV)
+        _, _, y_none = aqt.aqt_qmatmul_requant(*args, **kw, q_out=q2_d, s_out=s2_d)
+        assert y_none is None
+        assert aqt.aqt_device_status() == 0
+        assert torch.equal(q2_d, q_d) and torch.equal(s2_d.view(torch.int32), s_d.view(torch.int32))
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (128, 256, 128), (256, 512, 512), (300, 2048, 512), (1000, 512, 256),
+                                   (40, 144, 144), (5000, 1024, 384), (129, 2064, 96)])
+@pytest.mark.parametrize("act", [aqt.ACT_NONE, aqt.ACT_SWISH])
+def test_requant_w8a8(M, N, K, act):
+    _run(M, N, K, 8, 8, act, True, False, 8, aqt.ROUND_NEAREST_EVEN, False)
+
+
+@pytest.mark.parametrize("bits_a,bits_w,bits_out,pack_out", [(8, 4, 8, False), (4, 4, 4, True), (8, 4, 4, False), (4, 8, 8, False)])
+@pytest.mark.parametrize("rounding", [aqt.ROUND_NEAREST_EVEN, aqt.ROUND_HALF_UP_FLOOR])
+def test_requant_bit_widths_and_rounding(bits_a, bits_w, bits_out, pack_out, rounding):
+    _run(700, 1024, 512, bits_a, bits_w, aqt.ACT_SWISH, True, False, bits_out, rounding, pack_out)
+    _run(333, 512, 256, bits_a, bits_w, aqt.ACT_NONE, False, False, bits_out, rounding, pack_out, special_rows=True)
+
+
+@pytest.mark.parametrize("M,N,K", [(256, 512, 512), (1300, 512, 128), (77, 1024, 512)])
+@pytest.mark.parametrize("act", [aqt.ACT_NONE, aqt.ACT_SWISH])
+def test_requant_with_residual_stream(M, N, K, act):
+    _run(M, N, K, 8, 4, act, True, True, 8, aqt.ROUND_NEAREST_EVEN, False)
+
+
+def test_requant_many_tiles_per_cta():
+    """More m-tiles than groups of CTAs: every TMEM buffer and both exchange slots are reused."""
+    _run(12800, 2048, 512, 8, 4, aqt.ACT_SWISH, False, False, 8, aqt.ROUND_NEAREST_EVEN, False)
+
+
+def test_requant_unfused_shapes_go_through_y():
+    """K > 512 and GLU are not taken by the fused kernel: the call runs the two steps through y."""
+    _run(200, 512, 2048, 8, 4, aqt.ACT_NONE, True, True, 8, aqt.ROUND_NEAREST_EVEN, False)
+    rng = np.random.default_rng(3)
+    xq, wq = _codes(rng, 64, 1024, 8), _codes(rng, 256, 1024, 8)
+    with pytest.raises(aqt.AqtError) as e:
+        aqt.aqt_qmatmul_requant(_dev(xq), _dev(np.ones(64, np.float32)), _dev(wq), _dev(np.ones(256, np.float32)), K=1024)
+    assert e.value.status == -3
