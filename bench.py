@@ -30,7 +30,8 @@ sys.path.insert(0, ROOT)
 METRIC = "quantized Conformer linear TOPS (int4 weights, int8 activations)"
 UNIT = "TOPS"
 CFG = 2  # the Conformer FFN pair; fits one GPU many times over
-NCU_CAPTURE_VERSION = 101  # library version the ncu traffic figures below were captured at
+NCU_CAPTURE_VERSION = 0  # library version the ncu traffic figures below were captured at
+NCU_TRAFFIC = {}         # call index -> DRAM bytes per launch (profiles/)
 
 
 def _peaks():
@@ -199,19 +200,21 @@ def run_ours(args):
     for i, s in enumerate(specs):
         wt = torch.from_numpy(gen.layer_weight(w, 0, i, s, seed=0)).to(dev)
         layers.append(QuantLinear.from_float(s, wt))
-    R = 6  # rotating input/output sets: x + u + y of one step exceed the 126 MB L2 already
+    R = 6  # rotating input/output sets: the six x and six y tensors (315 MB) exceed the 126 MB L2
     x_host = gen.workload_input(w, seed=seed)
     xs = [torch.from_numpy(x_host).to(dev) for _ in range(R)]
     ys = [torch.empty((M, specs[1].N), dtype=torch.float32, device=dev) for _ in range(R)]
-    u = torch.empty((M, specs[0].N), dtype=torch.float32, device=dev)
     q1 = torch.empty((M, specs[0].K), dtype=torch.int8, device=dev)
     q2 = torch.empty((M, specs[1].K), dtype=torch.int8, device=dev)
     s1 = torch.empty(M, dtype=torch.float32, device=dev)
     s2 = torch.empty(M, dtype=torch.float32, device=dev)
-    ws = torch.empty(max(aqt.aqt_workspace_bytes(aqt.OP_QMATMUL, M, s.N, s.K, s.bits_a, s.bits_w) for s in specs) + 256,
-                     dtype=torch.uint8, device=dev)
+    ws = torch.empty(max(max(aqt.aqt_workspace_bytes(op, M, s.N, s.K, s.bits_a, s.bits_w) for s in specs)
+                         for op in (aqt.OP_QMATMUL, aqt.OP_QMATMUL_REQUANT)) + 256, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
-    names = ["quantize(x) 12800x512", "qmatmul 512->2048 swish", "quantize(u) 12800x2048", "qmatmul 2048->512"]
+    # One step = the whole FFN pair: the hidden tensor u = Swish(W1 x) is quantized per row inside
+    # the first matmul's epilogue and only ever exists as codes + row scales.
+    names = ["quantize(x) 12800x512", "qmatmul 512->2048 swish + quantize(u) rows (one kernel)", "qmatmul 2048->512"]
+    NC = len(names)
 
     # pre-marshalled C-ABI calls (one set per rotating buffer) so that Python stays ahead of the GPU
     def make_calls(st):
@@ -219,9 +222,9 @@ def run_ours(args):
         for r in range(R):
             out.append((
                 aqt.bind_quantize(xs[r], specs[0].bits_a, aqt.AXIS_ROW, aqt.ROUND_NEAREST_EVEN, False, q1, s1, st),
-                aqt.bind_qmatmul(q1, s1, layers[0].wq, layers[0].s_w, None, None, 1.0, specs[0].K, 8, specs[0].bits_w,
-                                 specs[0].act, aqt.SCALE_ROW, u, ws, st),
-                aqt.bind_quantize(u, specs[1].bits_a, aqt.AXIS_ROW, aqt.ROUND_NEAREST_EVEN, False, q2, s2, st),
+                aqt.bind_qmatmul_requant(q1, s1, layers[0].wq, layers[0].s_w, None, None, 1.0, specs[0].K, 8, specs[0].bits_w,
+                                         specs[0].act, aqt.SCALE_ROW, specs[1].bits_a, aqt.ROUND_NEAREST_EVEN, False, q2, s2, None,
+                                         ws, st),
                 aqt.bind_qmatmul(q2, s2, layers[1].wq, layers[1].s_w, None, None, 1.0, specs[1].K, 8, specs[1].bits_w,
                                  specs[1].act, aqt.SCALE_ROW, ys[r], ws, st)))
         return out
@@ -231,10 +234,11 @@ def run_ours(args):
     def step(i, events=None):
         c = calls[i % R]
         if events is None:
-            c[0](); c[1](); c[2](); c[3]()
+            for f in c:
+                f()
             return
         events[0].record(stream)
-        for j in range(4):
+        for j in range(NC):
             c[j]()
             events[j + 1].record(stream)
 
@@ -277,7 +281,7 @@ def run_ours(args):
         sampler.start()
         time.sleep(0.3)
     n_instr = len([i for i in range(args.steps) if i % (R + 1) == 0]) if graph is not None else args.steps
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(n_instr)]
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(NC + 1)] for _ in range(n_instr)]
     e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e_begin.record(stream)
@@ -299,7 +303,7 @@ def run_ours(args):
     status = aqt.aqt_device_status()
     evs = evs[:k]
 
-    per_call_ms = [statistics.mean(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(len(evs))) for j in range(4)]
+    per_call_ms = [statistics.mean(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(len(evs))) for j in range(NC)]
     t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -361,32 +365,43 @@ def run_ours(args):
     s0, s1_ = specs
     alg_bytes = [
         4 * M * s0.K + M * s0.K + 4 * M,                                              # quantize(x): read fp32, write codes + scales
-        M * s0.K + s0.K * s0.N // 2 + 8 * s0.N + 4 * M + 4 * M * s0.N,                # GEMM 1: codes, int4 weights, scales, fp32 out
-        4 * M * s1_.K + M * s1_.K + 4 * M,                                            # quantize(u)
-        M * s1_.K + s1_.K * s1_.N // 2 + 8 * s1_.N + 4 * M + 4 * M * s1_.N,           # GEMM 2
+        M * s0.K + s0.K * s0.N // 2 + 8 * s0.N + 4 * M + M * s0.N + 4 * M,            # GEMM 1: codes, int4 weights, scales in; codes + scales out
+        M * s1_.K + s1_.K * s1_.N // 2 + 8 * s1_.N + 4 * M + 4 * M * s1_.N,           # GEMM 2: codes, int4 weights, scales in; fp32 out
     ]
     kernels = [{"call": names[j], "ms": per_call_ms[j], "algorithmic_bytes": alg_bytes[j],
-                "gbs": alg_bytes[j] / (per_call_ms[j] * 1e-3) / 1e9, "share": per_call_ms[j] / sum(per_call_ms)} for j in range(4)]
-    # DRAM traffic per launch of the GEMM kernels from the committed ncu capture
-    # (profiles/qgemm_i8_ffn_pair_ncu.md: dram__bytes_read.sum + dram__bytes_write.sum).  The write
-    # part undercounts: most of the output is still in the 126 MB L2 when the kernel ends.
-    ncu_traffic = {1: 7174912 + 46349824, 3: 27342336 + 254720} if aqt.aqt_version() == NCU_CAPTURE_VERSION else {}
-    dom = max(range(4), key=lambda j: per_call_ms[j])
-    achieved = kernels[dom]["gbs"]
-    roofline = {"bound": "hbm", "kernel": names[dom], "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "peak_source": "of " + peak_kind, "traffic": ncu_traffic.get(dom), "calls": kernels}
+                "gbs": alg_bytes[j] / (per_call_ms[j] * 1e-3) / 1e9, "share": per_call_ms[j] / sum(per_call_ms)} for j in range(NC)]
+    # DRAM traffic per launch from the committed ncu captures (dram__bytes_read.sum +
+    # dram__bytes_write.sum); the write part undercounts what is still in L2 when the kernel ends.
+    ncu_traffic = NCU_TRAFFIC if aqt.aqt_version() == NCU_CAPTURE_VERSION else {}
+    dom = max(range(NC), key=lambda j: per_call_ms[j])
+    if dom == 1:
+        # The fused kernel moves 33 MB (5 us of HBM time) and is bound by arithmetic instead: the
+        # Swish needs two special-function operations (2^x, reciprocal) per element, and an SM
+        # retires 16 of those per clock.  peak = 16 x SMs x the maximum SM clock.
+        props = torch.cuda.get_device_properties(dev)
+        sm_max_mhz = (clocks or {}).get("sm_max_mhz") or 1965
+        sfu_peak = 16 * props.multi_processor_count * sm_max_mhz * 1e6 / 1e9      # Gop/s
+        sfu_achieved = 2.0 * M * s0.N / (per_call_ms[1] * 1e-3) / 1e9
+        roofline = {"bound": "alu", "kernel": names[1], "achieved": sfu_achieved, "peak": sfu_peak, "unit": "Gop/s",
+                    "frac": sfu_achieved / sfu_peak, "peak_source": "special-function unit: 16 op/clk/SM x %d SMs x %d MHz" %
+                    (props.multi_processor_count, sm_max_mhz), "hbm_frac": kernels[1]["gbs"] / peak,
+                    "traffic": ncu_traffic.get(1), "calls": kernels}
+    else:
+        achieved = kernels[dom]["gbs"]
+        roofline = {"bound": "hbm", "kernel": names[dom], "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "peak_source": "of " + peak_kind, "traffic": ncu_traffic.get(dom), "calls": kernels}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int8", "data": "synthetic",
             "config": {"workload": w.name, "M": M, "d_model": w.d, "ff": w.ff, "bits_w": 4, "bits_a": 8, "a_scale": "per-row",
-                       "rounding": "nearest-even", "l2": "rotating %d input/output sets; x + u + y of one step (157 MB) exceed the 126 MB L2" % R,
+                       "rounding": "nearest-even", "l2": "rotating %d input/output sets (x and y: 315 MB) exceed the 126 MB L2" % R,
                        "parallelism": "replicas x%d (rows sharded, no collective)" % world},
             "frames_per_s": world * args.steps * M / (total_ms * 1e-3),
             "clocks": clocks, "device_status": status,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 4 * M * s0.K, "d2h_bytes_per_step": 4 * M * s1_.N,
                     "ms_per_step": float(te.item()) / args.steps, "streams": n_lanes},
-            "gpu_launches": args.steps * 5, "sum_call_ms_per_step": sum(per_call_ms),
+            "gpu_launches": args.steps * 4, "sum_call_ms_per_step": sum(per_call_ms),
             "launch_mode": ("cuda graph of %d steps x %d replays + %d call-by-call steps with per-call events" % (R, replays, len(evs)))
             if graph is not None else "call by call",
             "roofline": roofline}

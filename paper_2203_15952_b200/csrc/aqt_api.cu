@@ -289,6 +289,7 @@ int aqt_qmatmul_requant(const void* xq, const float* s_x, int s_x_kind, const vo
   p.n_out = (int)N;
   p.tiles_m = p.tiles_n = p.k_blocks = 0;
   p.small_acc = (K * (int64_t)(qmax_of(bits_a) + 1) * (qmax_of(bits_w) + 1) <= (1ll << 22)) ? 1 : 0;
+  rp.q_out = nullptr;
   rp.s_out = s_out;
   rp.exchange = nullptr;
   rp.qmax_out = qmax_of(bits_out);

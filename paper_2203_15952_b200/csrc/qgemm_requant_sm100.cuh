@@ -15,13 +15,15 @@
 //                     columns it came from; the last of the four warps that share a row quadrant
 //                     merges their maxima and stores them, tagged valid in the sign bit (a
 //                     maximum is never negative), into the CTA's words of the exchange area
-//   pass 2 (tile j-1) reads the row's words of all n-tiles (requested before pass 1 of tile j, so
-//                     the round trip overlaps it), waits for any that is not yet valid, forms the
-//                     scale from the final maximum, u from TMEM, codes, TMA store; the TMEM
-//                     buffer goes back to the MMA
-// Every word carries its own validity, so no counter, fence or atomic on global memory is needed.
-// Pass 2 of a tile runs after pass 1 of the next one, so the exchange has a tile's worth of time
-// to complete; four TMEM buffers of 128 columns keep the tensor core two tiles ahead.
+//   exchange warp     for each tile in turn: reads the words of all n-tiles (128 rows per 512-byte
+//                     request, all requests in flight together), again until every one is valid,
+//                     and leaves the final maximum of each row in shared memory
+//   pass 2 (tile j-2) scale from the final maximum, u from TMEM, codes, stores; the TMEM buffer
+//                     goes back to the MMA
+// Every word carries its own validity, so no counter, fence or atomic on global memory is needed,
+// and the epilogue warps never wait on global memory.
+// Pass 2 of a tile runs after pass 1 of the tile two further on, so the exchange has two tiles'
+// worth of time to complete; four TMEM buffers of 128 columns keep the tensor core one tile ahead.
 // All CTAs must be resident at once (they wait on one another): the launch is cooperative and
 // the grid never exceeds one CTA per SM.  Every wait is bounded as in the plain GEMM.
 #pragma once
@@ -32,6 +34,7 @@ namespace aqt {
 
 struct RequantParams {
   GemmParams g;         // act: NONE or SWISH
+  uint8_t* q_out;       // codes of the output: int8 [M, N] or packed nibbles [M, N/2], dense
   float* s_out;         // [M] scales of the output rows
   uint32_t* exchange;   // [tiles_m][tiles_n][128]: bit pattern of a CTA's row maximum | 0x80000000; zero on entry
   int qmax_out;         // 127 or 7
@@ -43,20 +46,18 @@ template <bool WITH_Y>
 struct RequantCfg {
   static constexpr int BN = 128;
   static constexpr int EW = 16;
-  static constexpr int kThreads = 32 * (2 + EW);
-  static constexpr int kStages = WITH_Y ? 4 : 6;
+  static constexpr int kThreads = 32 * (2 + EW + 1);  // producer, MMA issuer, epilogue warps, exchange warp
+  static constexpr int kStages = WITH_Y ? 5 : 7;
   static constexpr int kABytes = kBM * kBK;
   static constexpr int kBBytes = BN * kBK;
   static constexpr int kResidentBytes = kWsMaxKBlocks * kBBytes;
-  static constexpr int kCodeBufBytes = 32 * 32;                  // per warp: 32 rows x 32 codes
-  static constexpr int kCodeBytes = EW * kCodeBufBytes;
   static constexpr int kYBytes = WITH_Y ? EW * kStageBufBytes : 0;
   static constexpr int kPackedBBytes = kWsMaxKBlocks * BN * 64;  // packed weights wait here for the unpack
-  static constexpr int kEpiBytes = (kCodeBytes + kYBytes) > kPackedBBytes ? (kCodeBytes + kYBytes) : kPackedBBytes;
+  static constexpr int kEpiBytes = kYBytes > kPackedBBytes ? kYBytes : kPackedBBytes;
   static constexpr int kScaleBytes = 2 * BN * 4;
   static constexpr int kTmemCols = 4 * BN;
   static constexpr int kSmemBytes = kStages * kABytes + kResidentBytes + kEpiBytes + kScaleBytes + 1024;
-  static_assert(kSmemBytes + 1024 <= 232448, "must fit the 227 KB a CTA can opt into");
+  static_assert(kSmemBytes + 13312 <= 232448, "must fit the 227 KB a CTA can opt into");
 };
 
 __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r)[32]) {
@@ -72,9 +73,9 @@ __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-__device__ __forceinline__ uint32_t ld_relaxed_gpu(const uint32_t* p) {
-  uint32_t v;
-  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+__device__ __forceinline__ uint4 ld_relaxed_gpu_v4(const uint32_t* p) {
+  uint4 v;
+  asm volatile("ld.relaxed.gpu.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
   return v;
 }
 __device__ __forceinline__ void st_relaxed_gpu(uint32_t* p, uint32_t v) {
@@ -82,37 +83,39 @@ __device__ __forceinline__ void st_relaxed_gpu(uint32_t* p, uint32_t v) {
 }
 
 constexpr uint32_t kValidBit = 0x80000000u;
-constexpr int kPrefetchWords = 16;  // exchange words per row requested ahead of pass 1 (covers N <= 2048)
+// Pass 2 of a tile runs kLag tiles behind its pass 1, which is the time the exchange has to
+// complete; with four TMEM buffers that leaves the MMA one tile of lookahead.  kSlots tiles'
+// worth of shared-memory exchange state (maxima parts, arrival counts, scale constants).
+constexpr int kLag = 2;
+constexpr int kSlots = 4;
+constexpr int kExchangeBatch = 16;  // exchange loads the exchange warp keeps in flight (one round trip for N <= 2048)
 
-// Bounded wait for an exchange word to become valid; `w` is what an earlier load returned.
-__device__ __forceinline__ bool wait_valid(const uint32_t* p, uint32_t& w, volatile int* abort_flag, uint64_t t_start) {
-  for (uint32_t spin = 1; (w & kValidBit) == 0u; ++spin) {
-    w = ld_relaxed_gpu(p);
-    if ((spin & 0x3F) == 0) {
-      if (*abort_flag) return false;
-      if (global_timer_ns() - t_start > kWaitLimitNs) {
-        *abort_flag = 1;
-        atomicExch(&g_device_status, AQT_ERR_TIMEOUT);
-        return false;
-      }
-    }
+// Called between polls of a bounded wait: false once the CTA is aborting or the limit has passed
+// (which then sets both the CTA's abort flag and the device status word).
+__device__ __forceinline__ bool keep_waiting(volatile int* abort_flag, uint64_t t_start) {
+  if (*abort_flag) return false;
+  if (global_timer_ns() - t_start > kWaitLimitNs) {
+    *abort_flag = 1;
+    atomicExch(&g_device_status, AQT_ERR_TIMEOUT);
+    return false;
   }
   return true;
 }
 
-// Codes of four values whose row scale constants are known (fast path of the quantizer: the
+// Codes of two values whose row scale constants are known (fast path of the quantizer: the
 // correctly rounded quotient by one multiply and two fused multiply-adds).  Rounding by adding
 // 1.5 * 2^23: the sum's low mantissa bits are the integer in two's complement, so the code's
 // byte is the low byte of the sum's bit pattern.  Nearest-even is the add's own rounding; the
 // figure's floor(v + 0.5) is the binary32 add of 0.5 followed by an add rounded towards minus
 // infinity.  Exact for |v| < 2^22; here |v| <= 127 (1 + 2^-23).
 template <int ROUNDING>
-__device__ __forceinline__ uint32_t code_bits(float x, float s, float r) {
-  const float q0 = __fmul_rn(x, r);
-  const float e = __fmaf_rn(-q0, s, x);
-  const float v = __fmaf_rn(e, r, q0);
-  if (ROUNDING == AQT_ROUND_HALF_UP_FLOOR) return __float_as_uint(__fadd_rd(__fadd_rn(v, 0.5f), 12582912.0f));
-  return __float_as_uint(__fadd_rn(v, 12582912.0f));
+__device__ __forceinline__ float2 code_bits2(float2 x, float2 s_neg, float2 r) {
+  const float2 q0 = __fmul2_rn(x, r);
+  const float2 e = __ffma2_rn(q0, s_neg, x);  // x - q0 s, exact
+  const float2 v = __ffma2_rn(e, r, q0);
+  const float2 magic = make_float2(12582912.0f, 12582912.0f);
+  if (ROUNDING == AQT_ROUND_HALF_UP_FLOOR) return __fadd2_rd(__fadd2_rn(v, make_float2(0.5f, 0.5f)), magic);
+  return __fadd2_rn(v, magic);
 }
 __device__ __forceinline__ uint32_t low_bytes(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   const uint32_t lo = __byte_perm(a, b, 0x0040);
@@ -130,10 +133,13 @@ __device__ __forceinline__ uint32_t nibbles_of(uint32_t w0, uint32_t w1) {
 template <int ROUNDING, bool PACK>
 __device__ __forceinline__ void codes32(const uint32_t (&u)[32], const ScaleCtx& c, int qmax, uint32_t (&w)[8]) {
   if (c.fast) {
+    const float2 s_neg = make_float2(-c.s, -c.s), r2 = make_float2(c.r, c.r);
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
-      w[j] = low_bytes(code_bits<ROUNDING>(__uint_as_float(u[4 * j]), c.s, c.r), code_bits<ROUNDING>(__uint_as_float(u[4 * j + 1]), c.s, c.r),
-                       code_bits<ROUNDING>(__uint_as_float(u[4 * j + 2]), c.s, c.r), code_bits<ROUNDING>(__uint_as_float(u[4 * j + 3]), c.s, c.r));
+    for (int j = 0; j < 8; ++j) {
+      const float2 c01 = code_bits2<ROUNDING>(make_float2(__uint_as_float(u[4 * j]), __uint_as_float(u[4 * j + 1])), s_neg, r2);
+      const float2 c23 = code_bits2<ROUNDING>(make_float2(__uint_as_float(u[4 * j + 2]), __uint_as_float(u[4 * j + 3])), s_neg, r2);
+      w[j] = low_bytes(__float_as_uint(c01.x), __float_as_uint(c01.y), __float_as_uint(c23.x), __float_as_uint(c23.y));
+    }
   } else {
 #pragma unroll
     for (int j = 0; j < 8; ++j)
@@ -148,10 +154,10 @@ __device__ __forceinline__ void codes32(const uint32_t (&u)[32], const ScaleCtx&
   }
 }
 
-template <bool BPACK, bool SMALL, bool WITH_Y>
-__global__ void __launch_bounds__(32 * 18, 1)
+template <bool BPACK, bool SMALL, bool WITH_Y, int ROUNDING, bool PACK_OUT>
+__global__ void __launch_bounds__(32 * 19, 1)
 qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                     const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_y,
+                     const __grid_constant__ CUtensorMap tm_y,
                      const __grid_constant__ CUtensorMap tm_r, const RequantParams rp) {
   using Cfg = RequantCfg<WITH_Y>;
   constexpr int BN = Cfg::BN, EW = Cfg::EW, STAGES = Cfg::kStages, HALF = BN / 2;
@@ -165,18 +171,21 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
   __shared__ uint64_t res_bar[EW];    // WITH_Y: residual tile landed in a warp's fp32 staging buffer
   __shared__ uint64_t b_loaded_bar;
   __shared__ uint64_t b_ready_bar;
-  __shared__ uint32_t amax_part[2][4][kBM];  // row maxima per column part of the tile in pass 1 (even / odd tiles)
-  // Warps of a row quadrant that have written their part (running counts, even / odd tiles).  A warp
-  // can be in pass 1 of tile j + 1 while another is still in pass 1 of tile j, but not of tile
-  // j + 2 (its pass 2 of tile j needs this quadrant's maxima of tile j published): two counters.
-  __shared__ uint32_t quad_arrivals[2][4];
+  __shared__ uint32_t amax_part[kSlots][4][kBM];  // row maxima per column part of the tile in pass 1 (slot = tile mod kSlots)
+  // Warps of a row quadrant that have written their part (running counts).  A warp can be in pass 1
+  // of tile j + kLag while another is still in pass 1 of tile j + 1, never further ahead (its pass 2
+  // of tile j needs this quadrant's maxima of tile j published): kSlots > kLag counters suffice.
+  __shared__ uint32_t quad_arrivals[kSlots][4];
+  __shared__ __align__(16) uint32_t row_amax[kSlots][kBM];  // final row maxima (bit patterns) of a tile awaiting pass 2
+  __shared__ uint64_t ctx_ready_bar[kSlots];  // the exchange warp has filled row_amax[.]
+  __shared__ uint64_t ctx_free_bar[kSlots];   // every epilogue warp has read its rows of row_amax[.]
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t smem_ring = smem_base;
   const uint32_t smem_res_b = smem_ring + STAGES * Cfg::kABytes;
-  const uint32_t smem_epi = smem_res_b + Cfg::kResidentBytes;  // code staging, then (WITH_Y) fp32 staging
+  const uint32_t smem_epi = smem_res_b + Cfg::kResidentBytes;  // packed weights before the unpack, then (WITH_Y) fp32 staging
   const uint32_t smem_scale = smem_epi + Cfg::kEpiBytes;
 
   const int warp = threadIdx.x >> 5;
@@ -193,7 +202,6 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     abort_flag = 0;
     tma_prefetch_desc(&tm_a);
     tma_prefetch_desc(&tm_b);
-    tma_prefetch_desc(&tm_q);
     if (WITH_Y) tma_prefetch_desc(&tm_y);
     if (WITH_Y && p.residual != nullptr) tma_prefetch_desc(&tm_r);
     for (int s = 0; s < STAGES; ++s) {
@@ -207,6 +215,10 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     for (int w = 0; w < EW; ++w) mbar_init(smem_u32(&res_bar[w]), 1);
     mbar_init(smem_u32(&b_loaded_bar), 1);
     mbar_init(smem_u32(&b_ready_bar), EW);
+    for (int b = 0; b < kSlots; ++b) {
+      mbar_init(smem_u32(&ctx_ready_bar[b]), 1);
+      mbar_init(smem_u32(&ctx_free_bar[b]), EW);
+    }
     fence_barrier_init();
     fence_proxy_async_smem();
   }
@@ -224,7 +236,7 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     asm volatile("st.shared.f32 [%0], %1;" ::"r"(smem_scale + t * 4), "f"(wv) : "memory");
     asm volatile("st.shared.f32 [%0], %1;" ::"r"(smem_scale + (BN + t) * 4), "f"(bv) : "memory");
   }
-  if (threadIdx.x < 8) quad_arrivals[threadIdx.x >> 2][threadIdx.x & 3] = 0u;
+  if (threadIdx.x < 4 * kSlots) quad_arrivals[threadIdx.x >> 2][threadIdx.x & 3] = 0u;
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -287,6 +299,50 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         if (ok) tc_commit(smem_u32(&tmem_full_bar[buf]));
       }
     }
+  } else if (warp == 2 + EW) {
+    // ------------------------------------------------------------------ exchange warp
+    // Lane l owns rows 4l .. 4l+3 of the tile: one 16-byte load per n-tile (the warp's request
+    // covers the n-tile's 128 words), kExchangeBatch of them in flight.
+    bool ok = true;
+    for (int i = 0; ok && i < n_my; ++i) {
+      const int tm = group + i * groups;
+      const uint32_t par = i % kSlots, ph = (i / kSlots) & 1;
+      if (!mbar_wait(smem_u32(&ctx_free_bar[par]), ph ^ 1, &abort_flag, t_start)) break;
+      const uint32_t* xt = rp.exchange + (size_t)tm * p.tiles_n * kBM + 4 * lane;
+      uint4 m4 = make_uint4(0u, 0u, 0u, 0u);
+      for (int t0 = 0; ok && t0 < p.tiles_n; t0 += kExchangeBatch) {
+        // all loads of the batch in flight at once; the whole batch is asked for again until every word is valid
+        for (uint32_t spin = 1;; ++spin) {
+          uint4 w[kExchangeBatch];
+#pragma unroll
+          for (int t = 0; t < kExchangeBatch; ++t)
+            w[t] = t0 + t < p.tiles_n ? ld_relaxed_gpu_v4(xt + (size_t)(t0 + t) * kBM) : make_uint4(kValidBit, kValidBit, kValidBit, kValidBit);
+          uint32_t all = kValidBit;
+          uint4 b4 = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+          for (int t = 0; t < kExchangeBatch; ++t) {
+            all &= w[t].x & w[t].y & w[t].z & w[t].w;
+            b4.x = max(b4.x, w[t].x & ~kValidBit);
+            b4.y = max(b4.y, w[t].y & ~kValidBit);
+            b4.z = max(b4.z, w[t].z & ~kValidBit);
+            b4.w = max(b4.w, w[t].w & ~kValidBit);
+          }
+          if (__all_sync(0xffffffffu, (all & kValidBit) != 0u)) {
+            m4.x = max(m4.x, b4.x);
+            m4.y = max(m4.y, b4.y);
+            m4.z = max(m4.z, b4.z);
+            m4.w = max(m4.w, b4.w);
+            break;
+          }
+          if ((spin & 0xF) == 0 && !__all_sync(0xffffffffu, keep_waiting(&abort_flag, t_start))) { ok = false; break; }  // warp-uniform
+        }
+      }
+      if (!__all_sync(0xffffffffu, ok)) break;
+      // final maxima of rows 4l .. 4l+3 for the epilogue warps
+      *reinterpret_cast<uint4*>(&row_amax[par][4 * lane]) = m4;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctx_ready_bar[par]));
+    }
   } else {
     // ------------------------------------------------------------------ epilogue warps
     const int ew = warp - 2;
@@ -294,8 +350,7 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     const int cpart = ew >> 2;   // which 32 columns of the tile
     const int col = cpart * 32;
     const int row_in_tile = quad * 32 + lane;
-    const uint32_t code_buf = smem_epi + ew * Cfg::kCodeBufBytes;
-    const uint32_t y_buf = smem_epi + Cfg::kCodeBytes + ew * kStageBufBytes;
+      const uint32_t y_buf = smem_epi + ew * kStageBufBytes;
     const uint32_t c_sw = smem_scale + (uint32_t)col * 4, c_bias = c_sw + BN * 4;
     const bool has_res = WITH_Y && p.residual != nullptr;
     const int oc = tn * BN + col;  // first output column of this warp
@@ -339,14 +394,7 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       tma_load_2d(y_buf, &tm_r, cols_ok ? oc : 0, r0 < p.M ? r0 : 0, smem_u32(&res_bar[ew]));
     }
 
-    for (int i = 0; ok && i <= n_my; ++i) {
-      // exchange words of tile i - 1 for this thread's row, one per n-tile: requested now, used in pass 2
-      uint32_t xw[kPrefetchWords];
-      const uint32_t* xrow = rp.exchange + (size_t)(group + (i > 0 ? i - 1 : 0) * groups) * p.tiles_n * kBM + row_in_tile;
-      if (i >= 1) {
-#pragma unroll
-        for (int t = 0; t < kPrefetchWords; ++t) xw[t] = t < p.tiles_n ? ld_relaxed_gpu(xrow + (size_t)t * kBM) : kValidBit;
-      }
+    for (int i = 0; ok && i < n_my + kLag; ++i) {
       if (i < n_my) {
         // -------------------------------------------------------------- pass 1 of tile i
         const int tm = group + i * groups;
@@ -362,10 +410,7 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         tmem_ld_32x32(taddr, acc);
         tmem_ld_wait();
         dequant32<SMALL>(acc, sx, c_sw, c_bias, a);
-        if (p.act == AQT_ACT_SWISH) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) a[j] = a[j] * sigmoid_f(a[j]);
-        }
+        if (p.act == AQT_ACT_SWISH) swish32(a);
         if (has_res) {
           if (!mbar_wait(smem_u32(&res_bar[ew]), i & 1, &abort_flag, t_start)) { ok = false; break; }
 #pragma unroll
@@ -388,20 +433,20 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         }
         tmem_st_32x32(taddr, acc);
         // this warp's part of the row maxima (columns beyond N contribute nothing)
-        amax_part[i & 1][cpart][row_in_tile] = cols_ok ? __float_as_uint(amax) : 0u;
-        tmem_st_wait();
+        amax_part[i % kSlots][cpart][row_in_tile] = cols_ok ? __float_as_uint(amax) : 0u;
         __syncwarp();
         int last = 0;
         if (lane == 0) {
           __threadfence_block();
-          last = (atomicAdd(&quad_arrivals[i & 1][quad], 1u) & 3u) == 3u ? 1 : 0;
+          last = (atomicAdd(&quad_arrivals[i % kSlots][quad], 1u) & 3u) == 3u ? 1 : 0;
           __threadfence_block();
         }
         last = __shfl_sync(0xffffffffu, last, 0);
         if (last) {
           // the last of the quadrant's four warps publishes the CTA's maxima of these 32 rows
-          const uint32_t v = max(max(amax_part[i & 1][0][row_in_tile], amax_part[i & 1][1][row_in_tile]),
-                                 max(amax_part[i & 1][2][row_in_tile], amax_part[i & 1][3][row_in_tile]));
+          const uint32_t sl = i % kSlots;
+          const uint32_t v = max(max(amax_part[sl][0][row_in_tile], amax_part[sl][1][row_in_tile]),
+                                 max(amax_part[sl][2][row_in_tile], amax_part[sl][3][row_in_tile]));
           st_relaxed_gpu(rp.exchange + ((size_t)tm * p.tiles_n + tn) * kBM + row_in_tile, v | kValidBit);
         }
 
@@ -434,58 +479,40 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         }
 
       }
-      if (i >= 1) {
-        // -------------------------------------------------------------- pass 2 of tile i - 1
-        const int tm = group + (i - 1) * groups;
-        const uint32_t buf = (i - 1) & 3;
+      if (i >= kLag) {
+        // -------------------------------------------------------------- pass 2 of tile i - kLag
+        const int j = i - kLag;
+        const int tm = group + j * groups;
+        const uint32_t buf = j & 3;
         const int row0_warp = tm * kBM + quad * 32;
-        const int m = row0_warp + lane;
-        uint32_t amax_bits = 0u;
-        bool valid = true;
-#pragma unroll
-        for (int t = 0; t < kPrefetchWords; ++t) {
-          if (t < p.tiles_n) valid = valid && wait_valid(xrow + (size_t)t * kBM, xw[t], &abort_flag, t_start);
-          amax_bits = max(amax_bits, xw[t] & ~kValidBit);
-        }
-        for (int t = kPrefetchWords; valid && t < p.tiles_n; ++t) {
-          uint32_t w = 0u;
-          valid = wait_valid(xrow + (size_t)t * kBM, w, &abort_flag, t_start);
-          amax_bits = max(amax_bits, w & ~kValidBit);
-        }
-        if (!__all_sync(0xffffffffu, valid)) { ok = false; break; }
-        const float amax = __uint_as_float(amax_bits);
+        const uint32_t par = j % kSlots;
+        if (!mbar_wait(smem_u32(&ctx_ready_bar[par]), (j / kSlots) & 1, &abort_flag, t_start)) { ok = false; break; }
+        const float amax = __uint_as_float(row_amax[par][row_in_tile]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctx_free_bar[par]));
         const ScaleCtx c = make_scale_ctx(amax, rp.qmax_out);
-        if (tn == 0 && cpart == 0 && m < p.M) rp.s_out[m] = c.s;
+        if (tn == 0 && cpart == 0 && row0_warp + lane < p.M) rp.s_out[row0_warp + lane] = c.s;
         const uint32_t taddr = tmem_base + buf * BN + ((uint32_t)(quad * 32) << 16) + col;
         uint32_t u[32], w[8];
+        tmem_st_wait();  // this warp's stores of pass 1 (long complete)
         tmem_ld_32x32(taddr, u);
         tmem_ld_wait();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[buf]));
-        if (rp.pack_out) {
-          if (rp.rounding == AQT_ROUND_HALF_UP_FLOOR) codes32<AQT_ROUND_HALF_UP_FLOOR, true>(u, c, rp.qmax_out, w);
-          else codes32<AQT_ROUND_NEAREST_EVEN, true>(u, c, rp.qmax_out, w);
-        } else {
-          if (rp.rounding == AQT_ROUND_HALF_UP_FLOOR) codes32<AQT_ROUND_HALF_UP_FLOOR, false>(u, c, rp.qmax_out, w);
-          else codes32<AQT_ROUND_NEAREST_EVEN, false>(u, c, rp.qmax_out, w);
-        }
-        if (lane == 0) tma_store_wait_read<0>();  // the store that last used the code buffer has read it out
-        __syncwarp();
-        if (rp.pack_out) {
-          // 32 rows of 16 bytes, dense
-          asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(code_buf + lane * 16), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
-        } else {
-          // 32 rows of 32 bytes under the 32-byte swizzle: 16-byte half h of row r sits at h ^ ((r >> 2) & 1)
-          const uint32_t sw = (uint32_t)((lane >> 2) & 1);
-          asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(code_buf + lane * 32 + ((0u ^ sw) << 4)), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
-          asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(code_buf + lane * 32 + ((1u ^ sw) << 4)), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
-        }
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) {
-          if (cols_ok && row0_warp < p.M) tma_store_2d(&tm_q, code_buf, rp.pack_out ? oc / 2 : oc, row0_warp);
-          tma_store_commit();
+        codes32<ROUNDING, PACK_OUT>(u, c, rp.qmax_out, w);
+        // Each thread holds 32 consecutive codes of its row: one or two 16-byte stores, each a
+        // whole 32-byte sector (or half of one for packed nibbles), straight to global memory.
+        const int m = row0_warp + lane;
+        if (m < p.M && cols_ok) {
+          if (PACK_OUT) {
+            uint4* dst = reinterpret_cast<uint4*>(rp.q_out + (size_t)m * (p.N / 2) + oc / 2);
+            *dst = make_uint4(w[0], w[1], w[2], w[3]);
+          } else {
+            uint4* dst = reinterpret_cast<uint4*>(rp.q_out + (size_t)m * p.N + oc);
+            dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+            if (oc + 16 < p.N) dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+          }
         }
       }
     }
@@ -519,7 +546,7 @@ static bool requant_applies(int64_t M, int64_t N, int64_t K, int act) {
   return M > 0 && ceil_div(K, kBK) <= kWsMaxKBlocks && ceil_div(N, 128) <= sms && (act == AQT_ACT_NONE || act == AQT_ACT_SWISH);
 }
 
-template <bool BPACK, bool SMALL, bool WITH_Y>
+template <bool BPACK, bool SMALL, bool WITH_Y, int ROUNDING, bool PACK_OUT>
 static int launch_requant_inst(const int8_t* a, const void* b, void* q_out, float* y, int64_t ldy, RequantParams rp,
                                void* exchange, cudaStream_t st) {
   using Cfg = RequantCfg<WITH_Y>;
@@ -533,15 +560,13 @@ static int launch_requant_inst(const int8_t* a, const void* b, void* q_out, floa
   rp.exchange = reinterpret_cast<uint32_t*>(exchange);
   AQT_RETURN_IF_CUDA(cudaMemsetAsync(exchange, 0, (size_t)p.tiles_m * p.tiles_n * kBM * 4, st));
 
-  CUtensorMap tm_a, tm_b, tm_q, tm_y, tm_r;
+  CUtensorMap tm_a, tm_b, tm_y, tm_r;
   int rc = make_map_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, a, (uint64_t)p.M, (uint64_t)p.K, (uint64_t)p.K, kBM, kBK);
   if (rc != AQT_OK) return rc;
   if (BPACK) rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, b, (uint64_t)p.N, (uint64_t)p.K / 2, (uint64_t)p.K / 2, Cfg::BN / 2, 64, 0);
   else rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, b, (uint64_t)p.N, (uint64_t)p.K, (uint64_t)p.K, Cfg::BN / 2, kBK);
   if (rc != AQT_OK) return rc;
-  if (rp.pack_out) rc = make_map_2d(&tm_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, q_out, (uint64_t)p.M, (uint64_t)p.N / 2, (uint64_t)p.N / 2, 32, 16, 0);
-  else rc = make_map_2d(&tm_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, q_out, (uint64_t)p.M, (uint64_t)p.N, (uint64_t)p.N, 32, 32, 32);
-  if (rc != AQT_OK) return rc;
+  rp.q_out = reinterpret_cast<uint8_t*>(q_out);
   tm_y = tm_a;
   tm_r = tm_a;
   if (WITH_Y) {
@@ -553,7 +578,7 @@ static int launch_requant_inst(const int8_t* a, const void* b, void* q_out, floa
       if (rc != AQT_OK) return rc;
     }
   }
-  auto kernel = qgemm_requant_kernel<BPACK, SMALL, WITH_Y>;
+  auto kernel = qgemm_requant_kernel<BPACK, SMALL, WITH_Y, ROUNDING, PACK_OUT>;
   static bool attr_set = false;
   if (!attr_set) {
     AQT_RETURN_IF_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
@@ -571,7 +596,7 @@ static int launch_requant_inst(const int8_t* a, const void* b, void* q_out, floa
   attr[0].val.cooperative = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  AQT_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, kernel, tm_a, tm_b, tm_q, tm_y, tm_r, rp));
+  AQT_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, kernel, tm_a, tm_b, tm_y, tm_r, rp));
   return AQT_LAUNCH_STATUS();
 }
 
@@ -580,7 +605,13 @@ static int launch_requant_inst(const int8_t* a, const void* b, void* q_out, floa
 static int launch_requant(const int8_t* a, const void* b, bool b_packed, void* q_out, float* y, int64_t ldy, const RequantParams& rp,
                           void* exchange, cudaStream_t st) {
   const bool small = rp.g.small_acc != 0;
-#define AQT_RQ(BP, SM, WY) launch_requant_inst<BP, SM, WY>(a, b, q_out, y, ldy, rp, exchange, st)
+#define AQT_RQ(BP, SM, WY)                                                                                                 \
+  (rp.pack_out ? (rp.rounding == AQT_ROUND_HALF_UP_FLOOR                                                                     \
+                      ? launch_requant_inst<BP, SM, WY, AQT_ROUND_HALF_UP_FLOOR, true>(a, b, q_out, y, ldy, rp, exchange, st) \
+                      : launch_requant_inst<BP, SM, WY, AQT_ROUND_NEAREST_EVEN, true>(a, b, q_out, y, ldy, rp, exchange, st)) \
+               : (rp.rounding == AQT_ROUND_HALF_UP_FLOOR                                                                     \
+                      ? launch_requant_inst<BP, SM, WY, AQT_ROUND_HALF_UP_FLOOR, false>(a, b, q_out, y, ldy, rp, exchange, st) \
+                      : launch_requant_inst<BP, SM, WY, AQT_ROUND_NEAREST_EVEN, false>(a, b, q_out, y, ldy, rp, exchange, st)))
   if (y != nullptr) {
     if (b_packed) return small ? AQT_RQ(true, true, true) : AQT_RQ(true, false, true);
     return small ? AQT_RQ(false, true, true) : AQT_RQ(false, false, true);

@@ -291,19 +291,47 @@ __device__ __forceinline__ float acc_to_float(uint32_t acc) {
   return __int2float_rn((int)acc);
 }
 
+// Two accumulators -> two floats (see acc_to_float); the subtraction is one packed add.
+template <bool SMALL>
+__device__ __forceinline__ float2 acc_to_float2(uint32_t a0, uint32_t a1) {
+  if (SMALL)
+    return __fadd2_rn(make_float2(__int_as_float(0x4B400000 + (int)a0), __int_as_float(0x4B400000 + (int)a1)),
+                      make_float2(-12582912.0f, -12582912.0f));
+  return make_float2(__int2float_rn((int)a0), __int2float_rn((int)a1));
+}
+
 // z[i] = fma(float(acc[i]) * sx, s_w[i], bias[i]) for 32 consecutive columns whose scales and
-// biases sit at `sw_smem` / `b_smem` (shared-memory byte addresses, 16-byte aligned).
+// biases sit at `sw_smem` / `b_smem` (shared-memory byte addresses, 16-byte aligned).  The
+// arithmetic runs on the packed two-lane fp32 instructions of this architecture (each lane an
+// ordinary round-to-nearest IEEE operation), which halves the issue slots it takes.
 template <bool SMALL>
 __device__ __forceinline__ void dequant32(const uint32_t (&acc)[32], float sx, uint32_t sw_smem, uint32_t b_smem, float (&z)[32]) {
+  const float2 sx2 = make_float2(sx, sx);
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     float w0, w1, w2, w3, b0, b1, b2, b3;
     asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(w0), "=f"(w1), "=f"(w2), "=f"(w3) : "r"(sw_smem + 16 * j));
     asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(b0), "=f"(b1), "=f"(b2), "=f"(b3) : "r"(b_smem + 16 * j));
-    z[4 * j + 0] = __fmaf_rn(__fmul_rn(acc_to_float<SMALL>(acc[4 * j + 0]), sx), w0, b0);
-    z[4 * j + 1] = __fmaf_rn(__fmul_rn(acc_to_float<SMALL>(acc[4 * j + 1]), sx), w1, b1);
-    z[4 * j + 2] = __fmaf_rn(__fmul_rn(acc_to_float<SMALL>(acc[4 * j + 2]), sx), w2, b2);
-    z[4 * j + 3] = __fmaf_rn(__fmul_rn(acc_to_float<SMALL>(acc[4 * j + 3]), sx), w3, b3);
+    const float2 z01 = __ffma2_rn(__fmul2_rn(acc_to_float2<SMALL>(acc[4 * j + 0], acc[4 * j + 1]), sx2), make_float2(w0, w1), make_float2(b0, b1));
+    const float2 z23 = __ffma2_rn(__fmul2_rn(acc_to_float2<SMALL>(acc[4 * j + 2], acc[4 * j + 3]), sx2), make_float2(w2, w3), make_float2(b2, b3));
+    z[4 * j + 0] = z01.x;
+    z[4 * j + 1] = z01.y;
+    z[4 * j + 2] = z23.x;
+    z[4 * j + 3] = z23.y;
+  }
+}
+
+// a[i] = a[i] * sigmoid(a[i]) (see sigmoid_f) for 32 values, two per instruction where the
+// operation is an IEEE multiply or add.
+__device__ __forceinline__ void swish32(float (&a)[32]) {
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const float2 z = make_float2(a[2 * j], a[2 * j + 1]);
+    const float2 t = __fmul2_rn(z, make_float2(-1.4426950408889634f, -1.4426950408889634f));
+    const float2 d = __fadd2_rn(make_float2(1.0f, 1.0f), make_float2(ex2_approx(t.x), ex2_approx(t.y)));
+    const float2 y = __fmul2_rn(z, make_float2(rcp_approx(d.x), rcp_approx(d.y)));
+    a[2 * j] = y.x;
+    a[2 * j + 1] = y.y;
   }
 }
 
@@ -673,10 +701,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           }
           if (Cfg::kScaleSlab) dequant32<SMALL>(acc, sx, c_sw, c_bias, a);
           else dequant32_gmem<SMALL>(acc, sx, p.s_w, p.bias, tn * BN + col, p.N, a);
-          if (p.act == AQT_ACT_SWISH) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) a[j] = a[j] * sigmoid_f(a[j]);
-          }
+          if (p.act == AQT_ACT_SWISH) swish32(a);
         } else {
           // gates first: g = sigmoid(z_gate); then the values are scaled by it
           float g[32];
@@ -714,10 +739,8 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           if (Cfg::kScaleSlab) dequant32<SMALL>(acc, sx, c_sw, c_bias, a);
           else dequant32_gmem<SMALL>(acc, sx, p.s_w, p.bias, oc, p.N / 2, a);
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            a[j] = a[j] * g[j];
-            if (p.act == AQT_ACT_GLU_SWISH) a[j] = a[j] * sigmoid_f(a[j]);
-          }
+          for (int j = 0; j < 32; ++j) a[j] = a[j] * g[j];
+          if (p.act == AQT_ACT_GLU_SWISH) swish32(a);
         }
 
         // the chunk this warp handles after this one (for the residual prefetch)

@@ -13,7 +13,10 @@ and are replaced by the identity:
     h <- h + W_pw2 . c                              pointwise 2
     h <- h + 1/2 * W_b2 . Swish(W_b1 . h)          feed-forward module b
 
-Residual adds are fp32 and are fused into the epilogue of the producing linear.
+Residual adds are fp32 and are fused into the epilogue of the producing linear.  Where a linear
+with K <= 512 and no GLU feeds another quantized linear, its epilogue also quantizes its output
+rows (aqt_qmatmul_requant): the fp32 tensor between the two is then written only if it is needed
+as well (the residual stream, or a parity check).
 """
 from __future__ import annotations
 
@@ -55,8 +58,10 @@ class LayerRunner:
     def __init__(self, M: int, layers: List[QuantLinear], device, a_scale_kind: int = aqt.SCALE_ROW,
                  rounding: int = aqt.ROUND_NEAREST_EVEN):
         self.M, self.device, self.a_scale_kind, self.rounding = M, device, a_scale_kind, rounding
-        need = max(aqt.aqt_workspace_bytes(aqt.OP_LINEAR_FWD, M, 3 * l.spec.N, l.spec.K, l.spec.bits_a, l.spec.bits_w) for l in layers)
+        need = max(max(aqt.aqt_workspace_bytes(op, M, 3 * l.spec.N, l.spec.K, l.spec.bits_a, l.spec.bits_w)
+                       for op in (aqt.OP_LINEAR_FWD, aqt.OP_QMATMUL_REQUANT)) for l in layers)
         self.workspace = torch.empty(need, dtype=torch.uint8, device=device)
+        self._codes: Dict[str, tuple] = {}
 
     def quantize_input(self, x: torch.Tensor, bits_a: int):
         """Activation codes (int8 containers) and scales of x, for several layers that read the
@@ -69,11 +74,36 @@ class LayerRunner:
         aqt.aqt_quantize(x, bits_a, axis, self.rounding, q_out=self._shared_q, scale_out=self._shared_s)
         return self._shared_q, self._shared_s
 
-    def matmul(self, layer: QuantLinear, xq: torch.Tensor, s_x: torch.Tensor, y: torch.Tensor) -> torch.Tensor:
+    def matmul(self, layer: QuantLinear, xq: torch.Tensor, s_x: torch.Tensor, y: torch.Tensor,
+               residual: Optional[torch.Tensor] = None, residual_scale: float = 1.0) -> torch.Tensor:
         """Integer matmul + epilogue of `layer` on already-quantized activations (int8 containers)."""
         s = layer.spec
-        return aqt.aqt_qmatmul(xq, s_x, layer.wq, layer.s_w, layer.bias, None, 1.0, K=s.K, bits_a=8, bits_w=s.bits_w, act=s.act,
-                               s_x_kind=self.a_scale_kind, y=y, workspace=self.workspace)
+        return aqt.aqt_qmatmul(xq, s_x, layer.wq, layer.s_w, layer.bias, residual, residual_scale, K=s.K, bits_a=8, bits_w=s.bits_w,
+                               act=s.act, s_x_kind=self.a_scale_kind, y=y, workspace=self.workspace)
+
+    def fuses_requant(self, layer: QuantLinear) -> bool:
+        """True if `layer`'s matmul can quantize its own output rows in its epilogue."""
+        s = layer.spec
+        return (self.a_scale_kind == aqt.SCALE_ROW and s.K <= 512 and s.K % 16 == 0 and s.act in (aqt.ACT_NONE, aqt.ACT_SWISH)
+                and s.N % 16 == 0 and s.N <= 128 * 148)
+
+    def code_buffers(self, role: str, cols: int):
+        """Codes (int8 containers) and row scales of an activation tensor, one pair of buffers per role."""
+        if role not in self._codes or self._codes[role][0].shape[1] != cols:
+            self._codes[role] = (torch.empty((self.M, cols), dtype=torch.int8, device=self.device),
+                                 torch.empty(self.M, dtype=torch.float32, device=self.device))
+        return self._codes[role]
+
+    def matmul_requant(self, layer: QuantLinear, xq: torch.Tensor, s_x: torch.Tensor, bits_out: int, role: str,
+                       y: Optional[torch.Tensor] = None, residual: Optional[torch.Tensor] = None, residual_scale: float = 1.0):
+        """`layer` on quantized activations, its output rows quantized to `bits_out` bits in the
+        epilogue.  Returns (codes, scales); y (fp32) is written too if given."""
+        s = layer.spec
+        q, sc = self.code_buffers(role, s.n_out)
+        aqt.aqt_qmatmul_requant(xq, s_x, layer.wq, layer.s_w, layer.bias, residual, residual_scale, K=s.K, bits_a=8,
+                                bits_w=s.bits_w, act=s.act, s_x_kind=self.a_scale_kind, bits_out=bits_out,
+                                rounding=self.rounding, pack_out=False, q_out=q, s_out=sc, y=y, workspace=self.workspace)
+        return q, sc
 
     def __call__(self, layer: QuantLinear, x: torch.Tensor, y: torch.Tensor, residual: Optional[torch.Tensor] = None,
                  residual_scale: float = 1.0) -> torch.Tensor:
@@ -84,17 +114,36 @@ class LayerRunner:
 
 
 class FfnPair:
-    """y = W_2 . Swish(W_1 . x): the second layer re-quantizes the first layer's fp32 output."""
+    """y = W_2 . Swish(W_1 . x).  The second layer consumes the first layer's output as codes and
+    row scales; the first matmul produces them in its epilogue when it can (`fused`), and the fp32
+    hidden tensor u is then written only with keep_u (parity checks)."""
 
-    def __init__(self, M: int, layers: List[QuantLinear], device, **kw):
+    def __init__(self, M: int, layers: List[QuantLinear], device, fused: bool = True, keep_u: bool = False, **kw):
         assert len(layers) == 2
         self.layers = layers
         self.run = LayerRunner(M, layers, device, **kw)
-        self.u = torch.empty((M, layers[0].spec.n_out), dtype=torch.float32, device=device)
+        self.fused = fused and self.run.fuses_requant(layers[0])
+        self.keep_u = keep_u or not self.fused
+        self.u = torch.empty((M, layers[0].spec.n_out), dtype=torch.float32, device=device) if self.keep_u else None
 
     def forward(self, x: torch.Tensor, y: torch.Tensor) -> torch.Tensor:
-        self.run(self.layers[0], x, self.u)
-        return self.run(self.layers[1], self.u, y)
+        if not self.fused:
+            self.run(self.layers[0], x, self.u)
+            return self.run(self.layers[1], self.u, y)
+        l0, l1 = self.layers
+        xq, xs = self.run.quantize_input(x, l0.spec.bits_a)
+        uq, us = self.run.matmul_requant(l0, xq, xs, l1.spec.bits_a, "u", y=self.u)
+        return self.run.matmul(l1, uq, us, y)
+
+    @property
+    def launches_per_step(self) -> int:
+        """Kernels of the library launched by one forward()."""
+        l0, l1 = self.layers
+        unpack2 = 1 if (l1.spec.bits_w == 4 and l1.spec.K > 512) else 0
+        if self.fused:
+            return 3 + unpack2
+        unpack1 = 1 if (l0.spec.bits_w == 4 and l0.spec.K > 512) else 0
+        return 4 + unpack1 + unpack2
 
     @property
     def ops(self) -> int:
@@ -128,8 +177,9 @@ class ConformerBlockLinears:
             if keep is not None:
                 keep[name] = t.clone()
 
-        run(L[0], h_in, self.u); note(L[0].spec.name, self.u)
-        run(L[1], self.u, self.h_a, residual=h_in, residual_scale=0.5); note(L[1].spec.name, self.h_a)
+        parity = keep is not None  # then every fp32 intermediate is written as well
+        self._ffn(L[0], L[1], h_in, self.h_a, 0.5, parity, note)
+        note(L[1].spec.name, self.h_a)
         # q, k, v read the same h: quantize it once (the codes do not depend on the consumer) and
         # run the three projections as one matmul over their concatenated output channels
         hq, hs = run.quantize_input(self.h_a, L[2].spec.bits_a)
@@ -137,12 +187,41 @@ class ConformerBlockLinears:
         aqt.aqt_qmatmul(hq, hs, wq, s_w, bias, None, 1.0, K=self.d, bits_a=8, bits_w=L[2].spec.bits_w, act=aqt.ACT_NONE,
                         s_x_kind=run.a_scale_kind, y=self.qkv, workspace=run.workspace)
         note(L[2].spec.name, self.q); note(L[3].spec.name, self.k); note(L[4].spec.name, self.v)
-        run(L[5], self.v, self.h_b, residual=self.h_a, residual_scale=1.0); note(L[5].spec.name, self.h_b)
-        run(L[6], self.h_b, self.c); note(L[6].spec.name, self.c)
-        run(L[7], self.c, self.h_a, residual=self.h_b, residual_scale=1.0); note(L[7].spec.name, self.h_a)
-        run(L[8], self.h_a, self.u); note(L[8].spec.name, self.u)
-        run(L[9], self.u, h_out, residual=self.h_a, residual_scale=0.5); note(L[9].spec.name, h_out)
+        # h_b = h_a + W_o v is needed both as fp32 (residual stream) and as codes (pointwise 1)
+        if run.fuses_requant(L[5]):
+            vq, vs = run.quantize_input(self.v, L[5].spec.bits_a)
+            bq, bs = run.matmul_requant(L[5], vq, vs, L[6].spec.bits_a, "h", y=self.h_b, residual=self.h_a, residual_scale=1.0)
+            note(L[5].spec.name, self.h_b)
+            run.matmul(L[6], bq, bs, self.c); note(L[6].spec.name, self.c)
+        else:
+            run(L[5], self.v, self.h_b, residual=self.h_a, residual_scale=1.0); note(L[5].spec.name, self.h_b)
+            run(L[6], self.h_b, self.c); note(L[6].spec.name, self.c)
+        # h_a = h_b + W_pw2 c, again as fp32 and as codes (first layer of feed-forward module b)
+        if run.fuses_requant(L[7]):
+            cq, cs = run.quantize_input(self.c, L[7].spec.bits_a)
+            aq, as_ = run.matmul_requant(L[7], cq, cs, L[8].spec.bits_a, "h", y=self.h_a, residual=self.h_b, residual_scale=1.0)
+            note(L[7].spec.name, self.h_a)
+            self._ffn(L[8], L[9], self.h_a, h_out, 0.5, parity, note, xq=aq, xs=as_)
+        else:
+            run(L[7], self.c, self.h_a, residual=self.h_b, residual_scale=1.0); note(L[7].spec.name, self.h_a)
+            self._ffn(L[8], L[9], self.h_a, h_out, 0.5, parity, note)
+        note(L[9].spec.name, h_out)
         return h_out
+
+    def _ffn(self, l0: QuantLinear, l1: QuantLinear, h: torch.Tensor, out: torch.Tensor, rs: float, parity: bool, note,
+             xq: Optional[torch.Tensor] = None, xs: Optional[torch.Tensor] = None) -> None:
+        """out = h + rs * W_1 . Swish(W_0 . h); xq, xs: codes and scales of h if already at hand."""
+        run = self.run
+        if run.fuses_requant(l0):
+            if xq is None:
+                xq, xs = run.quantize_input(h, l0.spec.bits_a)
+            uq, us = run.matmul_requant(l0, xq, xs, l1.spec.bits_a, "u", y=self.u if parity else None)
+            if parity:
+                note(l0.spec.name, self.u)
+            run.matmul(l1, uq, us, out, residual=h, residual_scale=rs)
+        else:
+            run(l0, h, self.u); note(l0.spec.name, self.u)
+            run(l1, self.u, out, residual=h, residual_scale=rs)
 
     def _fused_qkv(self, L: List[QuantLinear]):
         """Codes, scales and bias of the q, k, v projections stacked along the output channels

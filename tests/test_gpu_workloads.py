@@ -103,11 +103,19 @@ def test_cfg2_ffn_pair_full_size_sampled_rows():
     q2, s2 = aqt.aqt_quantize(u, 8, aqt.AXIS_ROW)
     y = aqt.aqt_qmatmul(q2, s2, gpu[1].wq, gpu[1].s_w, K=specs[1].K, bits_w=4)
     # the fused entry point gives the same bits
-    pair = FfnPair(w.M, gpu, DEV)
-    y2 = torch.empty_like(y)
-    pair.forward(xd, y2)
-    assert aqt.aqt_device_status() == 0
-    assert torch.equal(y.view(torch.int32), y2.view(torch.int32)) and torch.equal(u.view(torch.int32), pair.u.view(torch.int32))
+    # the pair as bench.py runs it (the first matmul quantizes its own output rows; u is never
+    # written), with u written as well, and as two separate layers: the same bits every way
+    for kw in (dict(), dict(keep_u=True), dict(fused=False)):
+        pair = FfnPair(w.M, gpu, DEV, **kw)
+        y2 = torch.full_like(y, float("nan"))
+        pair.forward(xd, y2)
+        assert aqt.aqt_device_status() == 0
+        assert torch.equal(y.view(torch.int32), y2.view(torch.int32)), kw
+        if pair.u is not None:
+            assert torch.equal(u.view(torch.int32), pair.u.view(torch.int32)), kw
+        else:
+            uq, us = pair.run.code_buffers("u", specs[0].N)
+            assert torch.equal(uq, q2) and torch.equal(us.view(torch.int32), s2.view(torch.int32))
     # codes and scales of both quantizer calls, bit for bit, on the sampled rows
     q_ref, s_ref = orc.quantize(x[rows], 8, orc.AXIS_ROW)
     assert np.array_equal(q1.cpu().numpy()[rows], q_ref) and np.array_equal(s1.cpu().numpy()[rows], s_ref)
