@@ -116,3 +116,29 @@ def test_requant_unfused_shapes_go_through_y():
     with pytest.raises(aqt.AqtError) as e:
         aqt.aqt_qmatmul_requant(_dev(xq), _dev(np.ones(64, np.float32)), _dev(wq), _dev(np.ones(256, np.float32)), K=1024)
     assert e.value.status == -3
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 512, 512), (16, 2048, 256), (127, 640, 128), (129, 2304, 512), (260, 4224, 64), (3000, 128, 512)])
+def test_requant_edge_shapes(M, N, K):
+    """One row, fewer m-tiles than groups of CTAs, a ragged last m-tile, more than sixteen n-tiles
+    (the exchange warp then reads the row maxima in several batches), a single n-tile."""
+    _run(M, N, K, 8, 8, aqt.ACT_SWISH, True, False, 8, aqt.ROUND_NEAREST_EVEN, False)
+    _run(M, N, K, 8, 4, aqt.ACT_NONE, False, M > 100, 4, aqt.ROUND_HALF_UP_FLOOR, True)
+
+
+def test_requant_argument_checks():
+    z8 = torch.zeros((64, 64), dtype=torch.int8, device=DEV)
+    w8 = torch.zeros((48, 64), dtype=torch.int8, device=DEV)
+    one = torch.ones(64, device=DEV)
+    with pytest.raises(aqt.AqtError) as e:   # N_out not a multiple of 16
+        aqt.aqt_qmatmul_requant(z8, one, w8[:40], one[:40], K=64)
+    assert e.value.status == -1
+    with pytest.raises(aqt.AqtError) as e:   # packing needs 4-bit output codes
+        aqt.aqt_qmatmul_requant(z8, one, w8, one[:48], K=64, bits_out=8, pack_out=True)
+    assert e.value.status == -1
+    with pytest.raises(aqt.AqtError) as e:   # packed rows need N_out % 32 == 0
+        aqt.aqt_qmatmul_requant(z8, one, w8, one[:48], K=64, bits_out=4, pack_out=True)
+    assert e.value.status == -1
+    q, s_, y = aqt.aqt_qmatmul_requant(z8[:0], one[:0], w8, one[:48], K=64)   # empty batch: nothing to do
+    assert q.shape == (0, 48) and y is None
+    assert aqt.aqt_device_status() == 0
