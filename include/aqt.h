@@ -32,7 +32,7 @@
 extern "C" {
 #endif
 
-#define AQT_VERSION 102
+#define AQT_VERSION 103
 
 /* status codes */
 #define AQT_OK 0
@@ -66,6 +66,7 @@ extern "C" {
 #define AQT_OP_QMATMUL 1
 #define AQT_OP_LINEAR_FWD 2
 #define AQT_OP_QMATMUL_REQUANT 3
+#define AQT_OP_LINEAR_WEIGHT_ONLY 4
 
 int aqt_version(void);
 const char* aqt_status_string(int status);
@@ -177,6 +178,32 @@ int aqt_linear_fwd(const float* x, int64_t ldx, const void* wq, const float* s_w
 int aqt_linear_fwd_host(const float* x, int x_on_host, const void* wq, const float* s_w, const float* bias,
                         int64_t M, int64_t N, int64_t K, int bits_a, int bits_w, int a_scale_kind, int rounding,
                         int act, float* y, int y_on_host, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * aqt_linear_fwd_weight_only -- the layer of the weight-only configurations (Section 4.1: "I8W":
+ * int8 weight, float32 activation; "I4W": int4 weight, float32 activation; "we still need to
+ * convert the weights to float during inference").  Activations are not quantized; the stored
+ * codes are converted to float and de-quantized by their channel scale (Section 2.2):
+ *   z[m][n] = s_w[n] * sum_k x[m][k] * float(wq[n][k]) + bias[n]
+ *   a = act(z);  y = residual ? fma(residual_scale, a, residual) : a
+ * Arithmetic: a float matmul on the tensor cores.  The weight codes are exact as floats; each
+ * activation enters its product with sign, exponent and the upper ten fraction bits of its
+ * binary32 value (the tf32 operand format; whether the dropped bits are truncated or rounded is
+ * the hardware's), products are exact and are summed into binary32 accumulators.  The result is
+ * therefore within 2^-10 * s_w[n] * sum_k |x[m][k] * wq[n][k]| (plus binary32 summation error) of
+ * the exact value of the formula, and equals it bit for bit when every x is a tf32 value and no
+ * partial sum needs more than 24 bits.
+ * x         fp32 [M, K], row pitch ldx elements.
+ * wq, s_w, bias, residual, ldr, residual_scale, act, y, ldy: as for aqt_qmatmul.
+ * workspace at least aqt_workspace_bytes(AQT_OP_LINEAR_WEIGHT_ONLY, M, N, K, 0, bits_w) bytes,
+ *           256-byte aligned: the weight codes as floats (4 * N * K bytes), rewritten every call.
+ * Limits: K % 4 == 0, ldx % 4 == 0, N % 4 == 0 (N % 8 == 0 for GLU), ldy % 4 == 0, ldr % 4 == 0;
+ * x, wq, y, residual, s_w, bias 16-byte aligned.  M == 0 or N == 0 is a no-op.
+ */
+int aqt_linear_fwd_weight_only(const float* x, int64_t ldx, const void* wq, const float* s_w, const float* bias,
+                               const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K,
+                               int bits_w, int act, float* y, int64_t ldy, void* workspace, size_t workspace_bytes,
+                               void* stream);
 
 /*
  * aqt_qmatmul_w4_noalloc -- aqt_qmatmul for int8 activations and 4-bit weights that needs no

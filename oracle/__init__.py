@@ -187,3 +187,27 @@ def linear_fwd(x, wq, s_w, bias=None, residual=None, residual_scale=1.0, bits_a=
     if rc != 0:
         raise ValueError("orc_linear_fwd: bad argument")
     return (y, xq, sx, acc) if return_parts else y
+
+
+def linear_weight_only_f64(x, wq, s_w, bias=None, residual=None, residual_scale=1.0, act=ACT_NONE, return_parts=False):
+    """The weight-only layer (float activations, integer weights de-quantized by their channel
+    scale) in double.  With return_parts also returns (z, mag): pre-activations and the magnitude
+    s_w * sum_k |x * wq| of each."""
+    x = np.asarray(x, dtype=np.float32)
+    assert x.ndim == 2 and x.strides[1] == 4
+    wq = np.ascontiguousarray(wq, dtype=np.int8)
+    M, K = x.shape
+    ldx = x.strides[0] // 4 if M > 1 else K
+    N = wq.shape[0]
+    assert wq.shape[1] == K
+    y = np.empty((M, _n_out(N, act)), dtype=np.float64)
+    z = np.empty((M, N), dtype=np.float64) if return_parts else None
+    mag = np.empty((M, N), dtype=np.float64) if return_parts else None
+    s_w = np.ascontiguousarray(s_w, dtype=np.float32)
+    bias = None if bias is None else np.ascontiguousarray(bias, dtype=np.float32)
+    residual = None if residual is None else np.ascontiguousarray(residual, dtype=np.float32)
+    rc = lib().orc_linear_weight_only_f64(_p(x), _i64(ldx), _p(wq), _p(s_w), _p(bias), _p(residual), _i64(y.shape[1]),
+                                          ctypes.c_float(residual_scale), _i64(M), _i64(N), _i64(K), act, _p(y), _p(z), _p(mag))
+    if rc != 0:
+        raise ValueError("orc_linear_weight_only_f64: bad argument")
+    return (y, z, mag) if return_parts else y

@@ -306,3 +306,49 @@ int orc_linear_fwd(const float* x, int64_t ldx, const int8_t* wq, const float* s
   if (!acc_out) free(acc);
   return rc;
 }
+
+/* The layer of the weight-only configurations of Section 4.1 ("I8W": int8 weight, float32
+ * activation; "I4W": int4 weight, float32 activation; the weights are converted to float at
+ * inference).  Activations are not quantized; de-quantization multiplies the codes by their
+ * channel scale (Section 2.2).  The plain definition, every operation in double:
+ *   z[m][n] = s_w[n] * sum_k x[m][k] * wq[n][k] + bias[n]
+ * (each product of a binary32 value and a code is exact in double; the sum is rounded only at the
+ * 2^-53 level.)  Activation and residual as in orc_epilogue_f64.
+ * y is double [M, n_out] dense.  Optional outputs, double [M, N] dense: z_out, the
+ * pre-activations; mag_out, s_w[n] * sum_k |x[m][k] * wq[n][k]|, the magnitude against which a
+ * float implementation's rounding is measured. */
+int orc_linear_weight_only_f64(const float* x, int64_t ldx, const int8_t* wq, const float* s_w, const float* bias,
+                               const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N,
+                               int64_t K, int act, double* y, double* z_out, double* mag_out) {
+  const int glu = (act == ORC_ACT_GLU || act == ORC_ACT_GLU_SWISH);
+  if (M < 0 || N < 0 || K < 0 || ldx < K) return -1;
+  if (glu && (N % 2 != 0)) return -1;
+  const int64_t n_out = glu ? N / 2 : N;
+#pragma omp parallel for schedule(static)
+  for (int64_t m = 0; m < M; ++m) {
+    double* z = (double*)malloc((size_t)(N + 1) * sizeof(double));
+    for (int64_t n = 0; n < N; ++n) {
+      double sum = 0.0, mag = 0.0;
+      for (int64_t k = 0; k < K; ++k) {
+        double p = (double)x[m * ldx + k] * (double)wq[n * K + k];
+        sum += p;
+        mag += fabs(p);
+      }
+      z[n] = (double)s_w[n] * sum + (bias ? (double)bias[n] : 0.0);
+      if (z_out) z_out[m * N + n] = z[n];
+      if (mag_out) mag_out[m * N + n] = fabs((double)s_w[n]) * mag;
+    }
+    for (int64_t j = 0; j < n_out; ++j) {
+      double a = z[j];
+      if (act == ORC_ACT_SWISH) a = z[j] * sigmoid_d(z[j]);
+      if (glu) {
+        a = z[j] * sigmoid_d(z[j + n_out]);
+        if (act == ORC_ACT_GLU_SWISH) a = a * sigmoid_d(a);
+      }
+      if (residual) a = (double)residual[m * ldr + j] + (double)residual_scale * a;
+      y[m * n_out + j] = a;
+    }
+    free(z);
+  }
+  return 0;
+}

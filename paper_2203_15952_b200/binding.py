@@ -20,11 +20,11 @@ AXIS_ROW, AXIS_COL, AXIS_TENSOR = 0, 1, 2
 ROUND_HALF_UP_FLOOR, ROUND_NEAREST_EVEN = 0, 1
 SCALE_ROW, SCALE_TENSOR = 0, 1
 ACT_NONE, ACT_SWISH, ACT_GLU, ACT_GLU_SWISH = 0, 1, 2, 3
-OP_QMATMUL, OP_LINEAR_FWD, OP_QMATMUL_REQUANT = 1, 2, 3
+OP_QMATMUL, OP_LINEAR_FWD, OP_QMATMUL_REQUANT, OP_LINEAR_WEIGHT_ONLY = 1, 2, 3, 4
 
 EXPORTS = ("aqt_version", "aqt_status_string", "aqt_quantize", "aqt_pack_int4", "aqt_unpack_int4", "aqt_qmatmul",
            "aqt_linear_fwd", "aqt_linear_fwd_host", "aqt_workspace_bytes", "aqt_device_status", "aqt_qmatmul_w4_noalloc",
-           "aqt_selftest_bounded_wait", "aqt_qmatmul_requant")
+           "aqt_selftest_bounded_wait", "aqt_qmatmul_requant", "aqt_linear_fwd_weight_only")
 NOALLOC_MAX_WEIGHT_BYTES = 4 << 20
 
 
@@ -124,6 +124,15 @@ def bind_linear_fwd(x, wq, s_w, bias, residual, residual_scale, bits_a, bits_w, 
                 _i64(residual.stride(0) if residual is not None else 0), ctypes.c_float(residual_scale), _i64(M), _i64(N),
                 _i64(K), int(bits_a), int(bits_w), int(a_scale_kind), int(rounding), int(act), _ptr(y), _i64(y.stride(0)),
                 _ptr(workspace), ctypes.c_size_t(workspace.numel()), _stream(stream))
+
+
+def bind_linear_fwd_weight_only(x, wq, s_w, bias, residual, residual_scale, bits_w, act, y, workspace, stream=None):
+    M, K = x.shape
+    N = wq.shape[0]
+    return bind("aqt_linear_fwd_weight_only", _ptr(x), _i64(x.stride(0)), _ptr(wq), _ptr(s_w), _ptr(bias), _ptr(residual),
+                _i64(residual.stride(0) if residual is not None else 0), ctypes.c_float(residual_scale), _i64(M), _i64(N),
+                _i64(K), int(bits_w), int(act), _ptr(y), _i64(y.stride(0)), _ptr(workspace),
+                ctypes.c_size_t(workspace.numel()), _stream(stream))
 
 
 def aqt_version() -> int:
@@ -277,6 +286,27 @@ def aqt_linear_fwd(x: torch.Tensor, wq: torch.Tensor, s_w: torch.Tensor, bias: O
         _i64(residual.stride(0) if residual is not None else 0), ctypes.c_float(residual_scale), _i64(M), _i64(N), _i64(K),
         int(bits_a), int(bits_w), int(a_scale_kind), int(rounding), int(act), _ptr(y), _i64(y.stride(0)), _ptr(workspace),
         ctypes.c_size_t(workspace.numel()), _stream(stream)))
+    return y
+
+
+def aqt_linear_fwd_weight_only(x: torch.Tensor, wq: torch.Tensor, s_w: torch.Tensor, bias: Optional[torch.Tensor] = None,
+                               residual: Optional[torch.Tensor] = None, residual_scale: float = 1.0, *, bits_w: int = 8,
+                               act: int = ACT_NONE, y: Optional[torch.Tensor] = None,
+                               workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """The weight-only layer (int8 / int4 weights, float activations): x fp32 [M, K] against the
+    codes wq [N, K] int8 or [N, K/2] uint8 packed, de-quantized by s_w after the float matmul."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.dim() == 2 and x.stride(1) == 1
+    M, K = x.shape
+    N = wq.shape[0]
+    if y is None:
+        y = torch.empty((M, _n_out(N, act)), dtype=torch.float32, device=x.device)
+    need = aqt_workspace_bytes(OP_LINEAR_WEIGHT_ONLY, M, N, K, 0, bits_w)
+    workspace = _workspace(need, workspace, x.device)
+    _check("aqt_linear_fwd_weight_only", lib().aqt_linear_fwd_weight_only(
+        _ptr(x), _i64(x.stride(0)), _ptr(wq), _ptr(s_w), _ptr(bias), _ptr(residual),
+        _i64(residual.stride(0) if residual is not None else 0), ctypes.c_float(residual_scale), _i64(M), _i64(N), _i64(K),
+        int(bits_w), int(act), _ptr(y), _i64(y.stride(0)), _ptr(workspace), ctypes.c_size_t(workspace.numel()),
+        _stream(stream)))
     return y
 
 

@@ -37,6 +37,8 @@ size_t ws_linear(int64_t M, int64_t N, int64_t K, int bits_w) {
   return round_up((size_t)M * (size_t)K, 256) + round_up((size_t)M * 4, 256) + ws_qmatmul(0, N, K, 8, bits_w);
 }
 
+size_t ws_weight_only(int64_t N, int64_t K) { return round_up((size_t)N * (size_t)K * 4, 256); }
+
 int validate_matmul_shape(int64_t M, int64_t N, int64_t K, int bits_a, int bits_w, int act, int s_x_kind) {
   if (M < 0 || N < 0 || K <= 0) return AQT_ERR_BADARG;
   if (!bits_ok(bits_a) || !bits_ok(bits_w) || !act_ok(act)) return AQT_ERR_BADARG;
@@ -136,6 +138,7 @@ size_t aqt_workspace_bytes(int op, int64_t M, int64_t N, int64_t K, int bits_a, 
   if (M < 0 || N < 0 || K < 0) return 0;
   if (op == AQT_OP_QMATMUL) return ws_qmatmul(M, N, K, bits_a, bits_w);
   if (op == AQT_OP_LINEAR_FWD) return ws_linear(M, N, K, bits_w);
+  if (op == AQT_OP_LINEAR_WEIGHT_ONLY) return ws_weight_only(N, K);
   if (op == AQT_OP_QMATMUL_REQUANT) return round_up(ws_qmatmul(M, N, K, bits_a, bits_w), 256) + requant_exchange_bytes(M, N);
   return 0;
 }
@@ -361,6 +364,53 @@ int aqt_linear_fwd_host(const float* x, int x_on_host, const void* wq, const flo
   if (rc != AQT_OK) return rc;
   if (y_on_host) AQT_RETURN_IF_CUDA(cudaMemcpyAsync(y, y_dev, (size_t)M * n_out * 4, cudaMemcpyDeviceToHost, st));
   return AQT_OK;
+}
+
+int aqt_linear_fwd_weight_only(const float* x, int64_t ldx, const void* wq, const float* s_w, const float* bias,
+                               const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K,
+                               int bits_w, int act, float* y, int64_t ldy, void* workspace, size_t workspace_bytes,
+                               void* stream) {
+  if (M < 0 || N < 0 || K <= 0 || !bits_ok(bits_w) || !act_ok(act)) return AQT_ERR_BADARG;
+  if (K % 4 != 0 || N % 4 != 0 || (is_glu(act) && N % 8 != 0)) return AQT_ERR_BADARG;
+  if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 29) || M * N >= (1ll << 40)) return AQT_ERR_UNSUPPORTED;
+  if (M == 0 || N == 0) return AQT_OK;
+  const int64_t n_out = is_glu(act) ? N / 2 : N;
+  if (x == nullptr || wq == nullptr || s_w == nullptr || y == nullptr) return AQT_ERR_BADARG;
+  if (ldx < K || ldy < n_out || (residual != nullptr && ldr < n_out)) return AQT_ERR_BADARG;
+  if (!is_aligned(x, 16) || !is_aligned(wq, 16) || !is_aligned(y, 16) || !is_aligned(s_w, 16) ||
+      (bias != nullptr && !is_aligned(bias, 16)) || (residual != nullptr && !is_aligned(residual, 16)))
+    return AQT_ERR_ALIGN;
+  if (ldx % 4 != 0 || ldy % 4 != 0 || (residual != nullptr && ldr % 4 != 0)) return AQT_ERR_ALIGN;
+  const size_t need = ws_weight_only(N, K);
+  if (workspace == nullptr || workspace_bytes < need) return AQT_ERR_WORKSPACE;
+  if (!is_aligned(workspace, 256)) return AQT_ERR_ALIGN;
+  int rc = check_device();
+  if (rc != AQT_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  // the weights converted to float (Section 4.1): the codes as binary32 integers, once per call;
+  // the channel scales stay outside the sum and are applied to the accumulators.
+  float* w_f = reinterpret_cast<float*>(workspace);
+  rc = launch_codes_to_float(wq, bits_w == 4, N * K, w_f, st);
+  if (rc != AQT_OK) return rc;
+  GemmParams p;
+  p.s_x = nullptr;
+  p.s_w = s_w;
+  p.bias = bias;
+  p.residual = residual;
+  p.acc_debug = nullptr;
+  p.ldr = ldr;
+  p.residual_scale = residual_scale;
+  p.s_x_kind = AQT_SCALE_TENSOR;
+  p.act = act;
+  p.M = (int)M;
+  p.N = (int)N;
+  p.K = (int)(4 * K);
+  p.kind = 1;
+  p.a_pitch = 4 * ldx;
+  p.n_out = (int)n_out;
+  p.tiles_m = p.tiles_n = p.k_blocks = 0;
+  p.small_acc = 0;
+  return launch_qgemm(reinterpret_cast<const int8_t*>(x), w_f, false, y, ldy, p, st);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -75,6 +75,29 @@ __global__ void __launch_bounds__(256) pack_int4_kernel(const int8_t* __restrict
   }
 }
 
+// Weight codes -> binary32 values of the same integers (exact; every code has at most 7
+// significant bits).  The float matmul of the weight-only layer reads these.  n codes, a multiple
+// of 4: dense int8, or nibble pairs if `packed`.  Four codes per thread and step.
+__global__ void __launch_bounds__(256) codes_to_float_kernel(const uint8_t* __restrict__ codes, bool packed, int64_t n,
+                                                             float* __restrict__ out) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < (n >> 2); i += stride) {
+    uint32_t w;
+    if (packed) {
+      uint32_t o1;
+      unpack_word((uint32_t)__ldg(reinterpret_cast<const uint16_t*>(codes) + i), w, o1);
+    } else {
+      w = __ldg(reinterpret_cast<const uint32_t*>(codes) + i);
+    }
+    float4 f;
+    f.x = (float)(int8_t)(w & 0xFF);
+    f.y = (float)(int8_t)((w >> 8) & 0xFF);
+    f.z = (float)(int8_t)((w >> 16) & 0xFF);
+    f.w = (float)(int8_t)(w >> 24);
+    reinterpret_cast<float4*>(out)[i] = f;
+  }
+}
+
 static unsigned flat_grid(int64_t work_items) {
   const int64_t want = ceil_div(work_items, 256);
   return (unsigned)(want < 1 ? 1 : (want > 148 * 32 ? 148 * 32 : want));
@@ -83,6 +106,12 @@ static unsigned flat_grid(int64_t work_items) {
 static int launch_unpack_int4(const uint8_t* packed, int64_t n_bytes, int8_t* q, cudaStream_t st) {
   const bool vec = is_aligned(packed, 8) && is_aligned(q, 16);
   unpack_int4_kernel<<<flat_grid(vec ? n_bytes / 8 + 8 : n_bytes), 256, 0, st>>>(packed, n_bytes, q, vec);
+  return AQT_LAUNCH_STATUS();
+}
+
+// codes: int8 [n] or packed nibbles [n / 2], 4-byte (2-byte if packed) aligned; out: float [n], 16-byte aligned; n % 4 == 0.
+static int launch_codes_to_float(const void* codes, bool packed, int64_t n, float* out, cudaStream_t st) {
+  codes_to_float_kernel<<<flat_grid(n / 4), 256, 0, st>>>(reinterpret_cast<const uint8_t*>(codes), packed, n, out);
   return AQT_LAUNCH_STATUS();
 }
 

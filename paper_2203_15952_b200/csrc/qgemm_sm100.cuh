@@ -79,7 +79,9 @@ struct GemmParams {
   float residual_scale;
   int s_x_kind;
   int act;
-  int M, N, K;
+  int M, N, K;  // K: bytes of contraction per operand row (= elements for 8-bit codes, 4 x elements for the float kind)
+  int kind = 0;       // 0: signed 8-bit codes, int32 accumulators; 1: binary32 operands used as tf32, binary32 accumulators
+  int64_t a_pitch = 0;  // bytes between rows of A; 0 = dense (K)
   int n_out;    // N, or N / 2 for the GLU forms
   int tiles_m, tiles_n, k_blocks;
   int small_acc;  // every |accumulator| < 2^22: the int -> float conversion can use the exponent trick
@@ -225,6 +227,26 @@ __device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// The float forms: A and B hold binary32 values of which the tensor core uses sign, exponent and
+// the upper ten fraction bits (tf32); products are summed into binary32 accumulators.  One
+// instruction covers K = 8 elements = 32 bytes, so operand tiles, swizzle and the descriptor
+// advance are byte-for-byte those of the 8-bit kind.
+__device__ __forceinline__ void tc_mma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_mma_tf32_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 // 32 lanes x 32 consecutive 32-bit columns: thread i of the warp receives lane (base + i).
 __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
@@ -255,6 +277,10 @@ __device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t saddr) {
 __host__ __device__ constexpr uint32_t idesc_i8(int bn, int m = kBM) {
   return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
+// The same for the float kind: D binary32, A and B tf32, both K-major.
+__host__ __device__ constexpr uint32_t idesc_tf32(int bn, int m = kBM) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
 
 // ------------------------------------------------------------------------------------------------
 // Epilogue math
@@ -282,19 +308,25 @@ __device__ __forceinline__ float sigmoid_f(float z) {
   return rcp_approx(1.0f + e);
 }
 
-// int32 accumulator -> float, round-to-nearest-even (exact below 2^24).  With SMALL the caller
-// guarantees |acc| < 2^22: adding the integer to the bit pattern of 1.5 * 2^23 and subtracting
-// that constant is exact and stays off the conversion unit.
-template <bool SMALL>
+// What a TMEM accumulator word holds and how it becomes a float (template argument ACCK):
+//   kAccInt32      int32, converted round-to-nearest-even (exact below 2^24)
+//   kAccInt32Small int32 with |acc| < 2^22 guaranteed by the caller: adding the integer to the bit
+//                  pattern of 1.5 * 2^23 and subtracting that constant is exact and stays off the
+//                  conversion unit
+//   kAccFloat      binary32 already (the float matmul of the weight-only layer)
+constexpr int kAccInt32 = 0, kAccInt32Small = 1, kAccFloat = 2;
+template <int ACCK>
 __device__ __forceinline__ float acc_to_float(uint32_t acc) {
-  if (SMALL) return __int_as_float(0x4B400000 + (int)acc) - 12582912.0f;
+  if (ACCK == kAccFloat) return __uint_as_float(acc);
+  if (ACCK == kAccInt32Small) return __int_as_float(0x4B400000 + (int)acc) - 12582912.0f;
   return __int2float_rn((int)acc);
 }
 
 // Two accumulators -> two floats (see acc_to_float); the subtraction is one packed add.
-template <bool SMALL>
+template <int ACCK>
 __device__ __forceinline__ float2 acc_to_float2(uint32_t a0, uint32_t a1) {
-  if (SMALL)
+  if (ACCK == kAccFloat) return make_float2(__uint_as_float(a0), __uint_as_float(a1));
+  if (ACCK == kAccInt32Small)
     return __fadd2_rn(make_float2(__int_as_float(0x4B400000 + (int)a0), __int_as_float(0x4B400000 + (int)a1)),
                       make_float2(-12582912.0f, -12582912.0f));
   return make_float2(__int2float_rn((int)a0), __int2float_rn((int)a1));
@@ -304,7 +336,7 @@ __device__ __forceinline__ float2 acc_to_float2(uint32_t a0, uint32_t a1) {
 // biases sit at `sw_smem` / `b_smem` (shared-memory byte addresses, 16-byte aligned).  The
 // arithmetic runs on the packed two-lane fp32 instructions of this architecture (each lane an
 // ordinary round-to-nearest IEEE operation), which halves the issue slots it takes.
-template <bool SMALL>
+template <int ACCK>
 __device__ __forceinline__ void dequant32(const uint32_t (&acc)[32], float sx, uint32_t sw_smem, uint32_t b_smem, float (&z)[32]) {
   const float2 sx2 = make_float2(sx, sx);
 #pragma unroll
@@ -312,8 +344,8 @@ __device__ __forceinline__ void dequant32(const uint32_t (&acc)[32], float sx, u
     float w0, w1, w2, w3, b0, b1, b2, b3;
     asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(w0), "=f"(w1), "=f"(w2), "=f"(w3) : "r"(sw_smem + 16 * j));
     asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(b0), "=f"(b1), "=f"(b2), "=f"(b3) : "r"(b_smem + 16 * j));
-    const float2 z01 = __ffma2_rn(__fmul2_rn(acc_to_float2<SMALL>(acc[4 * j + 0], acc[4 * j + 1]), sx2), make_float2(w0, w1), make_float2(b0, b1));
-    const float2 z23 = __ffma2_rn(__fmul2_rn(acc_to_float2<SMALL>(acc[4 * j + 2], acc[4 * j + 3]), sx2), make_float2(w2, w3), make_float2(b2, b3));
+    const float2 z01 = __ffma2_rn(__fmul2_rn(acc_to_float2<ACCK>(acc[4 * j + 0], acc[4 * j + 1]), sx2), make_float2(w0, w1), make_float2(b0, b1));
+    const float2 z23 = __ffma2_rn(__fmul2_rn(acc_to_float2<ACCK>(acc[4 * j + 2], acc[4 * j + 3]), sx2), make_float2(w2, w3), make_float2(b2, b3));
     z[4 * j + 0] = z01.x;
     z[4 * j + 1] = z01.y;
     z[4 * j + 2] = z23.x;
@@ -347,17 +379,17 @@ __device__ __forceinline__ float4 ld4_guard(const float* base, int n, int limit)
 }
 
 // The same with scales and biases read from global memory (warp-uniform addresses, served by L1).
-template <bool SMALL>
+template <int ACCK>
 __device__ __forceinline__ void dequant32_gmem(const uint32_t (&acc)[32], float sx, const float* s_w, const float* bias, int n0,
                                                int limit, float (&z)[32]) {
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     const float4 w = ld4_guard(s_w, n0 + 4 * j, limit);
     const float4 b = ld4_guard(bias, n0 + 4 * j, limit);
-    z[4 * j + 0] = __fmaf_rn(__fmul_rn(acc_to_float<SMALL>(acc[4 * j + 0]), sx), w.x, b.x);
-    z[4 * j + 1] = __fmaf_rn(__fmul_rn(acc_to_float<SMALL>(acc[4 * j + 1]), sx), w.y, b.y);
-    z[4 * j + 2] = __fmaf_rn(__fmul_rn(acc_to_float<SMALL>(acc[4 * j + 2]), sx), w.z, b.z);
-    z[4 * j + 3] = __fmaf_rn(__fmul_rn(acc_to_float<SMALL>(acc[4 * j + 3]), sx), w.w, b.w);
+    z[4 * j + 0] = __fmaf_rn(__fmul_rn(acc_to_float<ACCK>(acc[4 * j + 0]), sx), w.x, b.x);
+    z[4 * j + 1] = __fmaf_rn(__fmul_rn(acc_to_float<ACCK>(acc[4 * j + 1]), sx), w.y, b.y);
+    z[4 * j + 2] = __fmaf_rn(__fmul_rn(acc_to_float<ACCK>(acc[4 * j + 2]), sx), w.z, b.z);
+    z[4 * j + 3] = __fmaf_rn(__fmul_rn(acc_to_float<ACCK>(acc[4 * j + 3]), sx), w.w, b.w);
   }
 }
 
@@ -389,7 +421,7 @@ __device__ __forceinline__ bool tile_at(const GemmParams& p, int i, int& tm, int
   return tile < p.tiles_m * p.tiles_n;
 }
 
-template <int BN, int STAGES, int EW, bool WS, bool BPACK, bool SMALL, bool DEBUG, bool CTA2 = false>
+template <int BN, int STAGES, int EW, bool WS, bool BPACK, int ACCK, bool DEBUG, bool CTA2 = false>
 __global__ void __launch_bounds__(32 * (2 + EW), 1)
 qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                 const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_r, const GemmParams p) {
@@ -398,6 +430,8 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   constexpr int SBUFS = Cfg::kStageBufs;
   constexpr int TILE_M = CTA2 ? 2 * kBM : kBM;  // rows of a tile (of the pair's tile)
   static_assert(!BPACK || WS, "packed weights are unpacked into the resident slab");
+  constexpr bool TF32 = (ACCK == kAccFloat);  // float operands: no activation scale, accumulators are binary32
+  static_assert(!(TF32 && (BPACK || DEBUG)), "the float kind reads expanded weights and has no integer accumulators to dump");
   const uint32_t pair_rank = CTA2 ? cluster_ctarank() : 0u;  // 0 = leader: issues the MMAs, owns the barriers the pair shares
   const int row_in_tile = (int)pair_rank * kBM;               // this CTA's first row inside the tile
 
@@ -536,7 +570,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && pair_rank == 0) {
-      constexpr uint32_t idesc = idesc_i8(BN, TILE_M);
+      constexpr uint32_t idesc = TF32 ? idesc_tf32(BN, TILE_M) : idesc_i8(BN, TILE_M);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       if (WS) ok = mbar_wait(smem_u32(BPACK ? &b_ready_bar : &b_loaded_bar), 0, &abort_flag, t_start);
@@ -556,8 +590,14 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 #pragma unroll
           for (int kk = 0; kk < kBK / kMmaK; ++kk) {
             // advancing K inside the 128-byte swizzle row: +32 bytes = +2 in the 16-byte address field
-            if (CTA2) tc_mma_i8_pair(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
-            else tc_mma_i8(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+            const uint32_t accumulate = (kb | kk) != 0 ? 1u : 0u;
+            if (TF32) {
+              if (CTA2) tc_mma_tf32_pair(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, accumulate);
+              else tc_mma_tf32(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, accumulate);
+            } else {
+              if (CTA2) tc_mma_i8_pair(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, accumulate);
+              else tc_mma_i8(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, accumulate);
+            }
           }
           // stage reusable (in both CTAs of a pair) once these MMAs have read it
           if (CTA2) tc_commit_pair(smem_u32(&empty_bar[s]));
@@ -663,7 +703,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           }
         }
       }
-      const float sx = (p.s_x_kind == AQT_SCALE_ROW) ? (row_ok ? __ldg(p.s_x + m) : 0.0f) : __ldg(p.s_x);
+      const float sx = TF32 ? 1.0f : ((p.s_x_kind == AQT_SCALE_ROW) ? (row_ok ? __ldg(p.s_x + m) : 0.0f) : __ldg(p.s_x));
       __syncwarp();
 
       if (!mbar_wait(smem_u32(&tmem_full_bar[buf]), aph, &abort_flag, t_start)) break;
@@ -699,8 +739,8 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 if (n0 + j < p.N) p.acc_debug[(int64_t)m * p.N + n0 + j] = (int32_t)acc[j];
             }
           }
-          if (Cfg::kScaleSlab) dequant32<SMALL>(acc, sx, c_sw, c_bias, a);
-          else dequant32_gmem<SMALL>(acc, sx, p.s_w, p.bias, tn * BN + col, p.N, a);
+          if (Cfg::kScaleSlab) dequant32<ACCK>(acc, sx, c_sw, c_bias, a);
+          else dequant32_gmem<ACCK>(acc, sx, p.s_w, p.bias, tn * BN + col, p.N, a);
           if (p.act == AQT_ACT_SWISH) swish32(a);
         } else {
           // gates first: g = sigmoid(z_gate); then the values are scaled by it
@@ -715,8 +755,8 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 if (ng + j < p.N) p.acc_debug[(int64_t)m * p.N + ng + j] = (int32_t)acc[j];
             }
           }
-          if (Cfg::kScaleSlab) dequant32<SMALL>(acc, sx, c_sw + slab_gate_off, c_bias + slab_gate_off, g);
-          else dequant32_gmem<SMALL>(acc, sx, p.s_w, p.bias, p.N / 2 + oc, p.N, g);
+          if (Cfg::kScaleSlab) dequant32<ACCK>(acc, sx, c_sw + slab_gate_off, c_bias + slab_gate_off, g);
+          else dequant32_gmem<ACCK>(acc, sx, p.s_w, p.bias, p.N / 2 + oc, p.N, g);
 #pragma unroll
           for (int j = 0; j < 32; ++j) g[j] = sigmoid_f(g[j]);
           tmem_ld_32x32(lane_addr + col, acc);
@@ -736,8 +776,8 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 if (oc + j < p.N / 2) p.acc_debug[(int64_t)m * p.N + oc + j] = (int32_t)acc[j];
             }
           }
-          if (Cfg::kScaleSlab) dequant32<SMALL>(acc, sx, c_sw, c_bias, a);
-          else dequant32_gmem<SMALL>(acc, sx, p.s_w, p.bias, oc, p.N / 2, a);
+          if (Cfg::kScaleSlab) dequant32<ACCK>(acc, sx, c_sw, c_bias, a);
+          else dequant32_gmem<ACCK>(acc, sx, p.s_w, p.bias, oc, p.N / 2, a);
 #pragma unroll
           for (int j = 0; j < 32; ++j) a[j] = a[j] * g[j];
           if (p.act == AQT_ACT_GLU_SWISH) swish32(a);
@@ -927,7 +967,7 @@ static int pick_bn(int64_t M, int64_t N, bool glu, int sms) {
 }
 
 // b: weight codes as the kernel reads them -- int8 [N, K], or (BPACK) packed nibbles [N, K/2].
-template <int BN, int STAGES, int EW, bool WS, bool BPACK, bool SMALL, bool DEBUG, bool CTA2 = false>
+template <int BN, int STAGES, int EW, bool WS, bool BPACK, int ACCK, bool DEBUG, bool CTA2 = false>
 static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t ldy, const GemmParams& p0, cudaStream_t st) {
   using Cfg = GemmCfg<BN, STAGES, EW, WS, CTA2>;
   GemmParams p = p0;
@@ -942,7 +982,8 @@ static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t l
     if (WS && (p.k_blocks > kWsMaxKBlocks || p.tiles_n > sms)) return AQT_ERR_UNSUPPORTED;
   }
   CUtensorMap tm_a, tm_b, tm_y, tm_r;
-  int rc = make_map_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, a, (uint64_t)p.M, (uint64_t)p.K, (uint64_t)p.K, kBM, kBK);
+  int rc = make_map_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, a, (uint64_t)p.M, (uint64_t)p.K,
+                       (uint64_t)(p.a_pitch != 0 ? p.a_pitch : p.K), kBM, kBK);
   if (rc != AQT_OK) return rc;
   if (BPACK) {
     rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, b, (uint64_t)p.N, (uint64_t)p.K / 2, (uint64_t)p.K / 2, BN / 2, 64, 0);
@@ -960,7 +1001,7 @@ static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t l
   } else {
     tm_r = tm_y;  // never dereferenced
   }
-  auto kernel = qgemm_i8_kernel<BN, STAGES, EW, WS, BPACK, SMALL, DEBUG, CTA2>;
+  auto kernel = qgemm_i8_kernel<BN, STAGES, EW, WS, BPACK, ACCK, DEBUG, CTA2>;
   static bool attr_set = false;
   if (!attr_set) {
     AQT_RETURN_IF_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
@@ -994,9 +1035,15 @@ static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t l
 
 template <int BN, int STAGES, int EW, bool WS, bool BPACK, bool CTA2 = false>
 static int launch_qgemm_cfg(const int8_t* a, const void* b, float* y, int64_t ldy, const GemmParams& p, cudaStream_t st) {
-  if (p.acc_debug != nullptr) return launch_qgemm_inst<BN, STAGES, EW, WS, BPACK, false, true, CTA2>(a, b, y, ldy, p, st);
-  if (p.small_acc) return launch_qgemm_inst<BN, STAGES, EW, WS, BPACK, true, false, CTA2>(a, b, y, ldy, p, st);
-  return launch_qgemm_inst<BN, STAGES, EW, WS, BPACK, false, false, CTA2>(a, b, y, ldy, p, st);
+  if (p.kind == 1) {
+    if constexpr (!BPACK) {
+      if (p.acc_debug == nullptr) return launch_qgemm_inst<BN, STAGES, EW, WS, false, kAccFloat, false, CTA2>(a, b, y, ldy, p, st);
+    }
+    return AQT_ERR_UNSUPPORTED;
+  }
+  if (p.acc_debug != nullptr) return launch_qgemm_inst<BN, STAGES, EW, WS, BPACK, kAccInt32, true, CTA2>(a, b, y, ldy, p, st);
+  if (p.small_acc) return launch_qgemm_inst<BN, STAGES, EW, WS, BPACK, kAccInt32Small, false, CTA2>(a, b, y, ldy, p, st);
+  return launch_qgemm_inst<BN, STAGES, EW, WS, BPACK, kAccInt32, false, CTA2>(a, b, y, ldy, p, st);
 }
 
 // True if the weight-stationary kernel takes this shape (and can therefore unpack 4-bit weights itself).
