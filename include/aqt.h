@@ -66,7 +66,12 @@ extern "C" {
 #define AQT_OP_QMATMUL 1
 #define AQT_OP_LINEAR_FWD 2
 #define AQT_OP_QMATMUL_REQUANT 3
-#define AQT_OP_LINEAR_WEIGHT_ONLY 4
+#define AQT_OP_LINEAR_WEIGHT_ONLY 4    /* precision AQT_FLOAT_TF32   */
+#define AQT_OP_LINEAR_WEIGHT_ONLY_X2 5 /* precision AQT_FLOAT_TF32X2 */
+
+/* how float activations enter the tensor-core float matmul of the weight-only layer */
+#define AQT_FLOAT_TF32 0   /* one term: the upper ten fraction bits of each activation            */
+#define AQT_FLOAT_TF32X2 1 /* two terms x = hi + lo: about twenty-one significant bits, twice the work */
 
 int aqt_version(void);
 const char* aqt_status_string(int status);
@@ -193,17 +198,22 @@ int aqt_linear_fwd_host(const float* x, int x_on_host, const void* wq, const flo
  * therefore within 2^-10 * s_w[n] * sum_k |x[m][k] * wq[n][k]| (plus binary32 summation error) of
  * the exact value of the formula, and equals it bit for bit when every x is a tf32 value and no
  * partial sum needs more than 24 bits.
+ * precision AQT_FLOAT_TF32: as just described.  AQT_FLOAT_TF32X2: every activation is split
+ *           exactly into hi (its tf32 part) + lo, and one matmul over [hi | lo] against the
+ *           weights repeated sums both terms: the operand error drops from 2^-10 to 2^-20 of
+ *           the terms' magnitude for twice the tensor-core work and one more pass over x.
  * x         fp32 [M, K], row pitch ldx elements.
  * wq, s_w, bias, residual, ldr, residual_scale, act, y, ldy: as for aqt_qmatmul.
- * workspace at least aqt_workspace_bytes(AQT_OP_LINEAR_WEIGHT_ONLY, M, N, K, 0, bits_w) bytes,
- *           256-byte aligned: the weight codes as floats (4 * N * K bytes), rewritten every call.
+ * workspace at least aqt_workspace_bytes(AQT_OP_LINEAR_WEIGHT_ONLY or .._X2, M, N, K, 0, bits_w)
+ *           bytes, 256-byte aligned: the weight codes as floats (4 * N * K bytes; X2: 8 * N * K
+ *           and the split activations, 8 * M * K), rewritten every call.
  * Limits: K % 4 == 0, ldx % 4 == 0, N % 4 == 0 (N % 8 == 0 for GLU), ldy % 4 == 0, ldr % 4 == 0;
  * x, wq, y, residual, s_w, bias 16-byte aligned.  M == 0 or N == 0 is a no-op.
  */
 int aqt_linear_fwd_weight_only(const float* x, int64_t ldx, const void* wq, const float* s_w, const float* bias,
                                const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K,
-                               int bits_w, int act, float* y, int64_t ldy, void* workspace, size_t workspace_bytes,
-                               void* stream);
+                               int bits_w, int precision, int act, float* y, int64_t ldy, void* workspace,
+                               size_t workspace_bytes, void* stream);
 
 /*
  * aqt_qmatmul_w4_noalloc -- aqt_qmatmul for int8 activations and 4-bit weights that needs no

@@ -20,7 +20,8 @@ AXIS_ROW, AXIS_COL, AXIS_TENSOR = 0, 1, 2
 ROUND_HALF_UP_FLOOR, ROUND_NEAREST_EVEN = 0, 1
 SCALE_ROW, SCALE_TENSOR = 0, 1
 ACT_NONE, ACT_SWISH, ACT_GLU, ACT_GLU_SWISH = 0, 1, 2, 3
-OP_QMATMUL, OP_LINEAR_FWD, OP_QMATMUL_REQUANT, OP_LINEAR_WEIGHT_ONLY = 1, 2, 3, 4
+OP_QMATMUL, OP_LINEAR_FWD, OP_QMATMUL_REQUANT, OP_LINEAR_WEIGHT_ONLY, OP_LINEAR_WEIGHT_ONLY_X2 = 1, 2, 3, 4, 5
+FLOAT_TF32, FLOAT_TF32X2 = 0, 1
 
 EXPORTS = ("aqt_version", "aqt_status_string", "aqt_quantize", "aqt_pack_int4", "aqt_unpack_int4", "aqt_qmatmul",
            "aqt_linear_fwd", "aqt_linear_fwd_host", "aqt_workspace_bytes", "aqt_device_status", "aqt_qmatmul_w4_noalloc",
@@ -126,12 +127,13 @@ def bind_linear_fwd(x, wq, s_w, bias, residual, residual_scale, bits_a, bits_w, 
                 _ptr(workspace), ctypes.c_size_t(workspace.numel()), _stream(stream))
 
 
-def bind_linear_fwd_weight_only(x, wq, s_w, bias, residual, residual_scale, bits_w, act, y, workspace, stream=None):
+def bind_linear_fwd_weight_only(x, wq, s_w, bias, residual, residual_scale, bits_w, act, y, workspace, stream=None,
+                                precision=FLOAT_TF32):
     M, K = x.shape
     N = wq.shape[0]
     return bind("aqt_linear_fwd_weight_only", _ptr(x), _i64(x.stride(0)), _ptr(wq), _ptr(s_w), _ptr(bias), _ptr(residual),
                 _i64(residual.stride(0) if residual is not None else 0), ctypes.c_float(residual_scale), _i64(M), _i64(N),
-                _i64(K), int(bits_w), int(act), _ptr(y), _i64(y.stride(0)), _ptr(workspace),
+                _i64(K), int(bits_w), int(precision), int(act), _ptr(y), _i64(y.stride(0)), _ptr(workspace),
                 ctypes.c_size_t(workspace.numel()), _stream(stream))
 
 
@@ -291,7 +293,7 @@ def aqt_linear_fwd(x: torch.Tensor, wq: torch.Tensor, s_w: torch.Tensor, bias: O
 
 def aqt_linear_fwd_weight_only(x: torch.Tensor, wq: torch.Tensor, s_w: torch.Tensor, bias: Optional[torch.Tensor] = None,
                                residual: Optional[torch.Tensor] = None, residual_scale: float = 1.0, *, bits_w: int = 8,
-                               act: int = ACT_NONE, y: Optional[torch.Tensor] = None,
+                               precision: int = FLOAT_TF32, act: int = ACT_NONE, y: Optional[torch.Tensor] = None,
                                workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
     """The weight-only layer (int8 / int4 weights, float activations): x fp32 [M, K] against the
     codes wq [N, K] int8 or [N, K/2] uint8 packed, de-quantized by s_w after the float matmul."""
@@ -300,12 +302,12 @@ def aqt_linear_fwd_weight_only(x: torch.Tensor, wq: torch.Tensor, s_w: torch.Ten
     N = wq.shape[0]
     if y is None:
         y = torch.empty((M, _n_out(N, act)), dtype=torch.float32, device=x.device)
-    need = aqt_workspace_bytes(OP_LINEAR_WEIGHT_ONLY, M, N, K, 0, bits_w)
+    need = aqt_workspace_bytes(OP_LINEAR_WEIGHT_ONLY_X2 if precision == FLOAT_TF32X2 else OP_LINEAR_WEIGHT_ONLY, M, N, K, 0, bits_w)
     workspace = _workspace(need, workspace, x.device)
     _check("aqt_linear_fwd_weight_only", lib().aqt_linear_fwd_weight_only(
         _ptr(x), _i64(x.stride(0)), _ptr(wq), _ptr(s_w), _ptr(bias), _ptr(residual),
         _i64(residual.stride(0) if residual is not None else 0), ctypes.c_float(residual_scale), _i64(M), _i64(N), _i64(K),
-        int(bits_w), int(act), _ptr(y), _i64(y.stride(0)), _ptr(workspace), ctypes.c_size_t(workspace.numel()),
+        int(bits_w), int(precision), int(act), _ptr(y), _i64(y.stride(0)), _ptr(workspace), ctypes.c_size_t(workspace.numel()),
         _stream(stream)))
     return y
 

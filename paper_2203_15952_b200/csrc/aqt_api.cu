@@ -37,7 +37,11 @@ size_t ws_linear(int64_t M, int64_t N, int64_t K, int bits_w) {
   return round_up((size_t)M * (size_t)K, 256) + round_up((size_t)M * 4, 256) + ws_qmatmul(0, N, K, 8, bits_w);
 }
 
-size_t ws_weight_only(int64_t N, int64_t K) { return round_up((size_t)N * (size_t)K * 4, 256); }
+// one-term form: the weights as floats; two-term form: the weights twice and the split activations
+size_t ws_weight_only(int64_t M, int64_t N, int64_t K, int precision) {
+  if (precision == AQT_FLOAT_TF32X2) return round_up((size_t)N * (size_t)K * 8, 256) + round_up((size_t)M * (size_t)K * 8, 256);
+  return round_up((size_t)N * (size_t)K * 4, 256);
+}
 
 int validate_matmul_shape(int64_t M, int64_t N, int64_t K, int bits_a, int bits_w, int act, int s_x_kind) {
   if (M < 0 || N < 0 || K <= 0) return AQT_ERR_BADARG;
@@ -138,7 +142,8 @@ size_t aqt_workspace_bytes(int op, int64_t M, int64_t N, int64_t K, int bits_a, 
   if (M < 0 || N < 0 || K < 0) return 0;
   if (op == AQT_OP_QMATMUL) return ws_qmatmul(M, N, K, bits_a, bits_w);
   if (op == AQT_OP_LINEAR_FWD) return ws_linear(M, N, K, bits_w);
-  if (op == AQT_OP_LINEAR_WEIGHT_ONLY) return ws_weight_only(N, K);
+  if (op == AQT_OP_LINEAR_WEIGHT_ONLY) return ws_weight_only(0, N, K, AQT_FLOAT_TF32);
+  if (op == AQT_OP_LINEAR_WEIGHT_ONLY_X2) return ws_weight_only(M, N, K, AQT_FLOAT_TF32X2);
   if (op == AQT_OP_QMATMUL_REQUANT) return round_up(ws_qmatmul(M, N, K, bits_a, bits_w), 256) + requant_exchange_bytes(M, N);
   return 0;
 }
@@ -368,11 +373,12 @@ int aqt_linear_fwd_host(const float* x, int x_on_host, const void* wq, const flo
 
 int aqt_linear_fwd_weight_only(const float* x, int64_t ldx, const void* wq, const float* s_w, const float* bias,
                                const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K,
-                               int bits_w, int act, float* y, int64_t ldy, void* workspace, size_t workspace_bytes,
-                               void* stream) {
+                               int bits_w, int precision, int act, float* y, int64_t ldy, void* workspace,
+                               size_t workspace_bytes, void* stream) {
   if (M < 0 || N < 0 || K <= 0 || !bits_ok(bits_w) || !act_ok(act)) return AQT_ERR_BADARG;
+  if (precision != AQT_FLOAT_TF32 && precision != AQT_FLOAT_TF32X2) return AQT_ERR_BADARG;
   if (K % 4 != 0 || N % 4 != 0 || (is_glu(act) && N % 8 != 0)) return AQT_ERR_BADARG;
-  if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 29) || M * N >= (1ll << 40)) return AQT_ERR_UNSUPPORTED;
+  if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 28) || M * N >= (1ll << 40)) return AQT_ERR_UNSUPPORTED;
   if (M == 0 || N == 0) return AQT_OK;
   const int64_t n_out = is_glu(act) ? N / 2 : N;
   if (x == nullptr || wq == nullptr || s_w == nullptr || y == nullptr) return AQT_ERR_BADARG;
@@ -381,7 +387,7 @@ int aqt_linear_fwd_weight_only(const float* x, int64_t ldx, const void* wq, cons
       (bias != nullptr && !is_aligned(bias, 16)) || (residual != nullptr && !is_aligned(residual, 16)))
     return AQT_ERR_ALIGN;
   if (ldx % 4 != 0 || ldy % 4 != 0 || (residual != nullptr && ldr % 4 != 0)) return AQT_ERR_ALIGN;
-  const size_t need = ws_weight_only(N, K);
+  const size_t need = ws_weight_only(M, N, K, precision);
   if (workspace == nullptr || workspace_bytes < need) return AQT_ERR_WORKSPACE;
   if (!is_aligned(workspace, 256)) return AQT_ERR_ALIGN;
   int rc = check_device();
@@ -390,8 +396,22 @@ int aqt_linear_fwd_weight_only(const float* x, int64_t ldx, const void* wq, cons
   // the weights converted to float (Section 4.1): the codes as binary32 integers, once per call;
   // the channel scales stay outside the sum and are applied to the accumulators.
   float* w_f = reinterpret_cast<float*>(workspace);
-  rc = launch_codes_to_float(wq, bits_w == 4, N * K, w_f, st);
-  if (rc != AQT_OK) return rc;
+  const float* a_f = x;
+  int64_t k_mm = K, a_pitch = 4 * ldx;
+  if (precision == AQT_FLOAT_TF32X2) {
+    // x = hi + lo with hi a tf32 value: one matmul over [hi | lo] against [w | w]
+    float* x2 = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace) + round_up((size_t)N * (size_t)K * 8, 256));
+    rc = launch_codes_to_float_twice(wq, bits_w == 4, N, K, w_f, st);
+    if (rc != AQT_OK) return rc;
+    rc = launch_split_hi_lo(x, ldx, M, K, x2, st);
+    if (rc != AQT_OK) return rc;
+    a_f = x2;
+    k_mm = 2 * K;
+    a_pitch = 8 * K;
+  } else {
+    rc = launch_codes_to_float(wq, bits_w == 4, N * K, w_f, st);
+    if (rc != AQT_OK) return rc;
+  }
   GemmParams p;
   p.s_x = nullptr;
   p.s_w = s_w;
@@ -404,13 +424,13 @@ int aqt_linear_fwd_weight_only(const float* x, int64_t ldx, const void* wq, cons
   p.act = act;
   p.M = (int)M;
   p.N = (int)N;
-  p.K = (int)(4 * K);
+  p.K = (int)(4 * k_mm);
   p.kind = 1;
-  p.a_pitch = 4 * ldx;
+  p.a_pitch = a_pitch;
   p.n_out = (int)n_out;
   p.tiles_m = p.tiles_n = p.k_blocks = 0;
   p.small_acc = 0;
-  return launch_qgemm(reinterpret_cast<const int8_t*>(x), w_f, false, y, ldy, p, st);
+  return launch_qgemm(reinterpret_cast<const int8_t*>(a_f), w_f, false, y, ldy, p, st);
 }
 
 // ------------------------------------------------------------------------------------------------

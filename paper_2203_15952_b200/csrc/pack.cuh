@@ -98,6 +98,57 @@ __global__ void __launch_bounds__(256) codes_to_float_kernel(const uint8_t* __re
   }
 }
 
+// Two-term split of binary32 activations for the float matmul: hi = x with its lower thirteen
+// fraction bits cleared (a tf32 value), lo = x - hi (exact).  Row m of the output holds
+// [hi(x[m][0..K)) | lo(x[m][0..K))], so that one matmul over 2K against the weights repeated twice
+// sums x . w with about twenty-one significant bits per activation.  K % 4 == 0, ldx % 4 == 0.
+__global__ void __launch_bounds__(256) split_hi_lo_kernel(const float* __restrict__ x, int64_t ldx, int64_t M, int64_t K,
+                                                          float* __restrict__ out) {
+  const int64_t k4 = K >> 2, total = M * k4;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+    const int64_t m = i / k4, c = i - m * k4;
+    const float4 v = __ldg(reinterpret_cast<const float4*>(x + m * ldx) + c);
+    float4 hi, lo;
+    hi.x = __uint_as_float(__float_as_uint(v.x) & 0xFFFFE000u);
+    hi.y = __uint_as_float(__float_as_uint(v.y) & 0xFFFFE000u);
+    hi.z = __uint_as_float(__float_as_uint(v.z) & 0xFFFFE000u);
+    hi.w = __uint_as_float(__float_as_uint(v.w) & 0xFFFFE000u);
+    lo.x = __fsub_rn(v.x, hi.x);
+    lo.y = __fsub_rn(v.y, hi.y);
+    lo.z = __fsub_rn(v.z, hi.z);
+    lo.w = __fsub_rn(v.w, hi.w);
+    float4* row = reinterpret_cast<float4*>(out + m * 2 * K);
+    row[c] = hi;
+    row[k4 + c] = lo;
+  }
+}
+
+// The weight codes as floats, each row written twice: out [rows, 2K] = [w | w].
+__global__ void __launch_bounds__(256) codes_to_float_twice_kernel(const uint8_t* __restrict__ codes, bool packed, int64_t rows,
+                                                                   int64_t K, float* __restrict__ out) {
+  const int64_t k4 = K >> 2, total = rows * k4;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+    const int64_t r = i / k4, c = i - r * k4;
+    uint32_t w;
+    if (packed) {
+      uint32_t o1;
+      unpack_word((uint32_t)__ldg(reinterpret_cast<const uint16_t*>(codes) + i), w, o1);
+    } else {
+      w = __ldg(reinterpret_cast<const uint32_t*>(codes) + i);
+    }
+    float4 f;
+    f.x = (float)(int8_t)(w & 0xFF);
+    f.y = (float)(int8_t)((w >> 8) & 0xFF);
+    f.z = (float)(int8_t)((w >> 16) & 0xFF);
+    f.w = (float)(int8_t)(w >> 24);
+    float4* row = reinterpret_cast<float4*>(out + r * 2 * K);
+    row[c] = f;
+    row[k4 + c] = f;
+  }
+}
+
 static unsigned flat_grid(int64_t work_items) {
   const int64_t want = ceil_div(work_items, 256);
   return (unsigned)(want < 1 ? 1 : (want > 148 * 32 ? 148 * 32 : want));
@@ -112,6 +163,15 @@ static int launch_unpack_int4(const uint8_t* packed, int64_t n_bytes, int8_t* q,
 // codes: int8 [n] or packed nibbles [n / 2], 4-byte (2-byte if packed) aligned; out: float [n], 16-byte aligned; n % 4 == 0.
 static int launch_codes_to_float(const void* codes, bool packed, int64_t n, float* out, cudaStream_t st) {
   codes_to_float_kernel<<<flat_grid(n / 4), 256, 0, st>>>(reinterpret_cast<const uint8_t*>(codes), packed, n, out);
+  return AQT_LAUNCH_STATUS();
+}
+
+static int launch_split_hi_lo(const float* x, int64_t ldx, int64_t M, int64_t K, float* out, cudaStream_t st) {
+  split_hi_lo_kernel<<<flat_grid(M * K / 4), 256, 0, st>>>(x, ldx, M, K, out);
+  return AQT_LAUNCH_STATUS();
+}
+static int launch_codes_to_float_twice(const void* codes, bool packed, int64_t rows, int64_t K, float* out, cudaStream_t st) {
+  codes_to_float_twice_kernel<<<flat_grid(rows * K / 4), 256, 0, st>>>(reinterpret_cast<const uint8_t*>(codes), packed, rows, K, out);
   return AQT_LAUNCH_STATUS();
 }
 

@@ -1069,12 +1069,21 @@ static int launch_qgemm(const int8_t* a, const void* b, bool b_packed, float* y,
   // than the extra ring stages gain (measured at M = 12 800 .. 25 600).
   const int sms_ = sm_count() > 0 ? sm_count() : 148;
   bool deep_k = p.K >= 2048 && !glu && ceil_div(p.M, kBM) * ceil_div(p.N, 256) >= 4 * sms_;
+  // Float kind: a k-block takes as many tensor-core clocks as an 8-bit one but holds a quarter of
+  // the elements, so every shape is "deep" in bytes and the epilogue is a small part of a tile
+  // unless it evaluates an activation (measured: the four-warp epilogue wins at 12 800 x 512 x
+  // 2048 and 65 536 x 1024 x 4096 without activation, loses by 20-40 % with Swish).
+  const bool f32 = p.kind == 1;
+  if (f32) deep_k = p.act == AQT_ACT_NONE && p.K >= 8192;
   static const char* deep_env = getenv("AQT_DEEP");  // tuning aid: 0 / 1 overrides the deep-K choice
   if (deep_env != nullptr && !glu) deep_k = atoi(deep_env) != 0;
   static const char* no_pairs = getenv("AQT_NO_PAIRS");  // tuning aid: one CTA per tile
-  // Pairs pay off only for deep K and many tiles per pair (measured: +4 % at 65 536 x 1024 x 4096,
-  // slower than single CTAs at M = 12 800 .. 25 600); everything else takes one CTA per tile.
-  const bool pairs_ok = deep_k;
+  // Pairs pay off only for deep K and at least two full rounds of pair tiles (measured: +4 % at
+  // 65 536 x 1024 x 4096 with the deep configuration, +9 % at 25 600 x 512 x 2048 with the
+  // eight-warp epilogue, no gain at M = 12 800 or at K = 1024); everything else takes one CTA per tile.
+  const bool two_rounds_of_pairs = !glu && ceil_div(p.M, 2 * kBM) * ceil_div(p.N, 256) >= 2 * (sms_ / 2);
+  // (float kind, measured: pairs win 6-10 % at M >= 25 600, lose 10 % at 12 800 x 2048 x 512)
+  const bool pairs_ok = f32 ? (two_rounds_of_pairs && p.M >= 2 * kBM * (sms_ / 2)) : (deep_k || (p.K >= 2048 && two_rounds_of_pairs));
   if (no_pairs == nullptr && (pairs_ok || getenv("AQT_FORCE_PAIRS") != nullptr) && p.M > kBM) {
     // CTA pairs on 256-row tiles; width by the number of rounds over the pairs
     const int pairs = (sm_count() > 0 ? sm_count() : 148) / 2;
@@ -1088,6 +1097,7 @@ static int launch_qgemm(const int8_t* a, const void* b, bool b_packed, float* y,
     return deep_k ? launch_qgemm_cfg<128, 8, 4, false, false, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 6, 8, false, false, true>(a, b, y, ldy, p, st);
   }
   int bn = pick_bn(p.M, p.N, glu, sm_count() > 0 ? sm_count() : 148);
+  if (f32 && p.N >= 256) bn = 256;  // operand bytes per output are four times those of the 8-bit kind: the widest tile always wins
   // tuning aid: AQT_BN=64|128|256 in the environment overrides the tile-width heuristic
   static const char* force = getenv("AQT_BN");
   if (force != nullptr) {

@@ -5,6 +5,7 @@
     python -m paper_2203_15952_b200.shape_bench requant M N K [--act 0|1] [--bits-w 4|8] [--bits 4|8] [--with-y] [--residual]
     python -m paper_2203_15952_b200.shape_bench quantize M K [--bits 4|8]
     python -m paper_2203_15952_b200.shape_bench linear M N K [--act ..] [--bits-w ..] [--bits 4|8] [--per-tensor]
+    python -m paper_2203_15952_b200.shape_bench wonly M N K [--act ..] [--bits-w 4|8] [--residual] [--x2]
 
 Inputs are random codes / normals drawn on the GPU (seeded); several buffer sets are rotated so
 that consecutive launches do not find their inputs in L2.  With --sustain the call is repeated for
@@ -89,7 +90,7 @@ def _sustain(calls, seconds):
 
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("op", choices=["qmatmul", "requant", "quantize", "linear"])
+    ap.add_argument("op", choices=["qmatmul", "requant", "quantize", "linear", "wonly"])
     ap.add_argument("dims", type=int, nargs="+")
     ap.add_argument("--act", type=int, default=0)
     ap.add_argument("--bits-w", type=int, default=8)
@@ -97,6 +98,7 @@ def main(argv=None):
     ap.add_argument("--residual", action="store_true")
     ap.add_argument("--with-y", action="store_true", help="requant: also write the fp32 output")
     ap.add_argument("--per-tensor", action="store_true", help="linear: one activation scale for the whole tensor")
+    ap.add_argument("--x2", action="store_true", help="wonly: two-term (hi + lo) form of the float activations")
     ap.add_argument("--iters", type=int, default=30)
     ap.add_argument("--sets", type=int, default=4)
     ap.add_argument("--sustain", type=float, default=0.0)
@@ -172,6 +174,30 @@ def main(argv=None):
         ops = 2.0 * M * N * K
         nbytes = 4 * M * K + N * K * a.bits_w // 8 + 8 * N + 4 * M * n_out
         label = "linear M%d N%d K%d act%d a%d w%d %s" % (M, N, K, a.act, a.bits, a.bits_w, "per-tensor" if a.per_tensor else "per-row")
+    elif a.op == "wonly":
+        # weight-only layer: fp32 activations against integer weights (float matmul, tf32 operands)
+        M, N, K = a.dims
+        n_out = N // 2 if a.act >= 2 else N
+        wq = torch.randint(-7, 8, (N, K if a.bits_w == 8 else K // 2), generator=g, dtype=torch.int8, device=dev)
+        if a.bits_w == 4:
+            wq = wq.view(torch.uint8)
+        sw = torch.rand(N, generator=g, device=dev) * 1e-3
+        prec = aqt.FLOAT_TF32X2 if a.x2 else aqt.FLOAT_TF32
+        ws = torch.empty(aqt.aqt_workspace_bytes(aqt.OP_LINEAR_WEIGHT_ONLY_X2 if a.x2 else aqt.OP_LINEAR_WEIGHT_ONLY, M, N, K, 0, a.bits_w) + 256,
+                         dtype=torch.uint8, device=dev)
+        sets = []
+        for _ in range(a.sets):
+            x = torch.randn((M, K), generator=g, device=dev)
+            y = torch.empty((M, n_out), dtype=torch.float32, device=dev)
+            rr = torch.randn((M, n_out), generator=g, device=dev) if a.residual else None
+            sets.append((x, y, rr))
+
+        def make_calls(stream=None):
+            return [aqt.bind_linear_fwd_weight_only(x, wq, sw, None, rr, 0.5, a.bits_w, a.act, y, ws, stream, precision=prec)
+                    for (x, y, rr) in sets]
+        ops = 2.0 * M * N * K
+        nbytes = 4 * M * K + N * K * a.bits_w // 8 + 8 * N + 4 * M * n_out * (2 if a.residual else 1)
+        label = "wonly%s M%d N%d K%d act%d w%d res%d" % ("-x2" if a.x2 else "", M, N, K, a.act, a.bits_w, int(a.residual))
     else:
         M, K = a.dims
         sets = []

@@ -56,7 +56,7 @@ def _bound_out(act, z, dz, residual_scale, has_res, y_ref):
     return d + 2.0 ** -23 * np.abs(y_ref)
 
 
-def _check(M, N, K, bits_w, act, seed=0, residual=False, bias=True, ldx=None, x_scale=1.0):
+def _check(M, N, K, bits_w, act, seed=0, residual=False, bias=True, ldx=None, x_scale=1.0, precision=aqt.FLOAT_TF32):
     x = gen.normal(seed, 17, M, K, std=x_scale)
     wq, s_w, w_dev = _weights(seed, N, K, bits_w)
     b = gen.normal(seed, 19, 1, N, std=0.05)[0] if bias else None
@@ -71,11 +71,14 @@ def _check(M, N, K, bits_w, act, seed=0, residual=False, bias=True, ldx=None, x_
         xd = buf[:, :K]
     y = torch.full((M, n_out), float("nan"), dtype=torch.float32, device=DEV)
     aqt.aqt_linear_fwd_weight_only(xd, _dev(w_dev), _dev(s_w), None if b is None else _dev(b), None if res is None else _dev(res), 0.5,
-                                   bits_w=bits_w, act=act, y=y)
+                                   bits_w=bits_w, precision=precision, act=act, y=y)
     assert aqt.aqt_device_status() == 0
     got = y.cpu().numpy().astype(np.float64)
     assert np.all(np.isfinite(got))
-    dz = (2.0 ** -10 + K * 2.0 ** -24) * mag + 2.0 ** -23 * np.abs(z)
+    # two-term form: the dropped part of lo is below 2^-10 of lo, itself below 2^-10 of x; 2K summands
+    operand = 2.0 ** -10 if precision == aqt.FLOAT_TF32 else 2.0 ** -20
+    terms = K if precision == aqt.FLOAT_TF32 else 2 * K
+    dz = (operand + terms * 2.0 ** -24) * mag + 2.0 ** -23 * np.abs(z)
     tol = _bound_out(act, z, dz, 0.5, residual, y_ref)
     err = np.abs(got - y_ref)
     assert np.all(err <= tol), "max err/tol %.3g at %s" % ((err / tol).max(), np.unravel_index((err / tol).argmax(), err.shape))
@@ -100,6 +103,22 @@ def test_weight_only_residual_no_bias_and_padded_rows():
     _check(700, 512, 2048, 4, orc.ACT_NONE, seed=3, residual=True, bias=False)
     _check(130, 256, 100, 8, orc.ACT_NONE, seed=4, ldx=128)
     _check(130, 256, 512, 4, orc.ACT_SWISH, seed=5, ldx=516)
+
+
+@pytest.mark.parametrize("bits_w", [8, 4])
+@pytest.mark.parametrize("M,N,K", [(300, 512, 512), (257, 512, 2048), (129, 136, 100), (16, 64, 4)])
+def test_weight_only_two_term_form(M, N, K, bits_w):
+    _check(M, N, K, bits_w, orc.ACT_NONE, precision=aqt.FLOAT_TF32X2)
+    _check(M, N, K, bits_w, orc.ACT_SWISH, seed=1, residual=True, ldx=K + 8, precision=aqt.FLOAT_TF32X2)
+
+
+def test_weight_only_two_term_form_is_far_more_accurate():
+    """x = hi + lo exactly, hi a tf32 value: the operand error of the two-term form is about 2^-20
+    of the terms against 2^-10 for one term.  Measured against the same oracle values."""
+    e1, _, mag = _check(512, 512, 1024, 8, orc.ACT_NONE, seed=6, bias=False)
+    e2, _, _ = _check(512, 512, 1024, 8, orc.ACT_NONE, seed=6, bias=False, precision=aqt.FLOAT_TF32X2)
+    assert (e2 / mag).max() < 2.0 ** -18
+    assert np.median(e2 / mag) < np.median(e1 / mag) / 64
 
 
 def test_weight_only_error_is_of_tf32_size_not_larger():
@@ -157,11 +176,11 @@ def test_weight_only_argument_errors():
     i64, vp, f = ctypes.c_int64, ctypes.c_void_p, ctypes.c_float(1.0)
     one = vp(256)
 
-    def call(M, N, K, bits_w=8, act=0, x=one, ldx=None, ldy=None, ws=one, wsb=1 << 30):
+    def call(M, N, K, bits_w=8, act=0, x=one, ldx=None, ldy=None, ws=one, wsb=1 << 30, precision=0):
         ldx = K if ldx is None else ldx
         ldy = N if ldy is None else ldy
-        return L.aqt_linear_fwd_weight_only(x, i64(ldx), one, one, None, None, i64(0), f, i64(M), i64(N), i64(K), bits_w, act, one,
-                                            i64(ldy), ws, ctypes.c_size_t(wsb), None)
+        return L.aqt_linear_fwd_weight_only(x, i64(ldx), one, one, None, None, i64(0), f, i64(M), i64(N), i64(K), bits_w, precision,
+                                            act, one, i64(ldy), ws, ctypes.c_size_t(wsb), None)
     assert call(128, 256, 130) == -1            # K not a multiple of 4
     assert call(128, 250, 128) == -1            # N not a multiple of 4
     assert call(128, 260, 128, act=2) == -1     # GLU needs N % 8 == 0
@@ -171,5 +190,8 @@ def test_weight_only_argument_errors():
     assert call(128, 256, 128, x=vp(260)) == -2  # x not 16-byte aligned
     assert call(128, 256, 128, ws=None) == -4
     assert call(128, 256, 128, wsb=1000) == -4
+    assert call(128, 256, 128, precision=2) == -1
+    assert call(128, 256, 128, precision=1, wsb=4 * 256 * 128) == -4  # the two-term form needs the split activations too
     assert call(0, 256, 128) == 0               # empty: no-op
     assert aqt.aqt_workspace_bytes(aqt.OP_LINEAR_WEIGHT_ONLY, 128, 256, 128, 0, 4) == 4 * 256 * 128
+    assert aqt.aqt_workspace_bytes(aqt.OP_LINEAR_WEIGHT_ONLY_X2, 128, 256, 128, 0, 4) == 8 * 256 * 128 + 8 * 128 * 128
