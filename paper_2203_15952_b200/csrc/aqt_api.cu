@@ -253,7 +253,7 @@ int aqt_qmatmul_requant(const void* xq, const float* s_x, int s_x_kind, const vo
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
 
-  if (!requant_applies(M, N, K, act)) {
+  if (!requant_applies(M, N, K, act, y != nullptr, pack_out != 0)) {
     // Shapes the fused kernel does not take: the two steps one after the other, through y.
     if (y == nullptr) return AQT_ERR_UNSUPPORTED;
     rc = aqt_qmatmul(xq, s_x, s_x_kind, wq, s_w, bias, residual, ldr, residual_scale, M, N, K, bits_a, bits_w, act, y, ldy, nullptr,
@@ -294,7 +294,7 @@ int aqt_qmatmul_requant(const void* xq, const float* s_x, int s_x_kind, const vo
   p.M = (int)M;
   p.N = (int)N;
   p.K = (int)K;
-  p.n_out = (int)N;
+  p.n_out = (int)n_out;
   p.tiles_m = p.tiles_n = p.k_blocks = 0;
   p.small_acc = (K * (int64_t)(qmax_of(bits_a) + 1) * (qmax_of(bits_w) + 1) <= (1ll << 22)) ? 1 : 0;
   rp.q_out = nullptr;

@@ -71,6 +71,53 @@ __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r
       "r"(r[31])
       : "memory");
 }
+// 32 lanes x 16 consecutive 32-bit columns (the GLU form: a warp owns 16 value and 16 gate columns).
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_32x16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+      "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+// dequant32 / swish32 of qgemm_sm100.cuh on 16 columns.
+template <int ACCK>
+__device__ __forceinline__ void dequant16(const uint32_t (&acc)[16], float sx, uint32_t sw_smem, uint32_t b_smem, float (&z)[16]) {
+  const float2 sx2 = make_float2(sx, sx);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    float w0, w1, w2, w3, b0, b1, b2, b3;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(w0), "=f"(w1), "=f"(w2), "=f"(w3) : "r"(sw_smem + 16 * j));
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(b0), "=f"(b1), "=f"(b2), "=f"(b3) : "r"(b_smem + 16 * j));
+    const float2 z01 = __ffma2_rn(__fmul2_rn(acc_to_float2<ACCK>(acc[4 * j + 0], acc[4 * j + 1]), sx2), make_float2(w0, w1), make_float2(b0, b1));
+    const float2 z23 = __ffma2_rn(__fmul2_rn(acc_to_float2<ACCK>(acc[4 * j + 2], acc[4 * j + 3]), sx2), make_float2(w2, w3), make_float2(b2, b3));
+    z[4 * j + 0] = z01.x;
+    z[4 * j + 1] = z01.y;
+    z[4 * j + 2] = z23.x;
+    z[4 * j + 3] = z23.y;
+  }
+}
+__device__ __forceinline__ void swish16(float (&a)[16]) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const float2 z = make_float2(a[2 * j], a[2 * j + 1]);
+    const float2 t = __fmul2_rn(z, make_float2(-1.4426950408889634f, -1.4426950408889634f));
+    const float2 d = __fadd2_rn(make_float2(1.0f, 1.0f), make_float2(ex2_approx(t.x), ex2_approx(t.y)));
+    const float2 y = __fmul2_rn(z, make_float2(rcp_approx(d.x), rcp_approx(d.y)));
+    a[2 * j] = y.x;
+    a[2 * j + 1] = y.y;
+  }
+}
+
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ uint4 ld_relaxed_gpu_v4(const uint32_t* p) {
@@ -129,20 +176,20 @@ __device__ __forceinline__ uint32_t nibbles_of(uint32_t w0, uint32_t w1) {
   return __byte_perm(y0, y1, 0x6420);
 }
 
-// 32 values of one row -> 8 words of int8 codes (PACK: 4 words of nibbles).
-template <int ROUNDING, bool PACK>
-__device__ __forceinline__ void codes32(const uint32_t (&u)[32], const ScaleCtx& c, int qmax, uint32_t (&w)[8]) {
+// NV (32 or 16) values of one row -> NV / 4 words of int8 codes (PACK: NV / 8 words of nibbles).
+template <int ROUNDING, bool PACK, int NV>
+__device__ __forceinline__ void codes_of(const uint32_t (&u)[NV], const ScaleCtx& c, int qmax, uint32_t (&w)[NV / 4]) {
   if (c.fast) {
     const float2 s_neg = make_float2(-c.s, -c.s), r2 = make_float2(c.r, c.r);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
+    for (int j = 0; j < NV / 4; ++j) {
       const float2 c01 = code_bits2<ROUNDING>(make_float2(__uint_as_float(u[4 * j]), __uint_as_float(u[4 * j + 1])), s_neg, r2);
       const float2 c23 = code_bits2<ROUNDING>(make_float2(__uint_as_float(u[4 * j + 2]), __uint_as_float(u[4 * j + 3])), s_neg, r2);
       w[j] = low_bytes(__float_as_uint(c01.x), __float_as_uint(c01.y), __float_as_uint(c23.x), __float_as_uint(c23.y));
     }
   } else {
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
+    for (int j = 0; j < NV / 4; ++j)
       w[j] = low_bytes((uint32_t)quantize_elem<ROUNDING>(__uint_as_float(u[4 * j]), c, qmax),
                        (uint32_t)quantize_elem<ROUNDING>(__uint_as_float(u[4 * j + 1]), c, qmax),
                        (uint32_t)quantize_elem<ROUNDING>(__uint_as_float(u[4 * j + 2]), c, qmax),
@@ -150,18 +197,23 @@ __device__ __forceinline__ void codes32(const uint32_t (&u)[32], const ScaleCtx&
   }
   if (PACK) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) w[j] = nibbles_of(w[2 * j], w[2 * j + 1]);
+    for (int j = 0; j < NV / 8; ++j) w[j] = nibbles_of(w[2 * j], w[2 * j + 1]);
   }
 }
 
-template <bool BPACK, bool SMALL, bool WITH_Y, int ROUNDING, bool PACK_OUT>
+// GLU: a tile's 128 weight rows are 64 value channels and their 64 gate channels; it yields 64
+// output columns u = v * sigmoid(g) (then Swish for AQT_ACT_GLU_SWISH), 16 per epilogue warp.
+// The GLU form writes codes and scales only (no fp32 output, no residual, no nibble packing).
+template <bool BPACK, bool SMALL, bool WITH_Y, int ROUNDING, bool PACK_OUT, bool GLU = false>
 __global__ void __launch_bounds__(32 * 19, 1)
 qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                      const __grid_constant__ CUtensorMap tm_y,
                      const __grid_constant__ CUtensorMap tm_r, const RequantParams rp) {
   using Cfg = RequantCfg<WITH_Y>;
   constexpr int BN = Cfg::BN, EW = Cfg::EW, STAGES = Cfg::kStages, HALF = BN / 2;
+  static_assert(!GLU || (!WITH_Y && !PACK_OUT), "the GLU form writes int8 codes and scales only");
   const GemmParams& p = rp.g;
+  const int n_out = GLU ? p.N / 2 : p.N;  // output columns
 
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full_bar[STAGES];
@@ -227,9 +279,11 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     tmem_relinquish();
   }
   for (int t = threadIdx.x; t < BN; t += blockDim.x) {
-    const int n = tn * BN + t;
+    // scales and biases of the tile's weight rows: (GLU) values first, then gates
+    const int n = !GLU ? tn * BN + t : (t < HALF ? tn * HALF + t : p.N / 2 + tn * HALF + (t - HALF));
+    const int limit = (GLU && t < HALF) ? p.N / 2 : p.N;
     float wv = 0.0f, bv = 0.0f;
-    if (n < p.N) {
+    if (n < limit) {
       wv = __ldg(p.s_w + n);
       if (p.bias != nullptr) bv = __ldg(p.bias + n);
     }
@@ -248,7 +302,7 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       uint32_t it = 0;
       bool ok = true;
       {
-        const int row0 = tn * BN, row1 = tn * BN + HALF;
+        const int row0 = GLU ? tn * HALF : tn * BN, row1 = GLU ? p.N / 2 + tn * HALF : tn * BN + HALF;
         const uint32_t bar = smem_u32(&b_loaded_bar);
         if (BPACK) {
           mbar_arrive_expect_tx(bar, (uint32_t)p.k_blocks * BN * 64);
@@ -347,14 +401,14 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     // ------------------------------------------------------------------ epilogue warps
     const int ew = warp - 2;
     const int quad = warp & 3;   // TMEM lane quadrant this warp may access
-    const int cpart = ew >> 2;   // which 32 columns of the tile
-    const int col = cpart * 32;
+    const int cpart = ew >> 2;   // which 32 (GLU: 16) output columns of the tile
+    const int col = cpart * (GLU ? 16 : 32);
     const int row_in_tile = quad * 32 + lane;
       const uint32_t y_buf = smem_epi + ew * kStageBufBytes;
     const uint32_t c_sw = smem_scale + (uint32_t)col * 4, c_bias = c_sw + BN * 4;
     const bool has_res = WITH_Y && p.residual != nullptr;
-    const int oc = tn * BN + col;  // first output column of this warp
-    const bool cols_ok = oc < p.N;
+    const int oc = tn * (GLU ? HALF : BN) + col;  // first output column of this warp
+    const bool cols_ok = oc < n_out;
     bool ok = true;
 
     if (BPACK) {
@@ -405,33 +459,55 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         if (!mbar_wait(smem_u32(&tmem_full_bar[buf]), aph, &abort_flag, t_start)) { ok = false; break; }
         tc_fence_after();
         const uint32_t taddr = tmem_base + buf * BN + ((uint32_t)(quad * 32) << 16) + col;
-        uint32_t acc[32];
-        float a[32];
-        tmem_ld_32x32(taddr, acc);
-        tmem_ld_wait();
-        dequant32<SMALL>(acc, sx, c_sw, c_bias, a);
-        if (p.act == AQT_ACT_SWISH) swish32(a);
-        if (has_res) {
-          if (!mbar_wait(smem_u32(&res_bar[ew]), i & 1, &abort_flag, t_start)) { ok = false; break; }
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const uint32_t src = y_buf + lane * 128 + ((j ^ (lane & 7)) << 4);
-            float r0, r1, r2, r3;
-            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r0), "=f"(r1), "=f"(r2), "=f"(r3) : "r"(src) : "memory");
-            a[4 * j + 0] = __fmaf_rn(p.residual_scale, a[4 * j + 0], r0);
-            a[4 * j + 1] = __fmaf_rn(p.residual_scale, a[4 * j + 1], r1);
-            a[4 * j + 2] = __fmaf_rn(p.residual_scale, a[4 * j + 2], r2);
-            a[4 * j + 3] = __fmaf_rn(p.residual_scale, a[4 * j + 3], r3);
-          }
-          __syncwarp();
-        }
         float amax = 0.0f;
+        uint32_t acc[32];
+        float a[32];  // the non-GLU form's u, staged for the fp32 output further down
+        if constexpr (GLU) {
+          // gates first: g = sigmoid(z_gate); then the values are scaled by it
+          uint32_t accv[16], accg[16];
+          float av[16], g[16];
+          tmem_ld_32x16(taddr + HALF, accg);
+          tmem_ld_32x16(taddr, accv);
+          tmem_ld_wait();
+          dequant16<SMALL>(accg, sx, c_sw + HALF * 4, c_bias + HALF * 4, g);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          amax = fmaxf(amax, fabsf(a[j]));
-          acc[j] = __float_as_uint(a[j]);
+          for (int j = 0; j < 16; ++j) g[j] = sigmoid_f(g[j]);
+          dequant16<SMALL>(accv, sx, c_sw, c_bias, av);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) av[j] = av[j] * g[j];
+          if (p.act == AQT_ACT_GLU_SWISH) swish16(av);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            amax = fmaxf(amax, fabsf(av[j]));
+            accv[j] = __float_as_uint(av[j]);
+          }
+          tmem_st_32x16(taddr, accv);  // u replaces the value accumulators
+        } else {
+          tmem_ld_32x32(taddr, acc);
+          tmem_ld_wait();
+          dequant32<SMALL>(acc, sx, c_sw, c_bias, a);
+          if (p.act == AQT_ACT_SWISH) swish32(a);
+          if (has_res) {
+            if (!mbar_wait(smem_u32(&res_bar[ew]), i & 1, &abort_flag, t_start)) { ok = false; break; }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const uint32_t src = y_buf + lane * 128 + ((j ^ (lane & 7)) << 4);
+              float r0, r1, r2, r3;
+              asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r0), "=f"(r1), "=f"(r2), "=f"(r3) : "r"(src) : "memory");
+              a[4 * j + 0] = __fmaf_rn(p.residual_scale, a[4 * j + 0], r0);
+              a[4 * j + 1] = __fmaf_rn(p.residual_scale, a[4 * j + 1], r1);
+              a[4 * j + 2] = __fmaf_rn(p.residual_scale, a[4 * j + 2], r2);
+              a[4 * j + 3] = __fmaf_rn(p.residual_scale, a[4 * j + 3], r3);
+            }
+            __syncwarp();
+          }
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            amax = fmaxf(amax, fabsf(a[j]));
+            acc[j] = __float_as_uint(a[j]);
+          }
+          tmem_st_32x32(taddr, acc);
         }
-        tmem_st_32x32(taddr, acc);
         // this warp's part of the row maxima (columns beyond N contribute nothing)
         amax_part[i % kSlots][cpart][row_in_tile] = cols_ok ? __float_as_uint(amax) : 0u;
         __syncwarp();
@@ -493,25 +569,37 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         const ScaleCtx c = make_scale_ctx(amax, rp.qmax_out);
         if (tn == 0 && cpart == 0 && row0_warp + lane < p.M) rp.s_out[row0_warp + lane] = c.s;
         const uint32_t taddr = tmem_base + buf * BN + ((uint32_t)(quad * 32) << 16) + col;
-        uint32_t u[32], w[8];
-        tmem_st_wait();  // this warp's stores of pass 1 (long complete)
-        tmem_ld_32x32(taddr, u);
-        tmem_ld_wait();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[buf]));
-        codes32<ROUNDING, PACK_OUT>(u, c, rp.qmax_out, w);
-        // Each thread holds 32 consecutive codes of its row: one or two 16-byte stores, each a
-        // whole 32-byte sector (or half of one for packed nibbles), straight to global memory.
         const int m = row0_warp + lane;
-        if (m < p.M && cols_ok) {
-          if (PACK_OUT) {
-            uint4* dst = reinterpret_cast<uint4*>(rp.q_out + (size_t)m * (p.N / 2) + oc / 2);
-            *dst = make_uint4(w[0], w[1], w[2], w[3]);
-          } else {
-            uint4* dst = reinterpret_cast<uint4*>(rp.q_out + (size_t)m * p.N + oc);
-            dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-            if (oc + 16 < p.N) dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        tmem_st_wait();  // this warp's stores of pass 1 (long complete)
+        if constexpr (GLU) {
+          uint32_t u[16], w[4];
+          tmem_ld_32x16(taddr, u);
+          tmem_ld_wait();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[buf]));
+          codes_of<ROUNDING, false, 16>(u, c, rp.qmax_out, w);
+          // 16 consecutive codes of the row: one 16-byte store
+          if (m < p.M && cols_ok) *reinterpret_cast<uint4*>(rp.q_out + (size_t)m * n_out + oc) = make_uint4(w[0], w[1], w[2], w[3]);
+        } else {
+          uint32_t u[32], w[8];
+          tmem_ld_32x32(taddr, u);
+          tmem_ld_wait();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[buf]));
+          codes_of<ROUNDING, PACK_OUT, 32>(u, c, rp.qmax_out, w);
+          // Each thread holds 32 consecutive codes of its row: one or two 16-byte stores, each a
+          // whole 32-byte sector (or half of one for packed nibbles), straight to global memory.
+          if (m < p.M && cols_ok) {
+            if (PACK_OUT) {
+              uint4* dst = reinterpret_cast<uint4*>(rp.q_out + (size_t)m * (p.N / 2) + oc / 2);
+              *dst = make_uint4(w[0], w[1], w[2], w[3]);
+            } else {
+              uint4* dst = reinterpret_cast<uint4*>(rp.q_out + (size_t)m * p.N + oc);
+              dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+              if (oc + 16 < p.N) dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+            }
           }
         }
       }
@@ -540,13 +628,16 @@ static size_t requant_exchange_bytes(int64_t M, int64_t N) {
   return round_up((size_t)ceil_div(M, kBM) * (size_t)ceil_div(N, 128) * kBM * 4, 256);
 }
 
-// True if this kernel takes the shape.
-static bool requant_applies(int64_t M, int64_t N, int64_t K, int act) {
+// True if this kernel takes the call: K <= 512; NONE / Swish in every form, the GLU forms when
+// only int8 codes and scales are asked for (no fp32 output, hence no residual, no nibble packing).
+static bool requant_applies(int64_t M, int64_t N, int64_t K, int act, bool with_y, bool pack_out) {
   const int sms = sm_count() > 0 ? sm_count() : 148;
-  return M > 0 && ceil_div(K, kBK) <= kWsMaxKBlocks && ceil_div(N, 128) <= sms && (act == AQT_ACT_NONE || act == AQT_ACT_SWISH);
+  if (!(M > 0 && ceil_div(K, kBK) <= kWsMaxKBlocks && ceil_div(N, 128) <= sms)) return false;
+  if (act == AQT_ACT_NONE || act == AQT_ACT_SWISH) return true;
+  return !with_y && !pack_out;
 }
 
-template <bool BPACK, bool SMALL, bool WITH_Y, int ROUNDING, bool PACK_OUT>
+template <bool BPACK, bool SMALL, bool WITH_Y, int ROUNDING, bool PACK_OUT, bool GLU = false>
 static int launch_requant_inst(const int8_t* a, const void* b, void* q_out, float* y, int64_t ldy, RequantParams rp,
                                void* exchange, cudaStream_t st) {
   using Cfg = RequantCfg<WITH_Y>;
@@ -578,7 +669,7 @@ static int launch_requant_inst(const int8_t* a, const void* b, void* q_out, floa
       if (rc != AQT_OK) return rc;
     }
   }
-  auto kernel = qgemm_requant_kernel<BPACK, SMALL, WITH_Y, ROUNDING, PACK_OUT>;
+  auto kernel = qgemm_requant_kernel<BPACK, SMALL, WITH_Y, ROUNDING, PACK_OUT, GLU>;
   static bool attr_set = false;
   if (!attr_set) {
     AQT_RETURN_IF_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
@@ -605,6 +696,15 @@ static int launch_requant_inst(const int8_t* a, const void* b, void* q_out, floa
 static int launch_requant(const int8_t* a, const void* b, bool b_packed, void* q_out, float* y, int64_t ldy, const RequantParams& rp,
                           void* exchange, cudaStream_t st) {
   const bool small = rp.g.small_acc != 0;
+  if (rp.g.act == AQT_ACT_GLU || rp.g.act == AQT_ACT_GLU_SWISH) {
+    if (y != nullptr || rp.pack_out) return AQT_ERR_UNSUPPORTED;
+#define AQT_RQ_GLU(BP, SM)                                                                                                        \
+  (rp.rounding == AQT_ROUND_HALF_UP_FLOOR ? launch_requant_inst<BP, SM, false, AQT_ROUND_HALF_UP_FLOOR, false, true>(a, b, q_out, y, ldy, rp, exchange, st) \
+                                          : launch_requant_inst<BP, SM, false, AQT_ROUND_NEAREST_EVEN, false, true>(a, b, q_out, y, ldy, rp, exchange, st))
+    if (b_packed) return small ? AQT_RQ_GLU(true, true) : AQT_RQ_GLU(true, false);
+    return small ? AQT_RQ_GLU(false, true) : AQT_RQ_GLU(false, false);
+#undef AQT_RQ_GLU
+  }
 #define AQT_RQ(BP, SM, WY)                                                                                                 \
   (rp.pack_out ? (rp.rounding == AQT_ROUND_HALF_UP_FLOOR                                                                     \
                       ? launch_requant_inst<BP, SM, WY, AQT_ROUND_HALF_UP_FLOOR, true>(a, b, q_out, y, ldy, rp, exchange, st) \

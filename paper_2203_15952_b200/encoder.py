@@ -14,9 +14,9 @@ and are replaced by the identity:
     h <- h + 1/2 * W_b2 . Swish(W_b1 . h)          feed-forward module b
 
 Residual adds are fp32 and are fused into the epilogue of the producing linear.  Where a linear
-with K <= 512 and no GLU feeds another quantized linear, its epilogue also quantizes its output
-rows (aqt_qmatmul_requant): the fp32 tensor between the two is then written only if it is needed
-as well (the residual stream, or a parity check).
+with K <= 512 feeds another quantized linear, its epilogue also quantizes its output rows
+(aqt_qmatmul_requant): the fp32 tensor between the two is then written only if it is needed as
+well (the residual stream, or a parity check; the GLU layer only fuses when it is not).
 """
 from __future__ import annotations
 
@@ -81,11 +81,14 @@ class LayerRunner:
         return aqt.aqt_qmatmul(xq, s_x, layer.wq, layer.s_w, layer.bias, residual, residual_scale, K=s.K, bits_a=8, bits_w=s.bits_w,
                                act=s.act, s_x_kind=self.a_scale_kind, y=y, workspace=self.workspace)
 
-    def fuses_requant(self, layer: QuantLinear) -> bool:
-        """True if `layer`'s matmul can quantize its own output rows in its epilogue."""
+    def fuses_requant(self, layer: QuantLinear, with_y: bool = True) -> bool:
+        """True if `layer`'s matmul can quantize its own output rows in its epilogue (the GLU
+        forms only when the fp32 output is not wanted as well)."""
         s = layer.spec
-        return (self.a_scale_kind == aqt.SCALE_ROW and s.K <= 512 and s.K % 16 == 0 and s.act in (aqt.ACT_NONE, aqt.ACT_SWISH)
-                and s.N % 16 == 0 and s.N <= 128 * 148)
+        ok = self.a_scale_kind == aqt.SCALE_ROW and s.K <= 512 and s.K % 16 == 0 and s.n_out % 16 == 0 and s.N <= 128 * 148
+        if s.act in (aqt.ACT_GLU, aqt.ACT_GLU_SWISH):
+            return ok and not with_y
+        return ok
 
     def code_buffers(self, role: str, cols: int):
         """Codes (int8 containers) and row scales of an activation tensor, one pair of buffers per role."""
@@ -178,6 +181,7 @@ class ConformerBlockLinears:
                 keep[name] = t.clone()
 
         parity = keep is not None  # then every fp32 intermediate is written as well
+        c_codes = None
         self._ffn(L[0], L[1], h_in, self.h_a, 0.5, parity, note)
         note(L[1].spec.name, self.h_a)
         # q, k, v read the same h: quantize it once (the codes do not depend on the consumer) and
@@ -192,13 +196,17 @@ class ConformerBlockLinears:
             vq, vs = run.quantize_input(self.v, L[5].spec.bits_a)
             bq, bs = run.matmul_requant(L[5], vq, vs, L[6].spec.bits_a, "h", y=self.h_b, residual=self.h_a, residual_scale=1.0)
             note(L[5].spec.name, self.h_b)
-            run.matmul(L[6], bq, bs, self.c); note(L[6].spec.name, self.c)
+            if not parity and run.fuses_requant(L[6], with_y=False) and run.fuses_requant(L[7]):
+                # c = Swish(GLU(W_pw1 h)) is only read by pointwise 2: it leaves pointwise 1 as codes
+                c_codes = run.matmul_requant(L[6], bq, bs, L[7].spec.bits_a, "c")
+            else:
+                run.matmul(L[6], bq, bs, self.c); note(L[6].spec.name, self.c)
         else:
             run(L[5], self.v, self.h_b, residual=self.h_a, residual_scale=1.0); note(L[5].spec.name, self.h_b)
             run(L[6], self.h_b, self.c); note(L[6].spec.name, self.c)
         # h_a = h_b + W_pw2 c, again as fp32 and as codes (first layer of feed-forward module b)
         if run.fuses_requant(L[7]):
-            cq, cs = run.quantize_input(self.c, L[7].spec.bits_a)
+            cq, cs = c_codes if c_codes is not None else run.quantize_input(self.c, L[7].spec.bits_a)
             aq, as_ = run.matmul_requant(L[7], cq, cs, L[8].spec.bits_a, "h", y=self.h_a, residual=self.h_b, residual_scale=1.0)
             note(L[7].spec.name, self.h_a)
             self._ffn(L[8], L[9], self.h_a, h_out, 0.5, parity, note, xq=aq, xs=as_)

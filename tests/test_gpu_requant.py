@@ -108,8 +108,43 @@ def test_requant_many_tiles_per_cta():
     _run(12800, 2048, 512, 8, 4, aqt.ACT_SWISH, False, False, 8, aqt.ROUND_NEAREST_EVEN, False)
 
 
+@pytest.mark.parametrize("act", [aqt.ACT_GLU, aqt.ACT_GLU_SWISH])
+@pytest.mark.parametrize("M,N,K,bits_w", [(128, 128, 128, 8), (300, 1024, 512, 4), (1000, 2048, 256, 4), (77, 288, 144, 8),
+                                           (2600, 1024, 512, 8), (129, 4224, 64, 4)])
+def test_requant_glu_forms(act, M, N, K, bits_w):
+    """The GLU forms (a tile = 64 value + 64 gate channels -> 64 output columns).  With y the call
+    runs matmul + quantizer through y, which is checked against the oracle like every other form;
+    without y the fused kernel must give the very same codes and scales."""
+    for rounding, bits_out in ((aqt.ROUND_NEAREST_EVEN, 8), (aqt.ROUND_HALF_UP_FLOOR, 4)):
+        rng = np.random.default_rng(11 + M + N + K + bits_out)
+        xq, wq = _codes(rng, M, K, 8), _codes(rng, N, K, bits_w)
+        s_x = rng.uniform(1e-3, 5e-2, M).astype(np.float32)
+        s_w = rng.uniform(1e-4, 5e-3, N).astype(np.float32)
+        bias = (rng.standard_normal(N) * 0.1).astype(np.float32)
+        acc_ref = orc.int_matmul(xq, wq)
+        y64 = orc.epilogue_f64(acc_ref, s_x, aqt.SCALE_ROW, s_w, bias, None, 0.0, act)
+        z = orc.epilogue_f64(acc_ref, s_x, aqt.SCALE_ROW, s_w, None, None, 0.0, aqt.ACT_NONE)
+        wq_d = _dev(orc.pack_int4(wq)) if bits_w == 4 else _dev(wq)
+        args = (_dev(xq), _dev(s_x), wq_d, _dev(s_w), _dev(bias), None, 1.0)
+        kw = dict(K=K, bits_a=8, bits_w=bits_w, act=act, bits_out=bits_out, rounding=rounding, pack_out=False)
+        n_out = N // 2
+        q_y, s_y, y_d = aqt.aqt_qmatmul_requant(*args, **kw, want_y=True)          # two steps through y
+        q_d = torch.full((M, n_out), 0x55, dtype=torch.int8, device=DEV)
+        s_d = torch.full((M,), float("nan"), dtype=torch.float32, device=DEV)
+        _, _, y_none = aqt.aqt_qmatmul_requant(*args, **kw, q_out=q_d, s_out=s_d)    # the fused kernel
+        assert y_none is None and aqt.aqt_device_status() == 0
+        y = y_d.cpu().numpy()
+        mag = np.maximum(np.maximum(np.abs(y64), np.abs(z[:, :n_out])), np.abs(bias)[None, :n_out])
+        assert np.all(np.abs(y - y64) <= 1e-6 * mag + 1e-30)
+        q_ref, s_ref = orc.quantize(y, bits_out, orc.AXIS_ROW, rounding)
+        assert np.array_equal(s_y.cpu().numpy().view(np.uint32), s_ref.view(np.uint32)) and np.array_equal(q_y.cpu().numpy(), q_ref)
+        assert np.array_equal(s_d.cpu().numpy().view(np.uint32), s_ref.view(np.uint32)), "fused scales differ"
+        assert np.array_equal(q_d.cpu().numpy(), q_ref), "fused codes differ: %d" % (q_d.cpu().numpy() != q_ref).sum()
+
+
 def test_requant_unfused_shapes_go_through_y():
-    """K > 512 and GLU are not taken by the fused kernel: the call runs the two steps through y."""
+    """K > 512 (and the GLU forms with an fp32 output) are not taken by the fused kernel: the call
+    runs the two steps through y."""
     _run(200, 512, 2048, 8, 4, aqt.ACT_NONE, True, True, 8, aqt.ROUND_NEAREST_EVEN, False)
     rng = np.random.default_rng(3)
     xq, wq = _codes(rng, 64, 1024, 8), _codes(rng, 256, 1024, 8)
