@@ -439,6 +439,7 @@ def run_ours(args):
                                  "unit": UNIT}
     if world == 1 and not args.no_encoder:
         line["encoder"] = encoder_frames_per_s(dev)
+        line["encoder_large"] = encoder_frames_per_s(dev, steps=2, cfg=5)
         line["weight_only"] = weight_only_ffn_pair(dev)
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline()
@@ -446,15 +447,16 @@ def run_ours(args):
     return 0
 
 
-def encoder_frames_per_s(dev, steps: int = 5):
+def encoder_frames_per_s(dev, steps: int = 5, cfg: int = 4):
     """Second half of the metric: frames/s of the 17-block Conformer-encoder linear stack
-    (d = 512, ff = 2048, batch 64 x 400 frames, FFN weights int4, attention / pointwise weights int8,
-    int8 per-row activations, fp32 residual adds fused into the epilogues).  170 aqt_linear_fwd calls
-    per step, replayed from a CUDA graph.  Weights are N(0, 1/fan_in) drawn on the GPU (seeded)."""
+    (cfg 4: d = 512, ff = 2048, batch 64 x 400 frames, FFN weights int4, attention / pointwise weights
+    int8; cfg 5: d = 1024, ff = 4096, batch 128 x 512 frames, int4 weights; int8 per-row activations,
+    fp32 residual adds fused into the epilogues).  170 linears per step, replayed from a CUDA graph.
+    Weights are N(0, 1/fan_in) drawn on the GPU (seeded)."""
     import torch
     from paper_2203_15952_b200 import inputs as gen
     from paper_2203_15952_b200.encoder import EncoderStack, QuantLinear
-    w = gen.WORKLOADS[4]
+    w = gen.WORKLOADS[cfg]
     specs = gen.workload_layers(w)
     g = torch.Generator(device=dev).manual_seed(4)
     blocks = []
@@ -462,6 +464,10 @@ def encoder_frames_per_s(dev, steps: int = 5):
         blocks.append([QuantLinear.from_float(s, torch.randn((s.N, s.K), generator=g, device=dev) * (s.K ** -0.5)) for s in specs])
     stack = EncoderStack(w.M, w.d, w.ff, blocks, dev)
     x = torch.randn((w.M, w.d), generator=g, device=dev)
+    if w.x_dist == "student_t3":  # heavy-tailed block-0 input: Student-t with 3 degrees of freedom, unit variance
+        chi = sum(torch.randn((w.M, w.d), generator=g, device=dev) ** 2 for _ in range(3)) / 3.0
+        x = x / torch.sqrt(chi) / (3.0 ** 0.5)
+        del chi
     stream = torch.cuda.current_stream()
     side = torch.cuda.Stream()
     side.wait_stream(stream)

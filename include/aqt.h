@@ -143,8 +143,8 @@ int aqt_qmatmul(const void* xq, const float* s_x, int s_x_kind, const void* wq, 
  * workspace at least aqt_workspace_bytes(AQT_OP_QMATMUL_REQUANT, ...) bytes, 256-byte aligned:
  *           what aqt_qmatmul needs plus the area through which CTAs exchange row maxima.
  * Limits: those of aqt_qmatmul, and N_out % 16 == 0 (N_out % 32 == 0 if pack_out).  The fused
- * kernel takes K <= 512 with act NONE or SWISH, and the GLU forms when only int8 codes and scales
- * are asked for (y == NULL, pack_out == 0); it is launched cooperatively (its CTAs wait on one
+ * kernel takes K <= 512 with act NONE or SWISH, the GLU forms when only int8 codes and scales
+ * are asked for (y == NULL, pack_out == 0), and 512 < K <= 1024 when y == NULL; it is launched cooperatively (its CTAs wait on one
  * another, with the same bounded waits as everything else) on at most one CTA per SM.
  * Other calls run the two steps one after the other through y and return
  * AQT_ERR_UNSUPPORTED if y is NULL.

@@ -272,7 +272,7 @@ int aqt_qmatmul_requant(const void* xq, const float* s_x, int s_x_kind, const vo
   const void* b_codes = wq;
   bool b_packed = false;
   if (bits_w == 4) {
-    if (K % 32 == 0) {
+    if (K % 32 == 0 && K <= 512) {  // the deep-K form (512 < K <= 1024) has no room to unpack in shared memory
       b_packed = true;
     } else {
       rc = launch_unpack_int4(reinterpret_cast<const uint8_t*>(wq), N * K / 2, reinterpret_cast<int8_t*>(ws), st);

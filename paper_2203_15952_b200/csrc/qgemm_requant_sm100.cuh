@@ -42,17 +42,24 @@ struct RequantParams {
   int pack_out;         // 1: two 4-bit codes per byte
 };
 
-template <bool WITH_Y>
+// DEEP: the resident weight slab holds eight k-blocks (K <= 1024, the d = 1024 encoder's first
+// FFN layers and pointwise 1) instead of four.  That leaves no room for the fp32 staging buffers
+// or for the packed weights, so this form writes codes and scales only and reads int8 weights
+// (4-bit ones are sign-extended into the workspace beforehand).
+constexpr int kRequantDeepKBlocks = 8;
+template <bool WITH_Y, bool DEEP = false>
 struct RequantCfg {
+  static_assert(!(DEEP && WITH_Y), "the deep-K form has no room for fp32 staging");
+  static constexpr int kKBlocks = DEEP ? kRequantDeepKBlocks : kWsMaxKBlocks;
   static constexpr int BN = 128;
   static constexpr int EW = 16;
   static constexpr int kThreads = 32 * (2 + EW + 1);  // producer, MMA issuer, epilogue warps, exchange warp
-  static constexpr int kStages = WITH_Y ? 5 : 7;
+  static constexpr int kStages = (WITH_Y || DEEP) ? 5 : 7;
   static constexpr int kABytes = kBM * kBK;
   static constexpr int kBBytes = BN * kBK;
-  static constexpr int kResidentBytes = kWsMaxKBlocks * kBBytes;
+  static constexpr int kResidentBytes = kKBlocks * kBBytes;
   static constexpr int kYBytes = WITH_Y ? EW * kStageBufBytes : 0;
-  static constexpr int kPackedBBytes = kWsMaxKBlocks * BN * 64;  // packed weights wait here for the unpack
+  static constexpr int kPackedBBytes = DEEP ? 0 : kWsMaxKBlocks * BN * 64;  // packed weights wait here for the unpack
   static constexpr int kEpiBytes = kYBytes > kPackedBBytes ? kYBytes : kPackedBBytes;
   static constexpr int kScaleBytes = 2 * BN * 4;
   static constexpr int kTmemCols = 4 * BN;
@@ -204,13 +211,14 @@ __device__ __forceinline__ void codes_of(const uint32_t (&u)[NV], const ScaleCtx
 // GLU: a tile's 128 weight rows are 64 value channels and their 64 gate channels; it yields 64
 // output columns u = v * sigmoid(g) (then Swish for AQT_ACT_GLU_SWISH), 16 per epilogue warp.
 // The GLU form writes codes and scales only (no fp32 output, no residual, no nibble packing).
-template <bool BPACK, bool SMALL, bool WITH_Y, int ROUNDING, bool PACK_OUT, bool GLU = false>
+template <bool BPACK, bool SMALL, bool WITH_Y, int ROUNDING, bool PACK_OUT, bool GLU = false, bool DEEP = false>
 __global__ void __launch_bounds__(32 * 19, 1)
 qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                      const __grid_constant__ CUtensorMap tm_y,
                      const __grid_constant__ CUtensorMap tm_r, const RequantParams rp) {
-  using Cfg = RequantCfg<WITH_Y>;
+  using Cfg = RequantCfg<WITH_Y, DEEP>;
   constexpr int BN = Cfg::BN, EW = Cfg::EW, STAGES = Cfg::kStages, HALF = BN / 2;
+  static_assert(!(DEEP && BPACK), "the deep-K form reads int8 weights");
   static_assert(!GLU || (!WITH_Y && !PACK_OUT), "the GLU form writes int8 codes and scales only");
   const GemmParams& p = rp.g;
   const int n_out = GLU ? p.N / 2 : p.N;  // output columns
@@ -632,22 +640,24 @@ static size_t requant_exchange_bytes(int64_t M, int64_t N) {
 // only int8 codes and scales are asked for (no fp32 output, hence no residual, no nibble packing).
 static bool requant_applies(int64_t M, int64_t N, int64_t K, int act, bool with_y, bool pack_out) {
   const int sms = sm_count() > 0 ? sm_count() : 148;
-  if (!(M > 0 && ceil_div(K, kBK) <= kWsMaxKBlocks && ceil_div(N, 128) <= sms)) return false;
-  if (act == AQT_ACT_NONE || act == AQT_ACT_SWISH) return true;
-  return !with_y && !pack_out;
+  if (!(M > 0 && ceil_div(N, 128) <= sms)) return false;
+  const bool glu = !(act == AQT_ACT_NONE || act == AQT_ACT_SWISH);
+  if (ceil_div(K, kBK) <= kWsMaxKBlocks) return !glu || (!with_y && !pack_out);
+  // 512 < K <= 1024: codes and scales only
+  return ceil_div(K, kBK) <= kRequantDeepKBlocks && !with_y && (!glu || !pack_out);
 }
 
-template <bool BPACK, bool SMALL, bool WITH_Y, int ROUNDING, bool PACK_OUT, bool GLU = false>
+template <bool BPACK, bool SMALL, bool WITH_Y, int ROUNDING, bool PACK_OUT, bool GLU = false, bool DEEP = false>
 static int launch_requant_inst(const int8_t* a, const void* b, void* q_out, float* y, int64_t ldy, RequantParams rp,
                                void* exchange, cudaStream_t st) {
-  using Cfg = RequantCfg<WITH_Y>;
+  using Cfg = RequantCfg<WITH_Y, DEEP>;
   GemmParams& p = rp.g;
   p.tiles_m = (int)ceil_div(p.M, kBM);
   p.tiles_n = (int)ceil_div(p.N, Cfg::BN);
   p.k_blocks = (int)ceil_div(p.K, kBK);
   const int sms = sm_count();
   if (sms <= 0) return AQT_ERR_CUDA;
-  if (p.k_blocks > kWsMaxKBlocks || p.tiles_n > sms) return AQT_ERR_UNSUPPORTED;
+  if (p.k_blocks > Cfg::kKBlocks || p.tiles_n > sms) return AQT_ERR_UNSUPPORTED;
   rp.exchange = reinterpret_cast<uint32_t*>(exchange);
   AQT_RETURN_IF_CUDA(cudaMemsetAsync(exchange, 0, (size_t)p.tiles_m * p.tiles_n * kBM * 4, st));
 
@@ -669,7 +679,7 @@ static int launch_requant_inst(const int8_t* a, const void* b, void* q_out, floa
       if (rc != AQT_OK) return rc;
     }
   }
-  auto kernel = qgemm_requant_kernel<BPACK, SMALL, WITH_Y, ROUNDING, PACK_OUT, GLU>;
+  auto kernel = qgemm_requant_kernel<BPACK, SMALL, WITH_Y, ROUNDING, PACK_OUT, GLU, DEEP>;
   static bool attr_set = false;
   if (!attr_set) {
     AQT_RETURN_IF_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
@@ -696,7 +706,19 @@ static int launch_requant_inst(const int8_t* a, const void* b, void* q_out, floa
 static int launch_requant(const int8_t* a, const void* b, bool b_packed, void* q_out, float* y, int64_t ldy, const RequantParams& rp,
                           void* exchange, cudaStream_t st) {
   const bool small = rp.g.small_acc != 0;
-  if (rp.g.act == AQT_ACT_GLU || rp.g.act == AQT_ACT_GLU_SWISH) {
+  const bool glu = rp.g.act == AQT_ACT_GLU || rp.g.act == AQT_ACT_GLU_SWISH;
+  if (ceil_div(rp.g.K, kBK) > kWsMaxKBlocks) {
+    // deep-K form: int8 weights, codes and scales only
+    if (y != nullptr || b_packed || (glu && rp.pack_out)) return AQT_ERR_UNSUPPORTED;
+#define AQT_RQ_DEEP(SM, PK, GL)                                                                                                   \
+  (rp.rounding == AQT_ROUND_HALF_UP_FLOOR ? launch_requant_inst<false, SM, false, AQT_ROUND_HALF_UP_FLOOR, PK, GL, true>(a, b, q_out, y, ldy, rp, exchange, st) \
+                                          : launch_requant_inst<false, SM, false, AQT_ROUND_NEAREST_EVEN, PK, GL, true>(a, b, q_out, y, ldy, rp, exchange, st))
+    if (glu) return small ? AQT_RQ_DEEP(true, false, true) : AQT_RQ_DEEP(false, false, true);
+    if (rp.pack_out) return small ? AQT_RQ_DEEP(true, true, false) : AQT_RQ_DEEP(false, true, false);
+    return small ? AQT_RQ_DEEP(true, false, false) : AQT_RQ_DEEP(false, false, false);
+#undef AQT_RQ_DEEP
+  }
+  if (glu) {
     if (y != nullptr || rp.pack_out) return AQT_ERR_UNSUPPORTED;
 #define AQT_RQ_GLU(BP, SM)                                                                                                        \
   (rp.rounding == AQT_ROUND_HALF_UP_FLOOR ? launch_requant_inst<BP, SM, false, AQT_ROUND_HALF_UP_FLOOR, false, true>(a, b, q_out, y, ldy, rp, exchange, st) \

@@ -85,8 +85,8 @@ class LayerRunner:
         """True if `layer`'s matmul can quantize its own output rows in its epilogue (the GLU
         forms only when the fp32 output is not wanted as well)."""
         s = layer.spec
-        ok = self.a_scale_kind == aqt.SCALE_ROW and s.K <= 512 and s.K % 16 == 0 and s.n_out % 16 == 0 and s.N <= 128 * 148
-        if s.act in (aqt.ACT_GLU, aqt.ACT_GLU_SWISH):
+        ok = self.a_scale_kind == aqt.SCALE_ROW and s.K <= 1024 and s.K % 16 == 0 and s.n_out % 16 == 0 and s.N <= 128 * 148
+        if s.act in (aqt.ACT_GLU, aqt.ACT_GLU_SWISH) or s.K > 512:
             return ok and not with_y
         return ok
 
@@ -125,7 +125,7 @@ class FfnPair:
         assert len(layers) == 2
         self.layers = layers
         self.run = LayerRunner(M, layers, device, **kw)
-        self.fused = fused and self.run.fuses_requant(layers[0])
+        self.fused = fused and self.run.fuses_requant(layers[0], with_y=keep_u)
         self.keep_u = keep_u or not self.fused
         self.u = torch.empty((M, layers[0].spec.n_out), dtype=torch.float32, device=device) if self.keep_u else None
 
@@ -181,7 +181,6 @@ class ConformerBlockLinears:
                 keep[name] = t.clone()
 
         parity = keep is not None  # then every fp32 intermediate is written as well
-        c_codes = None
         self._ffn(L[0], L[1], h_in, self.h_a, 0.5, parity, note)
         note(L[1].spec.name, self.h_a)
         # q, k, v read the same h: quantize it once (the codes do not depend on the consumer) and
@@ -192,26 +191,37 @@ class ConformerBlockLinears:
                         s_x_kind=run.a_scale_kind, y=self.qkv, workspace=run.workspace)
         note(L[2].spec.name, self.q); note(L[3].spec.name, self.k); note(L[4].spec.name, self.v)
         # h_b = h_a + W_o v is needed both as fp32 (residual stream) and as codes (pointwise 1)
+        bq = bs = cq = cs = None
         if run.fuses_requant(L[5]):
             vq, vs = run.quantize_input(self.v, L[5].spec.bits_a)
             bq, bs = run.matmul_requant(L[5], vq, vs, L[6].spec.bits_a, "h", y=self.h_b, residual=self.h_a, residual_scale=1.0)
-            note(L[5].spec.name, self.h_b)
-            if not parity and run.fuses_requant(L[6], with_y=False) and run.fuses_requant(L[7]):
-                # c = Swish(GLU(W_pw1 h)) is only read by pointwise 2: it leaves pointwise 1 as codes
-                c_codes = run.matmul_requant(L[6], bq, bs, L[7].spec.bits_a, "c")
-            else:
-                run.matmul(L[6], bq, bs, self.c); note(L[6].spec.name, self.c)
         else:
-            run(L[5], self.v, self.h_b, residual=self.h_a, residual_scale=1.0); note(L[5].spec.name, self.h_b)
-            run(L[6], self.h_b, self.c); note(L[6].spec.name, self.c)
+            run(L[5], self.v, self.h_b, residual=self.h_a, residual_scale=1.0)
+        note(L[5].spec.name, self.h_b)
+        # c = Swish(GLU(W_pw1 h_b)) is only read by pointwise 2: it leaves pointwise 1 as codes when it can
+        if not parity and run.fuses_requant(L[6], with_y=False):
+            if bq is None:
+                bq, bs = run.quantize_input(self.h_b, L[6].spec.bits_a)
+            cq, cs = run.matmul_requant(L[6], bq, bs, L[7].spec.bits_a, "c")
+        elif bq is not None:
+            run.matmul(L[6], bq, bs, self.c)
+        else:
+            run(L[6], self.h_b, self.c)
+        if cq is None:
+            note(L[6].spec.name, self.c)
         # h_a = h_b + W_pw2 c, again as fp32 and as codes (first layer of feed-forward module b)
         if run.fuses_requant(L[7]):
-            cq, cs = c_codes if c_codes is not None else run.quantize_input(self.c, L[7].spec.bits_a)
+            if cq is None:
+                cq, cs = run.quantize_input(self.c, L[7].spec.bits_a)
             aq, as_ = run.matmul_requant(L[7], cq, cs, L[8].spec.bits_a, "h", y=self.h_a, residual=self.h_b, residual_scale=1.0)
             note(L[7].spec.name, self.h_a)
             self._ffn(L[8], L[9], self.h_a, h_out, 0.5, parity, note, xq=aq, xs=as_)
         else:
-            run(L[7], self.c, self.h_a, residual=self.h_b, residual_scale=1.0); note(L[7].spec.name, self.h_a)
+            if cq is not None:
+                run.matmul(L[7], cq, cs, self.h_a, residual=self.h_b, residual_scale=1.0)
+            else:
+                run(L[7], self.c, self.h_a, residual=self.h_b, residual_scale=1.0)
+            note(L[7].spec.name, self.h_a)
             self._ffn(L[8], L[9], self.h_a, h_out, 0.5, parity, note)
         note(L[9].spec.name, h_out)
         return h_out
@@ -220,7 +230,7 @@ class ConformerBlockLinears:
              xq: Optional[torch.Tensor] = None, xs: Optional[torch.Tensor] = None) -> None:
         """out = h + rs * W_1 . Swish(W_0 . h); xq, xs: codes and scales of h if already at hand."""
         run = self.run
-        if run.fuses_requant(l0):
+        if run.fuses_requant(l0, with_y=parity):
             if xq is None:
                 xq, xs = run.quantize_input(h, l0.spec.bits_a)
             uq, us = run.matmul_requant(l0, xq, xs, l1.spec.bits_a, "u", y=self.u if parity else None)

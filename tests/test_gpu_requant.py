@@ -108,9 +108,21 @@ def test_requant_many_tiles_per_cta():
     _run(12800, 2048, 512, 8, 4, aqt.ACT_SWISH, False, False, 8, aqt.ROUND_NEAREST_EVEN, False)
 
 
+@pytest.mark.parametrize("M,N,K,bits_w,act", [(300, 1024, 1024, 4, aqt.ACT_SWISH), (1500, 4096, 1024, 4, aqt.ACT_SWISH),
+                                               (129, 512, 640, 8, aqt.ACT_NONE), (700, 2048, 1024, 8, aqt.ACT_SWISH),
+                                               (260, 1024, 768, 4, aqt.ACT_NONE)])
+def test_requant_deep_k_form(M, N, K, bits_w, act):
+    """512 < K <= 1024 (the d = 1024 encoder): the fused kernel with an eight-k-block weight slab
+    takes the call when only codes and scales are wanted.  _run checks the two-step path (with y)
+    against the oracle and then the fused path (without y) against it, bit for bit."""
+    _run(M, N, K, 8, bits_w, act, True, False, 8, aqt.ROUND_NEAREST_EVEN, False)
+    # (the huge-scale special row stays finite only with 4-bit weights at this depth)
+    _run(M, N, K, 8, bits_w, act, False, False, 4, aqt.ROUND_HALF_UP_FLOOR, True, special_rows=(bits_w == 4))
+
+
 @pytest.mark.parametrize("act", [aqt.ACT_GLU, aqt.ACT_GLU_SWISH])
 @pytest.mark.parametrize("M,N,K,bits_w", [(128, 128, 128, 8), (300, 1024, 512, 4), (1000, 2048, 256, 4), (77, 288, 144, 8),
-                                           (2600, 1024, 512, 8), (129, 4224, 64, 4)])
+                                           (2600, 1024, 512, 8), (129, 4224, 64, 4), (300, 2048, 1024, 4), (129, 512, 640, 8)])
 def test_requant_glu_forms(act, M, N, K, bits_w):
     """The GLU forms (a tile = 64 value + 64 gate channels -> 64 output columns).  With y the call
     runs matmul + quantizer through y, which is checked against the oracle like every other form;
@@ -143,13 +155,13 @@ def test_requant_glu_forms(act, M, N, K, bits_w):
 
 
 def test_requant_unfused_shapes_go_through_y():
-    """K > 512 (and the GLU forms with an fp32 output) are not taken by the fused kernel: the call
-    runs the two steps through y."""
+    """K > 1024 (and K > 512 or the GLU forms with an fp32 output) are not taken by the fused
+    kernel: the call runs the two steps through y."""
     _run(200, 512, 2048, 8, 4, aqt.ACT_NONE, True, True, 8, aqt.ROUND_NEAREST_EVEN, False)
     rng = np.random.default_rng(3)
-    xq, wq = _codes(rng, 64, 1024, 8), _codes(rng, 256, 1024, 8)
+    xq, wq = _codes(rng, 64, 2048, 8), _codes(rng, 256, 2048, 8)
     with pytest.raises(aqt.AqtError) as e:
-        aqt.aqt_qmatmul_requant(_dev(xq), _dev(np.ones(64, np.float32)), _dev(wq), _dev(np.ones(256, np.float32)), K=1024)
+        aqt.aqt_qmatmul_requant(_dev(xq), _dev(np.ones(64, np.float32)), _dev(wq), _dev(np.ones(256, np.float32)), K=2048)
     assert e.value.status == -3
 
 
