@@ -233,6 +233,14 @@ def test_cfg5_heavy_tailed_rows_of_the_large_encoder():
     blk.forward(blocks_gpu[1], h0, h1, keep=keep)
     _check_block(w, specs, blocks_cpu[1], keep, h0.cpu().numpy()[rows], rows)
     assert aqt.aqt_device_status() == 0
+    # the production path (no intermediates kept: the first FFN layers and pointwise 1 hand codes
+    # to their consumers straight from their epilogues) gives the same bits as the checked one
+    h0_fused = torch.empty_like(h0)
+    h1_fused = torch.empty_like(h1)
+    blk.forward(blocks_gpu[0], _dev(x), h0_fused)
+    blk.forward(blocks_gpu[1], h0_fused, h1_fused)
+    assert aqt.aqt_device_status() == 0
+    assert torch.equal(h0_fused.view(torch.int32), h0.view(torch.int32)) and torch.equal(h1_fused.view(torch.int32), h1.view(torch.int32))
     # heavy tails: most codes of the first quantizer call collapse near zero
     q, s = aqt.aqt_quantize(_dev(x), 8, aqt.AXIS_ROW)
     q_ref, s_ref = orc.quantize(x[rows], 8, orc.AXIS_ROW)
