@@ -211,3 +211,25 @@ def linear_weight_only_f64(x, wq, s_w, bias=None, residual=None, residual_scale=
     if rc != 0:
         raise ValueError("orc_linear_weight_only_f64: bad argument")
     return (y, z, mag) if return_parts else y
+
+
+def linear_bwd_f64(dy, xq, s_x, wq, s_w, s_x_kind=SCALE_ROW, return_mags=False):
+    """Straight-through backward of the quantized linear layer in double: returns (dx [M, K],
+    dw [N, K], db [N]); with return_mags also the sums of absolute values of the same terms."""
+    dy = np.asarray(dy, dtype=np.float32)
+    assert dy.ndim == 2 and dy.strides[1] == 4
+    M, N = dy.shape
+    lddy = dy.strides[0] // 4 if M > 1 else N
+    xq = np.ascontiguousarray(xq, dtype=np.int8)
+    wq = np.ascontiguousarray(wq, dtype=np.int8)
+    K = xq.shape[1]
+    assert xq.shape == (M, K) and wq.shape == (N, K)
+    s_x = np.ascontiguousarray(s_x, dtype=np.float32)
+    s_w = np.ascontiguousarray(s_w, dtype=np.float32)
+    dx, dw, db = np.empty((M, K)), np.empty((N, K)), np.empty(N)
+    mags = (np.empty((M, K)), np.empty((N, K)), np.empty(N)) if return_mags else (None, None, None)
+    rc = lib().orc_linear_bwd_f64(_p(dy), _i64(lddy), _p(xq), _p(s_x), s_x_kind, _p(wq), _p(s_w), _i64(M), _i64(N), _i64(K),
+                                  _p(dx), _p(dw), _p(db), _p(mags[0]), _p(mags[1]), _p(mags[2]))
+    if rc != 0:
+        raise ValueError("orc_linear_bwd_f64: bad argument")
+    return (dx, dw, db) + (mags if return_mags else ())

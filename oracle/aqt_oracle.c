@@ -352,3 +352,62 @@ int orc_linear_weight_only_f64(const float* x, int64_t ldx, const int8_t* wq, co
   }
   return 0;
 }
+
+/* Backward of the quantized linear layer with straight-through quantizers.  The paper states only
+ * that the scale carries no gradient (Fig. 2: stop_gradient(scale)) and that training runs the
+ * same integer forward ("what you train is what you serve", Section 1); it does not print the
+ * backward products.  The plain straight-through definition is taken: the forward is
+ *   y[m][n] = sum_k xhat[m][k] * what[n][k] + bias[n],  xhat = s_x * xq,  what = s_w * wq,
+ * the quantizers pass gradients through unchanged (d xhat / d x = 1, d what / d w = 1), scales are
+ * constants.  With dy = dL/dy (for an activation the caller supplies dL/dz), every sum in double:
+ *   dx[m][k] = sum_n dy[m][n] * s_w[n] * wq[n][k]
+ *   dw[n][k] = sum_m dy[m][n] * s_x[m] * xq[m][k]       (same [N, K] layout as the codes)
+ *   db[n]    = sum_m dy[m][n]
+ * Optional magnitude outputs (sums of the absolute values of the same terms) bound the rounding
+ * of float implementations.  Any output pointer may be NULL.  dy has row pitch lddy. */
+int orc_linear_bwd_f64(const float* dy, int64_t lddy, const int8_t* xq, const float* s_x, int s_x_kind,
+                       const int8_t* wq, const float* s_w, int64_t M, int64_t N, int64_t K, double* dx,
+                       double* dw, double* db, double* dx_mag, double* dw_mag, double* db_mag) {
+  if (M < 0 || N < 0 || K < 0 || lddy < N) return -1;
+  if (dx) {
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+      for (int64_t k = 0; k < K; ++k) {
+        double s = 0.0, a = 0.0;
+        for (int64_t n = 0; n < N; ++n) {
+          double t = (double)dy[m * lddy + n] * (double)s_w[n] * (double)wq[n * K + k];
+          s += t;
+          a += fabs(t);
+        }
+        dx[m * K + k] = s;
+        if (dx_mag) dx_mag[m * K + k] = a;
+      }
+  }
+  if (dw) {
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < N; ++n)
+      for (int64_t k = 0; k < K; ++k) {
+        double s = 0.0, a = 0.0;
+        for (int64_t m = 0; m < M; ++m) {
+          double sx = s_x_kind == ORC_SCALE_ROW ? (double)s_x[m] : (double)s_x[0];
+          double t = (double)dy[m * lddy + n] * sx * (double)xq[m * K + k];
+          s += t;
+          a += fabs(t);
+        }
+        dw[n * K + k] = s;
+        if (dw_mag) dw_mag[n * K + k] = a;
+      }
+  }
+  if (db) {
+    for (int64_t n = 0; n < N; ++n) {
+      double s = 0.0, a = 0.0;
+      for (int64_t m = 0; m < M; ++m) {
+        s += (double)dy[m * lddy + n];
+        a += fabs((double)dy[m * lddy + n]);
+      }
+      db[n] = s;
+      if (db_mag) db_mag[n] = a;
+    }
+  }
+  return 0;
+}
