@@ -32,7 +32,7 @@
 extern "C" {
 #endif
 
-#define AQT_VERSION 103
+#define AQT_VERSION 104
 
 /* status codes */
 #define AQT_OK 0
@@ -68,6 +68,7 @@ extern "C" {
 #define AQT_OP_QMATMUL_REQUANT 3
 #define AQT_OP_LINEAR_WEIGHT_ONLY 4    /* precision AQT_FLOAT_TF32   */
 #define AQT_OP_LINEAR_WEIGHT_ONLY_X2 5 /* precision AQT_FLOAT_TF32X2 */
+#define AQT_OP_LINEAR_BWD 6
 
 /* how float activations enter the tensor-core float matmul of the weight-only layer */
 #define AQT_FLOAT_TF32 0   /* one term: the upper ten fraction bits of each activation            */
@@ -215,6 +216,37 @@ int aqt_linear_fwd_weight_only(const float* x, int64_t ldx, const void* wq, cons
                                const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K,
                                int bits_w, int precision, int act, float* y, int64_t ldy, void* workspace,
                                size_t workspace_bytes, void* stream);
+
+/*
+ * aqt_linear_bwd -- backward of the quantized linear layer with straight-through quantizers.
+ * The paper states that scales carry no gradient (Fig. 2: stop_gradient(scale)) and that training
+ * runs the same integer forward (Section 1); it does not print the backward products.  This is
+ * the plain straight-through definition: with xhat = s_x * xq and what = s_w * wq the de-quantized
+ * operands of the forward y = xhat . what^T + bias, quantizers passing gradients unchanged,
+ *   dx[m][k] = sum_n dy[m][n] * s_w[n] * wq[n][k]
+ *   dw[n][k] = sum_m dy[m][n] * s_x[m or 0] * xq[m][k]      (the [N, K] layout of the weight codes)
+ *   dbias[n] = sum_m dy[m][n]
+ * dy is the gradient with respect to the layer's pre-activation (for a layer with an activation
+ * or a residual the caller applies those derivatives first).
+ * Arithmetic: dx and dw are float matmuls on the tensor cores (tf32 operands: dy and the scaled
+ * codes each enter with their upper ten fraction bits; binary32 accumulation), so each is within
+ * (2^-9 + depth * 2^-24) of the sum of the absolute values of its terms, depth = N for dx, M for
+ * dw.  dbias is summed in binary32 in a fixed order (the same bits on every run).
+ * dy        fp32 [M, N], row pitch lddy.
+ * xq, s_x, s_x_kind, bits_a   the forward's activation codes and scales (as handed to aqt_qmatmul);
+ *           only read for dw.
+ * wq, s_w, bits_w             the weight codes and scales; only read for dx.
+ * dx        fp32 [M, K], row pitch lddx, or NULL.   dw  fp32 [N, K], row pitch lddw, or NULL.
+ * dbias     fp32 [N] or NULL.
+ * workspace at least aqt_workspace_bytes(AQT_OP_LINEAR_BWD, M, N, K, 0, 0) bytes, 256-byte
+ *           aligned: the transposed, scaled operands (4 * (K * N + (N + K) * M) bytes and change).
+ * Limits: K % 4 == 0, N % 4 == 0; lddy, lddx, lddw multiples of 4; dy, dx, dw 16-byte aligned;
+ * M, N, K < 2^28.  M == 0 or N == 0 is a no-op.
+ */
+int aqt_linear_bwd(const float* dy, int64_t lddy, const void* xq, const float* s_x, int s_x_kind, int bits_a,
+                   const void* wq, const float* s_w, int bits_w, int64_t M, int64_t N, int64_t K, float* dx,
+                   int64_t lddx, float* dw, int64_t lddw, float* dbias, void* workspace, size_t workspace_bytes,
+                   void* stream);
 
 /*
  * aqt_qmatmul_w4_noalloc -- aqt_qmatmul for int8 activations and 4-bit weights that needs no

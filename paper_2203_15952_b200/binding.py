@@ -20,12 +20,12 @@ AXIS_ROW, AXIS_COL, AXIS_TENSOR = 0, 1, 2
 ROUND_HALF_UP_FLOOR, ROUND_NEAREST_EVEN = 0, 1
 SCALE_ROW, SCALE_TENSOR = 0, 1
 ACT_NONE, ACT_SWISH, ACT_GLU, ACT_GLU_SWISH = 0, 1, 2, 3
-OP_QMATMUL, OP_LINEAR_FWD, OP_QMATMUL_REQUANT, OP_LINEAR_WEIGHT_ONLY, OP_LINEAR_WEIGHT_ONLY_X2 = 1, 2, 3, 4, 5
+OP_QMATMUL, OP_LINEAR_FWD, OP_QMATMUL_REQUANT, OP_LINEAR_WEIGHT_ONLY, OP_LINEAR_WEIGHT_ONLY_X2, OP_LINEAR_BWD = 1, 2, 3, 4, 5, 6
 FLOAT_TF32, FLOAT_TF32X2 = 0, 1
 
 EXPORTS = ("aqt_version", "aqt_status_string", "aqt_quantize", "aqt_pack_int4", "aqt_unpack_int4", "aqt_qmatmul",
            "aqt_linear_fwd", "aqt_linear_fwd_host", "aqt_workspace_bytes", "aqt_device_status", "aqt_qmatmul_w4_noalloc",
-           "aqt_selftest_bounded_wait", "aqt_qmatmul_requant", "aqt_linear_fwd_weight_only")
+           "aqt_selftest_bounded_wait", "aqt_qmatmul_requant", "aqt_linear_fwd_weight_only", "aqt_linear_bwd")
 NOALLOC_MAX_WEIGHT_BYTES = 4 << 20
 
 
@@ -310,6 +310,27 @@ def aqt_linear_fwd_weight_only(x: torch.Tensor, wq: torch.Tensor, s_w: torch.Ten
         int(bits_w), int(precision), int(act), _ptr(y), _i64(y.stride(0)), _ptr(workspace), ctypes.c_size_t(workspace.numel()),
         _stream(stream)))
     return y
+
+
+def aqt_linear_bwd(dy: torch.Tensor, xq: Optional[torch.Tensor], s_x: Optional[torch.Tensor], wq: Optional[torch.Tensor],
+                   s_w: Optional[torch.Tensor], *, K: int, bits_a: int = 8, bits_w: int = 8, s_x_kind: int = SCALE_ROW,
+                   want_dx: bool = True, want_dw: bool = True, want_dbias: bool = True,
+                   workspace: Optional[torch.Tensor] = None, stream=None):
+    """Straight-through backward of the quantized linear layer: returns (dx [M, K], dw [N, K],
+    dbias [N]), None for the ones not wanted.  dy fp32 [M, N]; codes and scales as in the forward."""
+    assert dy.is_cuda and dy.dtype == torch.float32 and dy.dim() == 2 and dy.stride(1) == 1
+    M, N = dy.shape
+    f32 = dict(dtype=torch.float32, device=dy.device)
+    dx = torch.empty((M, K), **f32) if want_dx else None
+    dw = torch.empty((N, K), **f32) if want_dw else None
+    db = torch.empty((N,), **f32) if want_dbias else None
+    need = aqt_workspace_bytes(OP_LINEAR_BWD, M, N, K, 0, 0)
+    workspace = _workspace(need, workspace, dy.device)
+    _check("aqt_linear_bwd", lib().aqt_linear_bwd(
+        _ptr(dy), _i64(dy.stride(0)), _ptr(xq), _ptr(s_x), int(s_x_kind), int(bits_a), _ptr(wq), _ptr(s_w), int(bits_w),
+        _i64(M), _i64(N), _i64(K), _ptr(dx), _i64(K), _ptr(dw), _i64(K), _ptr(db), _ptr(workspace),
+        ctypes.c_size_t(0 if workspace is None else workspace.numel()), _stream(stream)))
+    return dx, dw, db
 
 
 def linear_fwd_host_workspace_bytes(M: int, N: int, K: int, bits_a: int, bits_w: int, act: int,

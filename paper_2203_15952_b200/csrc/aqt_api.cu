@@ -1,6 +1,7 @@
 // C ABI of the quantized linear layer: argument validation and kernel launches.
 // Single translation unit: the kernels live in the headers included below.
 #include "aqt_common.cuh"
+#include "backward.cuh"
 #include "pack.cuh"
 #include "qgemm_sm100.cuh"
 #include "qgemm_requant_sm100.cuh"
@@ -41,6 +42,47 @@ size_t ws_linear(int64_t M, int64_t N, int64_t K, int bits_w) {
 size_t ws_weight_only(int64_t M, int64_t N, int64_t K, int precision) {
   if (precision == AQT_FLOAT_TF32X2) return round_up((size_t)N * (size_t)K * 8, 256) + round_up((size_t)M * (size_t)K * 8, 256);
   return round_up((size_t)N * (size_t)K * 4, 256);
+}
+
+// Backward: [ones K | column-sum partials | s_w-scaled W^T [K, N] | dy^T [N, ldm] | s_x-scaled xq^T [K, ldm]], ldm = M rounded up to 4
+struct BwdLayout {
+  size_t ones, partial, wt, dyt, xt, total;
+  int64_t ldm;
+};
+BwdLayout bwd_layout(int64_t M, int64_t N, int64_t K) {
+  BwdLayout L;
+  L.ldm = (M + 3) / 4 * 4;
+  L.ones = 0;
+  L.partial = L.ones + round_up((size_t)K * 4, 256);
+  L.wt = L.partial + round_up((size_t)colsum_chunks(M) * (size_t)N * 4, 256);
+  L.dyt = L.wt + round_up((size_t)K * (size_t)N * 4, 256);
+  L.xt = L.dyt + round_up((size_t)N * (size_t)L.ldm * 4, 256);
+  L.total = L.xt + round_up((size_t)K * (size_t)L.ldm * 4, 256);
+  return L;
+}
+
+// y[r][c] = sum_j a[r][j] * b[c][j] on the float kind of the GEMM (no scale, bias or activation).
+int float_gemm_nt(const float* a, int64_t lda, const float* b, int64_t rows, int64_t cols, int64_t depth, const float* ones, float* y,
+                  int64_t ldy, cudaStream_t st) {
+  GemmParams p;
+  p.s_x = nullptr;
+  p.s_w = ones;
+  p.bias = nullptr;
+  p.residual = nullptr;
+  p.acc_debug = nullptr;
+  p.ldr = 0;
+  p.residual_scale = 0.0f;
+  p.s_x_kind = AQT_SCALE_TENSOR;
+  p.act = AQT_ACT_NONE;
+  p.M = (int)rows;
+  p.N = (int)cols;
+  p.K = (int)(4 * depth);
+  p.kind = 1;
+  p.a_pitch = 4 * lda;
+  p.n_out = (int)cols;
+  p.tiles_m = p.tiles_n = p.k_blocks = 0;
+  p.small_acc = 0;
+  return launch_qgemm(reinterpret_cast<const int8_t*>(a), b, false, y, ldy, p, st);
 }
 
 int validate_matmul_shape(int64_t M, int64_t N, int64_t K, int bits_a, int bits_w, int act, int s_x_kind) {
@@ -144,6 +186,7 @@ size_t aqt_workspace_bytes(int op, int64_t M, int64_t N, int64_t K, int bits_a, 
   if (op == AQT_OP_LINEAR_FWD) return ws_linear(M, N, K, bits_w);
   if (op == AQT_OP_LINEAR_WEIGHT_ONLY) return ws_weight_only(0, N, K, AQT_FLOAT_TF32);
   if (op == AQT_OP_LINEAR_WEIGHT_ONLY_X2) return ws_weight_only(M, N, K, AQT_FLOAT_TF32X2);
+  if (op == AQT_OP_LINEAR_BWD) return bwd_layout(M, N, K).total;
   if (op == AQT_OP_QMATMUL_REQUANT) return round_up(ws_qmatmul(M, N, K, bits_a, bits_w), 256) + requant_exchange_bytes(M, N);
   return 0;
 }
@@ -431,6 +474,57 @@ int aqt_linear_fwd_weight_only(const float* x, int64_t ldx, const void* wq, cons
   p.tiles_m = p.tiles_n = p.k_blocks = 0;
   p.small_acc = 0;
   return launch_qgemm(reinterpret_cast<const int8_t*>(a_f), w_f, false, y, ldy, p, st);
+}
+
+int aqt_linear_bwd(const float* dy, int64_t lddy, const void* xq, const float* s_x, int s_x_kind, int bits_a, const void* wq,
+                   const float* s_w, int bits_w, int64_t M, int64_t N, int64_t K, float* dx, int64_t lddx, float* dw, int64_t lddw,
+                   float* dbias, void* workspace, size_t workspace_bytes, void* stream) {
+  if (M < 0 || N < 0 || K <= 0 || !bits_ok(bits_a) || !bits_ok(bits_w)) return AQT_ERR_BADARG;
+  if (s_x_kind != AQT_SCALE_ROW && s_x_kind != AQT_SCALE_TENSOR) return AQT_ERR_BADARG;
+  if (K % 4 != 0 || N % 4 != 0) return AQT_ERR_BADARG;
+  if (M >= (1ll << 28) || N >= (1ll << 28) || K >= (1ll << 28) || M * N >= (1ll << 40)) return AQT_ERR_UNSUPPORTED;
+  if (M == 0 || N == 0) return AQT_OK;
+  if (dy == nullptr || lddy < N) return AQT_ERR_BADARG;
+  if (dx != nullptr && (wq == nullptr || s_w == nullptr || lddx < K)) return AQT_ERR_BADARG;
+  if (dw != nullptr && (xq == nullptr || s_x == nullptr || lddw < K)) return AQT_ERR_BADARG;
+  if (!is_aligned(dy, 16) || lddy % 4 != 0) return AQT_ERR_ALIGN;
+  if (dx != nullptr && (!is_aligned(dx, 16) || lddx % 4 != 0)) return AQT_ERR_ALIGN;
+  if (dw != nullptr && (!is_aligned(dw, 16) || lddw % 4 != 0)) return AQT_ERR_ALIGN;
+  if (dbias != nullptr && !is_aligned(dbias, 4)) return AQT_ERR_ALIGN;
+  const BwdLayout L = bwd_layout(M, N, K);
+  if (workspace == nullptr || workspace_bytes < L.total) return AQT_ERR_WORKSPACE;
+  if (!is_aligned(workspace, 256)) return AQT_ERR_ALIGN;
+  int rc = check_device();
+  if (rc != AQT_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  float* ones = reinterpret_cast<float*>(ws + L.ones);
+  rc = launch_fill_f32(ones, K, 1.0f, st);
+  if (rc != AQT_OK) return rc;
+  if (dbias != nullptr) {
+    rc = launch_colsum(dy, lddy, M, N, reinterpret_cast<float*>(ws + L.partial), dbias, st);
+    if (rc != AQT_OK) return rc;
+  }
+  if (dx != nullptr) {
+    // dx = dy . (s_w wq): rows m, columns k, contraction n
+    float* wt = reinterpret_cast<float*>(ws + L.wt);
+    rc = launch_transpose_scale_codes(wq, bits_w == 4, s_w, true, N, K, wt, N, st);
+    if (rc != AQT_OK) return rc;
+    rc = float_gemm_nt(dy, lddy, wt, M, K, N, ones, dx, lddx, st);
+    if (rc != AQT_OK) return rc;
+  }
+  if (dw != nullptr) {
+    // dw = dy^T . (s_x xq): rows n, columns k, contraction m (padded with zeros to a multiple of 4)
+    float* dyt = reinterpret_cast<float*>(ws + L.dyt);
+    float* xt = reinterpret_cast<float*>(ws + L.xt);
+    rc = launch_transpose_f32(dy, lddy, M, N, dyt, L.ldm, st);
+    if (rc != AQT_OK) return rc;
+    rc = launch_transpose_scale_codes(xq, bits_a == 4, s_x, s_x_kind == AQT_SCALE_ROW, M, K, xt, L.ldm, st);
+    if (rc != AQT_OK) return rc;
+    rc = float_gemm_nt(dyt, L.ldm, xt, N, K, L.ldm, ones, dw, lddw, st);
+    if (rc != AQT_OK) return rc;
+  }
+  return AQT_OK;
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -1097,7 +1097,9 @@ static int launch_qgemm(const int8_t* a, const void* b, bool b_packed, float* y,
     return deep_k ? launch_qgemm_cfg<128, 8, 4, false, false, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 6, 8, false, false, true>(a, b, y, ldy, p, st);
   }
   int bn = pick_bn(p.M, p.N, glu, sm_count() > 0 ? sm_count() : 148);
-  if (f32 && p.N >= 256) bn = 256;  // operand bytes per output are four times those of the 8-bit kind: the widest tile always wins
+  // operand bytes per output are four times those of the 8-bit kind: the widest tile wins whenever it
+  // still gives every SM a tile (a weight gradient has few, very deep tiles and takes narrow ones)
+  if (f32 && p.N >= 256 && ceil_div(p.M, kBM) * ceil_div(p.N, 256) >= sms_) bn = 256;
   // tuning aid: AQT_BN=64|128|256 in the environment overrides the tile-width heuristic
   static const char* force = getenv("AQT_BN");
   if (force != nullptr) {

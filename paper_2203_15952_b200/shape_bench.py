@@ -6,6 +6,7 @@
     python -m paper_2203_15952_b200.shape_bench quantize M K [--bits 4|8]
     python -m paper_2203_15952_b200.shape_bench linear M N K [--act ..] [--bits-w ..] [--bits 4|8] [--per-tensor]
     python -m paper_2203_15952_b200.shape_bench wonly M N K [--act ..] [--bits-w 4|8] [--residual] [--x2]
+    python -m paper_2203_15952_b200.shape_bench bwd M N K [--bits-w 4|8]
 
 Inputs are random codes / normals drawn on the GPU (seeded); several buffer sets are rotated so
 that consecutive launches do not find their inputs in L2.  With --sustain the call is repeated for
@@ -90,7 +91,7 @@ def _sustain(calls, seconds):
 
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("op", choices=["qmatmul", "requant", "quantize", "linear", "wonly"])
+    ap.add_argument("op", choices=["qmatmul", "requant", "quantize", "linear", "wonly", "bwd"])
     ap.add_argument("dims", type=int, nargs="+")
     ap.add_argument("--act", type=int, default=0)
     ap.add_argument("--bits-w", type=int, default=8)
@@ -174,6 +175,28 @@ def main(argv=None):
         ops = 2.0 * M * N * K
         nbytes = 4 * M * K + N * K * a.bits_w // 8 + 8 * N + 4 * M * n_out
         label = "linear M%d N%d K%d act%d a%d w%d %s" % (M, N, K, a.act, a.bits, a.bits_w, "per-tensor" if a.per_tensor else "per-row")
+    elif a.op == "bwd":
+        # straight-through backward: dx, dw and dbias of one layer from dy and the forward's codes
+        import ctypes
+        M, N, K = a.dims
+        wq = torch.randint(-7, 8, (N, K if a.bits_w == 8 else K // 2), generator=g, dtype=torch.int8, device=dev)
+        if a.bits_w == 4:
+            wq = wq.view(torch.uint8)
+        sw = torch.rand(N, generator=g, device=dev) * 1e-3
+        xq = torch.randint(-127, 128, (M, K), generator=g, dtype=torch.int8, device=dev)
+        sx = torch.rand(M, generator=g, device=dev) * 1e-2
+        ws = torch.empty(aqt.aqt_workspace_bytes(aqt.OP_LINEAR_BWD, M, N, K, 0, 0) + 256, dtype=torch.uint8, device=dev)
+        sets = [(torch.randn((M, N), generator=g, device=dev), torch.empty((M, K), device=dev), torch.empty((N, K), device=dev),
+                 torch.empty(N, device=dev)) for _ in range(a.sets)]
+
+        def make_calls(stream=None):
+            return [aqt.bind("aqt_linear_bwd", aqt._ptr(dy), aqt._i64(N), aqt._ptr(xq), aqt._ptr(sx), aqt.SCALE_ROW, 8, aqt._ptr(wq),
+                             aqt._ptr(sw), int(a.bits_w), aqt._i64(M), aqt._i64(N), aqt._i64(K), aqt._ptr(dx), aqt._i64(K), aqt._ptr(dw),
+                             aqt._i64(K), aqt._ptr(db), aqt._ptr(ws), ctypes.c_size_t(ws.numel()), aqt._stream(stream))
+                    for (dy, dx, dw, db) in sets]
+        ops = 4.0 * M * N * K
+        nbytes = 4 * M * N + M * K + N * K * a.bits_w // 8 + 4 * M * K + 4 * N * K + 4 * (M + 2 * N)
+        label = "bwd M%d N%d K%d w%d" % (M, N, K, a.bits_w)
     elif a.op == "wonly":
         # weight-only layer: fp32 activations against integer weights (float matmul, tf32 operands)
         M, N, K = a.dims
