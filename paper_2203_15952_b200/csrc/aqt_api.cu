@@ -44,27 +44,52 @@ size_t ws_weight_only(int64_t M, int64_t N, int64_t K, int precision) {
   return round_up((size_t)N * (size_t)K * 4, 256);
 }
 
-// Backward: [ones K | column-sum partials | s_w-scaled W^T [K, N] | dy^T [N, ldm] | s_x-scaled xq^T [K, ldm]], ldm = M rounded up to 4
+// Backward workspace: [ones K | column-sum partials | s_w-scaled W^T [K, N] | dy^T | s_x-scaled xq^T | dw partials].
+// The weight gradient is an [N, K] output with a contraction of M: few, very deep tiles.  Its
+// contraction is therefore cut into `batches` chunks of `chunk` rows (a multiple of 32), each
+// batch a matmul of its own in the same launch (GemmParams::batch_tiles_m), and the batches'
+// outputs are added in order.  The split is chosen for the 148 SMs of the one device this library
+// is built for, so that the layout (and aqt_workspace_bytes) needs no CUDA call.
 struct BwdLayout {
-  size_t ones, partial, wt, dyt, xt, total;
-  int64_t ldm;
+  size_t ones, partial, wt, dyt, xt, dwp, total;
+  int64_t batches, chunk, n_pad;  // batches == 1: chunk is the padded pitch of the transposed operands
 };
 BwdLayout bwd_layout(int64_t M, int64_t N, int64_t K) {
   BwdLayout L;
-  L.ldm = (M + 3) / 4 * 4;
+  L.n_pad = round_up((size_t)N, 128);
+  const int64_t tiles = (L.n_pad / 128) * ceil_div(K, 256);
+  int64_t batches = 148 / (tiles > 0 ? tiles : 1);
+  if (batches > M / 512) batches = M / 512;  // a batch should still be some k-blocks deep
+  if (batches < 2) {
+    L.batches = 1;
+    L.chunk = (M + 3) / 4 * 4;
+    L.n_pad = N;
+  } else {
+    L.chunk = round_up((size_t)ceil_div(M, batches), kTrRows);
+    L.batches = ceil_div(M, L.chunk);
+  }
   L.ones = 0;
   L.partial = L.ones + round_up((size_t)K * 4, 256);
-  L.wt = L.partial + round_up((size_t)colsum_chunks(M) * (size_t)N * 4, 256);
+  // column-sum partials: one row of N per 128-row block of the transpose (or per 2048-row chunk of the stand-alone sum)
+  L.wt = L.partial + round_up((size_t)(transpose_row_blocks(L.batches * L.chunk) + colsum_chunks(M)) * (size_t)N * 4, 256);
   L.dyt = L.wt + round_up((size_t)K * (size_t)N * 4, 256);
-  L.xt = L.dyt + round_up((size_t)N * (size_t)L.ldm * 4, 256);
-  L.total = L.xt + round_up((size_t)K * (size_t)L.ldm * 4, 256);
+  L.xt = L.dyt + round_up((size_t)L.batches * L.n_pad * L.chunk * 4, 256);
+  L.dwp = L.xt + round_up((size_t)L.batches * K * L.chunk * 4, 256);
+  L.total = L.dwp + (L.batches > 1 ? round_up((size_t)L.batches * L.n_pad * K * 4, 256) : 0);
   return L;
 }
 
 // y[r][c] = sum_j a[r][j] * b[c][j] on the float kind of the GEMM (no scale, bias or activation).
+// batches > 1: a holds `batches` stacked [rows / batches, depth] blocks, b as many stacked [cols, depth] blocks,
+// and y receives the stacked [rows / batches, cols] products.
 int float_gemm_nt(const float* a, int64_t lda, const float* b, int64_t rows, int64_t cols, int64_t depth, const float* ones, float* y,
-                  int64_t ldy, cudaStream_t st) {
+                  int64_t ldy, cudaStream_t st, int64_t batches = 1) {
   GemmParams p;
+  if (batches > 1) {
+    p.batch_tiles_m = (int)(rows / batches / kBM);  // rows per batch are a multiple of the tile height
+    p.batch_b_rows = (int)cols;
+    p.b_rows = batches * cols;
+  }
   p.s_x = nullptr;
   p.s_w = ones;
   p.bias = nullptr;
@@ -501,28 +526,38 @@ int aqt_linear_bwd(const float* dy, int64_t lddy, const void* xq, const float* s
   float* ones = reinterpret_cast<float*>(ws + L.ones);
   rc = launch_fill_f32(ones, K, 1.0f, st);
   if (rc != AQT_OK) return rc;
-  if (dbias != nullptr) {
+  if (dbias != nullptr && dw == nullptr) {  // with dw the column sums come out of the transpose of dy
     rc = launch_colsum(dy, lddy, M, N, reinterpret_cast<float*>(ws + L.partial), dbias, st);
     if (rc != AQT_OK) return rc;
   }
   if (dx != nullptr) {
     // dx = dy . (s_w wq): rows m, columns k, contraction n
     float* wt = reinterpret_cast<float*>(ws + L.wt);
-    rc = launch_transpose_scale_codes(wq, bits_w == 4, s_w, true, N, K, wt, N, st);
+    rc = launch_transpose_scale_codes(wq, bits_w == 4, s_w, true, N, K, wt, N, N, K, st);
     if (rc != AQT_OK) return rc;
     rc = float_gemm_nt(dy, lddy, wt, M, K, N, ones, dx, lddx, st);
     if (rc != AQT_OK) return rc;
   }
   if (dw != nullptr) {
-    // dw = dy^T . (s_x xq): rows n, columns k, contraction m (padded with zeros to a multiple of 4)
+    // dw = dy^T . (s_x xq): rows n, columns k, contraction m (padded with zeros), cut into L.batches chunks
     float* dyt = reinterpret_cast<float*>(ws + L.dyt);
     float* xt = reinterpret_cast<float*>(ws + L.xt);
-    rc = launch_transpose_f32(dy, lddy, M, N, dyt, L.ldm, st);
+    const int64_t m_pad = L.batches * L.chunk;
+    rc = launch_transpose_f32(dy, lddy, M, N, dyt, m_pad, L.chunk, L.n_pad, dbias != nullptr ? reinterpret_cast<float*>(ws + L.partial) : nullptr,
+                              dbias, st);
     if (rc != AQT_OK) return rc;
-    rc = launch_transpose_scale_codes(xq, bits_a == 4, s_x, s_x_kind == AQT_SCALE_ROW, M, K, xt, L.ldm, st);
+    rc = launch_transpose_scale_codes(xq, bits_a == 4, s_x, s_x_kind == AQT_SCALE_ROW, M, K, xt, m_pad, L.chunk, K, st);
     if (rc != AQT_OK) return rc;
-    rc = float_gemm_nt(dyt, L.ldm, xt, N, K, L.ldm, ones, dw, lddw, st);
-    if (rc != AQT_OK) return rc;
+    if (L.batches == 1) {
+      rc = float_gemm_nt(dyt, L.chunk, xt, N, K, L.chunk, ones, dw, lddw, st);
+      if (rc != AQT_OK) return rc;
+    } else {
+      float* dwp = reinterpret_cast<float*>(ws + L.dwp);
+      rc = float_gemm_nt(dyt, L.chunk, xt, L.batches * L.n_pad, K, L.chunk, ones, dwp, K, st, L.batches);
+      if (rc != AQT_OK) return rc;
+      rc = launch_sum_batches(dwp, L.batches, L.n_pad, N, K, dw, lddw, st);
+      if (rc != AQT_OK) return rc;
+    }
   }
   return AQT_OK;
 }

@@ -82,6 +82,13 @@ struct GemmParams {
   int M, N, K;  // K: bytes of contraction per operand row (= elements for 8-bit codes, 4 x elements for the float kind)
   int kind = 0;       // 0: signed 8-bit codes, int32 accumulators; 1: binary32 operands used as tf32, binary32 accumulators
   int64_t a_pitch = 0;  // bytes between rows of A; 0 = dense (K)
+  // Batched form (streaming kernel, one CTA per tile): every batch_tiles_m consecutive m-tiles form
+  // one batch with its own block of batch_b_rows rows of B, stacked below one another (b_rows rows
+  // in all; 0 = N).  Used to split a very deep contraction over CTAs: batch s holds the s-th
+  // chunk of the contraction of both operands, and the batches' outputs are added afterwards.
+  int batch_tiles_m = 0;
+  int batch_b_rows = 0;
+  int64_t b_rows = 0;
   int n_out;    // N, or N / 2 for the GLU forms
   int tiles_m, tiles_n, k_blocks;
   int small_acc;  // every |accumulator| < 2^22: the int -> float conversion can use the exponent trick
@@ -561,8 +568,9 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
           tma_load_2d(stage, &tm_a, kb * kBK, tm * kBM, bar);
           if (!WS) {
-            tma_load_2d(stage + Cfg::kABytes, &tm_b, kb * kBK, row0, bar);
-            tma_load_2d(stage + Cfg::kABytes + HALF * kBK, &tm_b, kb * kBK, row1, bar);
+            const int b_batch = p.batch_tiles_m > 0 ? (tm / p.batch_tiles_m) * p.batch_b_rows : 0;  // this batch's rows of B
+            tma_load_2d(stage + Cfg::kABytes, &tm_b, kb * kBK, row0 + b_batch, bar);
+            tma_load_2d(stage + Cfg::kABytes + HALF * kBK, &tm_b, kb * kBK, row1 + b_batch, bar);
           }
         }
       }
@@ -988,9 +996,11 @@ static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t l
   if (BPACK) {
     rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, b, (uint64_t)p.N, (uint64_t)p.K / 2, (uint64_t)p.K / 2, BN / 2, 64, 0);
   } else {
-    rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, b, (uint64_t)p.N, (uint64_t)p.K, (uint64_t)p.K, BN / 2, kBK);
+    rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, b, (uint64_t)(p.b_rows != 0 ? p.b_rows : p.N), (uint64_t)p.K, (uint64_t)p.K, BN / 2,
+                     kBK);
   }
   if (rc != AQT_OK) return rc;
+  if (p.batch_tiles_m > 0 && (WS || CTA2)) return AQT_ERR_UNSUPPORTED;
   rc = make_map_2d(&tm_y, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, y, (uint64_t)p.M, (uint64_t)p.n_out, (uint64_t)ldy * 4, kStoreBoxRows,
                    kStoreBoxCols);
   if (rc != AQT_OK) return rc;
@@ -1058,7 +1068,8 @@ static bool qgemm_uses_ws(int64_t N, int64_t K) {
 // packed nibbles [N, K/2].  All dense, 16-byte aligned.
 static int launch_qgemm(const int8_t* a, const void* b, bool b_packed, float* y, int64_t ldy, const GemmParams& p, cudaStream_t st) {
   const bool glu = (p.act == AQT_ACT_GLU) || (p.act == AQT_ACT_GLU_SWISH);
-  if (qgemm_uses_ws(p.N, p.K)) {
+  const bool batched = p.batch_tiles_m > 0;  // streaming kernel, one CTA per tile
+  if (!batched && qgemm_uses_ws(p.N, p.K)) {
     // tile width 128; a GLU tile has 64 output columns, i.e. two chunks per lane quadrant
     if (glu) return b_packed ? launch_qgemm_cfg<128, 6, 8, true, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 6, 8, true, false>(a, b, y, ldy, p, st);
     return b_packed ? launch_qgemm_cfg<128, 6, 16, true, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 6, 16, true, false>(a, b, y, ldy, p, st);
@@ -1084,7 +1095,7 @@ static int launch_qgemm(const int8_t* a, const void* b, bool b_packed, float* y,
   const bool two_rounds_of_pairs = !glu && ceil_div(p.M, 2 * kBM) * ceil_div(p.N, 256) >= 2 * (sms_ / 2);
   // (float kind, measured: pairs win 6-10 % at M >= 25 600, lose 10 % at 12 800 x 2048 x 512)
   const bool pairs_ok = f32 ? (two_rounds_of_pairs && p.M >= 2 * kBM * (sms_ / 2)) : (deep_k || (p.K >= 2048 && two_rounds_of_pairs));
-  if (no_pairs == nullptr && (pairs_ok || getenv("AQT_FORCE_PAIRS") != nullptr) && p.M > kBM) {
+  if (!batched && no_pairs == nullptr && (pairs_ok || getenv("AQT_FORCE_PAIRS") != nullptr) && p.M > kBM) {
     // CTA pairs on 256-row tiles; width by the number of rounds over the pairs
     const int pairs = (sm_count() > 0 ? sm_count() : 148) / 2;
     const int64_t tiles_m2 = ceil_div(p.M, 2 * kBM);
