@@ -440,6 +440,7 @@ def run_ours(args):
     if world == 1 and not args.no_encoder:
         line["encoder"] = encoder_frames_per_s(dev)
         line["weight_only"] = weight_only_ffn_pair(dev)
+        line["backward"] = backward_ffn_layer(dev)
         line["encoder_large"] = encoder_frames_per_s(dev, steps=2, cfg=5)  # last: seconds of dense work that pull the clocks down
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline()
@@ -554,6 +555,54 @@ def weight_only_ffn_pair(dev, steps: int = 20):
             "frames_per_s": M / (ms * 1e-3), "dtype": "tf32", "gpu_launches_per_step": 4, "launch_mode": "cuda graph",
             "roofline": {"bound": "tensor", "achieved": tflops, "peak": peak, "unit": "TFLOP/s", "frac": tflops / peak,
                          "peak_source": "bf16 burst of %s x nominal tf32 : bf16 ratio 1/2" % kind, "traffic": None}}
+
+
+def backward_ffn_layer(dev, steps: int = 20):
+    """Straight-through backward (dx, dw, dbias) of the pair's first layer (M = 12 800, 512 -> 2048,
+    int4 weights, int8 activation codes) through aqt_linear_bwd, replayed from a CUDA graph over
+    rotating gradient buffers; 2 * 2 * M * N * K flops per call on the tensor cores' tf32 kind."""
+    import ctypes
+    import torch
+    from paper_2203_15952_b200 import binding as aqt
+    from paper_2203_15952_b200 import inputs as gen
+    w = gen.WORKLOADS[CFG]
+    s0 = gen.workload_layers(w)[0]
+    M, N, K = w.M, s0.N, s0.K
+    g = torch.Generator(device=dev).manual_seed(6)
+    wq = torch.randint(-7, 8, (N, K // 2), generator=g, dtype=torch.int8, device=dev).view(torch.uint8)
+    sw = torch.rand(N, generator=g, device=dev) * 1e-3
+    xq = torch.randint(-127, 128, (M, K), generator=g, dtype=torch.int8, device=dev)
+    sx = torch.rand(M, generator=g, device=dev) * 1e-2
+    ws = torch.empty(aqt.aqt_workspace_bytes(aqt.OP_LINEAR_BWD, M, N, K, 0, 0) + 256, dtype=torch.uint8, device=dev)
+    R = 3
+    sets = [(torch.randn((M, N), generator=g, device=dev), torch.empty((M, K), device=dev), torch.empty((N, K), device=dev),
+             torch.empty(N, device=dev)) for _ in range(R)]
+    stream = torch.cuda.current_stream()
+    side = torch.cuda.Stream()
+    side.wait_stream(stream)
+    with torch.cuda.stream(side):
+        calls = [aqt.bind("aqt_linear_bwd", aqt._ptr(dy), aqt._i64(N), aqt._ptr(xq), aqt._ptr(sx), aqt.SCALE_ROW, 8, aqt._ptr(wq),
+                          aqt._ptr(sw), 4, aqt._i64(M), aqt._i64(N), aqt._i64(K), aqt._ptr(dx), aqt._i64(K), aqt._ptr(dw), aqt._i64(K),
+                          aqt._ptr(db), aqt._ptr(ws), ctypes.c_size_t(ws.numel()), aqt._stream(side)) for (dy, dx, dw, db) in sets]
+        for c in calls:
+            c()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        for c in calls:
+            c()
+    graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        graph.replay()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / (steps * R)
+    tflops = 4.0 * M * N * K / (ms * 1e-3) / 1e12
+    return {"workload": "ffn_first_layer_M%d_N%d_K%d_w4a8_dx_dw_dbias" % (M, N, K), "value": tflops, "unit": "TFLOP/s", "ms_per_step": ms,
+            "dtype": "tf32", "gpu_launches_per_step": 9, "launch_mode": "cuda graph"}
 
 
 def main():
