@@ -171,6 +171,25 @@ def test_weight_only_full_size_ffn_layer_sampled_rows():
     assert np.all(np.abs(y.cpu().numpy()[rows].astype(np.float64) - y_ref) <= tol)
 
 
+@pytest.mark.parametrize("N,K,act,residual", [(512, 512, orc.ACT_NONE, True), (512, 2048, orc.ACT_NONE, False), (1024, 256, orc.ACT_SWISH, False)])
+def test_weight_only_many_rows_take_cta_pairs(N, K, act, residual):
+    """M = 19 072 rows: from 18 944 rows on (two rounds of 256-row tiles over the SM pairs) the
+    float kind runs on CTA pairs, with the eight-warp or (deep K, no activation) four-warp
+    epilogue.  Sampled rows against the oracle."""
+    M = 19072
+    x = gen.normal(9, 17, M, K)
+    wq, s_w, w_dev = _weights(9, N, K, 4)
+    res = gen.normal(9, 23, M, N) if residual else None
+    y = aqt.aqt_linear_fwd_weight_only(_dev(x), _dev(w_dev), _dev(s_w), None, None if res is None else _dev(res), 0.5, bits_w=4, act=act)
+    assert aqt.aqt_device_status() == 0
+    rows = np.unique(np.concatenate([np.arange(0, 260), np.arange(M - 260, M), np.random.default_rng(2).integers(0, M, 200)]))
+    y_ref, z, mag = orc.linear_weight_only_f64(x[rows], wq, s_w, residual=None if res is None else res[rows], residual_scale=0.5, act=act,
+                                               return_parts=True)
+    dz = (2.0 ** -10 + K * 2.0 ** -24) * mag + 2.0 ** -23 * np.abs(z)
+    tol = _bound_out(act, z, dz, 0.5, residual, y_ref)
+    assert np.all(np.abs(y.cpu().numpy()[rows].astype(np.float64) - y_ref) <= tol)
+
+
 def test_weight_only_argument_errors():
     L = aqt.lib()
     i64, vp, f = ctypes.c_int64, ctypes.c_void_p, ctypes.c_float(1.0)
