@@ -1104,8 +1104,14 @@ static int launch_qgemm(const int8_t* a, const void* b, bool b_packed, float* y,
     int bn2 = cost256 <= cost128 ? 256 : 128;
     static const char* force2 = getenv("AQT_BN");
     if (force2 != nullptr && (atoi(force2) == 128 || atoi(force2) == 256)) bn2 = atoi(force2);
-    if (bn2 == 256) return deep_k ? launch_qgemm_cfg<256, 6, 4, false, false, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<256, 4, 8, false, false, true>(a, b, y, ldy, p, st);
-    return deep_k ? launch_qgemm_cfg<128, 8, 4, false, false, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 6, 8, false, false, true>(a, b, y, ldy, p, st);
+    // The four-warp epilogue / deeper ring pays off for pairs only from K = 4096 bytes (measured at
+    // 65 536 x 1024 x 4096: 2753 vs 2671 TOPS burst, equal sustained; float kind 801 vs 752
+    // TFLOP/s); at K = 2048 the eight-warp epilogue with four stages is 20-27 % faster (41.1 vs
+    // 52.3 us at 37 888 x 512 x 2048, where the deep-K rule first applies; 83.1 vs 104.9 us at 65 536).
+    static const char* deep_pairs = getenv("AQT_DEEP_PAIRS");  // tuning aid: 0 / 1 overrides the choice
+    const bool dp = deep_pairs != nullptr ? atoi(deep_pairs) != 0 : (deep_k && p.K >= 4096);
+    if (bn2 == 256) return dp ? launch_qgemm_cfg<256, 6, 4, false, false, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<256, 4, 8, false, false, true>(a, b, y, ldy, p, st);
+    return dp ? launch_qgemm_cfg<128, 8, 4, false, false, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 6, 8, false, false, true>(a, b, y, ldy, p, st);
   }
   int bn = pick_bn(p.M, p.N, glu, sm_count() > 0 ? sm_count() : 148);
   // operand bytes per output are four times those of the 8-bit kind: the widest tile wins whenever it
