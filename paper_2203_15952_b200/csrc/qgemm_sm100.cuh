@@ -108,14 +108,19 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// One attempt.  The thread may stay suspended in the instruction for up to kTryWaitSuspendNs while
+// the phase is incomplete (it resumes at once when the phase completes), so a waiting warp costs
+// its scheduler a handful of instructions per 100 us instead of a spin loop's worth: the producer,
+// the MMA issuer and the exchange warp share their schedulers with the epilogue warps.
+constexpr uint32_t kTryWaitSuspendNs = 100000u;
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t done;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(done)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(kTryWaitSuspendNs)
       : "memory");
   return done != 0;
 }
@@ -126,7 +131,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
                                           uint64_t limit_ns = kWaitLimitNs) {
   for (uint32_t spin = 1;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((spin & 0xFF) == 0) {
+    if ((spin & 0x3) == 0) {  // an attempt can last kTryWaitSuspendNs: look at the clock every few
       if (*abort_flag) return false;
       if (global_timer_ns() - t_start > limit_ns) {
         *abort_flag = 1;
