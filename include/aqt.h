@@ -32,7 +32,7 @@
 extern "C" {
 #endif
 
-#define AQT_VERSION 105
+#define AQT_VERSION 106
 
 /* status codes */
 #define AQT_OK 0
