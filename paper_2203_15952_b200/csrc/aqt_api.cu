@@ -516,6 +516,7 @@ int aqt_linear_bwd(const float* dy, int64_t lddy, const void* xq, const float* s
   if (dx != nullptr && (!is_aligned(dx, 16) || lddx % 4 != 0)) return AQT_ERR_ALIGN;
   if (dw != nullptr && (!is_aligned(dw, 16) || lddw % 4 != 0)) return AQT_ERR_ALIGN;
   if (dbias != nullptr && !is_aligned(dbias, 4)) return AQT_ERR_ALIGN;
+  if ((dx != nullptr && !is_aligned(wq, 16)) || (dw != nullptr && !is_aligned(xq, 16))) return AQT_ERR_ALIGN;
   const BwdLayout L = bwd_layout(M, N, K);
   if (workspace == nullptr || workspace_bytes < L.total) return AQT_ERR_WORKSPACE;
   if (!is_aligned(workspace, 256)) return AQT_ERR_ALIGN;

@@ -11,6 +11,7 @@
 #pragma once
 
 #include "aqt_common.cuh"
+#include "pack.cuh"
 
 namespace aqt {
 
@@ -36,21 +37,31 @@ __global__ void __launch_bounds__(256) transpose_scale_codes_kernel(const uint8_
   __shared__ float tile[kTrRows][kTrTile + 1];
   const int64_t r0 = (int64_t)blockIdx.y * kTrRows, c0 = (int64_t)blockIdx.x * kTrTile;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;  // 32 x 8
-#pragma unroll 4
-  for (int i = ty; i < kTrRows; i += 8) {
-    const int64_t r = r0 + i, c = c0 + tx;
-    float v = 0.0f;
+  // load: four codes (one 32-bit word, or two packed bytes) per thread and step; eight threads cover a row of the tile
+#pragma unroll
+  for (int j = 0; j < kTrRows * kTrTile / 4 / 256; ++j) {
+    const int w = threadIdx.x + 256 * j;
+    const int i = w >> 3, cw = w & 7;
+    const int64_t r = r0 + i, c = c0 + 4 * cw;  // C is a multiple of 4, so a word is inside the row or outside it
+    float v0 = 0.0f, v1 = 0.0f, v2 = 0.0f, v3 = 0.0f;
     if (r < R && c < C) {
-      int code;
+      uint32_t word;
       if (packed) {
-        const uint32_t b = codes[r * (C / 2) + (c >> 1)];
-        code = (c & 1) ? ((int)(b << 24) >> 28) : ((int)(b << 28) >> 28);
+        uint32_t hi;
+        unpack_word((uint32_t)__ldg(reinterpret_cast<const uint16_t*>(codes + r * (C / 2) + (c >> 1))), word, hi);
       } else {
-        code = (int)(int8_t)codes[r * C + c];
+        word = __ldg(reinterpret_cast<const uint32_t*>(codes + r * C + c));
       }
-      v = __fmul_rn(__ldg(scale + (per_row ? r : 0)), (float)code);
+      const float sc = __ldg(scale + (per_row ? r : 0));
+      v0 = __fmul_rn(sc, (float)(int8_t)(word & 0xFF));
+      v1 = __fmul_rn(sc, (float)(int8_t)((word >> 8) & 0xFF));
+      v2 = __fmul_rn(sc, (float)(int8_t)((word >> 16) & 0xFF));
+      v3 = __fmul_rn(sc, (float)(int8_t)(word >> 24));
     }
-    tile[i][tx] = v;
+    tile[i][4 * cw + 0] = v0;
+    tile[i][4 * cw + 1] = v1;
+    tile[i][4 * cw + 2] = v2;
+    tile[i][4 * cw + 3] = v3;
   }
   __syncthreads();
   const int64_t s0 = r0 / chunk, in_chunk = r0 - s0 * chunk;  // the tile's chunk and its first row inside it
