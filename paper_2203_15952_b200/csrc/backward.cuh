@@ -150,11 +150,22 @@ __global__ void __launch_bounds__(256) colsum_stage1_kernel(const float* __restr
 }
 __global__ void __launch_bounds__(256) colsum_stage2_kernel(const float* __restrict__ partial, int64_t chunks, int64_t C,
                                                             float* __restrict__ out) {
-  const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= C) return;
+  // 32 columns per block; thread (tx, ty) adds the chunks j = ty, ty + 8, ... of column tx in order,
+  // then the eight sums of a column are added in order: a fixed grouping, the same bits on every run
+  __shared__ float acc[8][kTrTile];
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int64_t c = (int64_t)blockIdx.x * kTrTile + tx;
   float t = 0.0f;
-  for (int64_t j = 0; j < chunks; ++j) t = __fadd_rn(t, partial[j * C + c]);
-  out[c] = t;
+  if (c < C)
+    for (int64_t j = ty; j < chunks; j += 8) t = __fadd_rn(t, __ldg(partial + j * C + c));
+  acc[ty][tx] = t;
+  __syncthreads();
+  if (ty == 0 && c < C) {
+    float u = acc[0][tx];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) u = __fadd_rn(u, acc[i][tx]);
+    out[c] = u;
+  }
 }
 
 __global__ void __launch_bounds__(256) fill_f32_kernel(float* __restrict__ p, int64_t n, float v) {
@@ -194,11 +205,11 @@ static int launch_colsum(const float* x, int64_t ldx, int64_t R, int64_t C, floa
   colsum_stage1_kernel<<<dim3((unsigned)ceil_div(C, kTrTile), (unsigned)chunks), 256, 0, st>>>(x, ldx, R, C, partial);
   int rc = AQT_LAUNCH_STATUS();
   if (rc != AQT_OK) return rc;
-  colsum_stage2_kernel<<<(unsigned)ceil_div(C, 256), 256, 0, st>>>(partial, chunks, C, out);
+  colsum_stage2_kernel<<<(unsigned)ceil_div(C, kTrTile), 256, 0, st>>>(partial, chunks, C, out);
   return AQT_LAUNCH_STATUS();
 }
 static int launch_colsum_stage2(const float* partial, int64_t chunks, int64_t C, float* out, cudaStream_t st) {
-  colsum_stage2_kernel<<<(unsigned)ceil_div(C, 256), 256, 0, st>>>(partial, chunks, C, out);
+  colsum_stage2_kernel<<<(unsigned)ceil_div(C, kTrTile), 256, 0, st>>>(partial, chunks, C, out);
   return AQT_LAUNCH_STATUS();
 }
 static int launch_fill_f32(float* p, int64_t n, float v, cudaStream_t st) {
