@@ -56,12 +56,19 @@ struct GemmCfg {
   static constexpr int kTmemCols = 2 * BN;  // two accumulator buffers; a power of two >= 32
   // Output staging buffers per warp: two let a warp fill one while the bulk store of the other is
   // still being read; with sixteen warps each warp stores once per tile and one is enough.
-  static constexpr int kStageBufs = (EW == 16) ? 1 : 2;
+  // "Lean" epilogue: where the ring, two staging buffers per warp and the scale slabs together
+  // would not fit (a fourth ring stage bought with eight epilogue warps), a warp keeps one staging
+  // buffer and reads scales and biases through L1.  A load takes about 2200 clocks from issue to
+  // arrival, so the ring depth sets the k-block rate: three stages give 705 clocks per k-block
+  // against 554 of MMA time, four give the MMA rate.
+  static constexpr bool kLean = !WS && EW == 8 &&
+                                STAGES * kStageBytes + EW * 2 * kStageBufBytes + EW * 2 * (BN / (EW / 4)) * 4 + 1024 + 512 > 232448;
+  static constexpr int kStageBufs = (EW == 16 || kLean) ? 1 : 2;
   static constexpr int kEpiBytes = EW * kStageBufs * kStageBufBytes;
   // Scales and biases of the tile's columns in shared memory: one slab per CTA when the n-tile is
   // fixed (WS), one per warp (its own columns) with EW >= 8 otherwise; with EW == 4 they are read
   // through L1 instead (the epilogue is a small part of a deep-K tile).
-  static constexpr bool kScaleSlab = WS || (EW >= 8);
+  static constexpr bool kScaleSlab = WS || (EW >= 8 && !kLean);
   static constexpr int kSlabFloats = WS ? BN : BN / (EW / 4);  // per array (s_w, bias)
   static constexpr int kScaleBytes = !kScaleSlab ? 0 : (WS ? 2 * BN * 4 : EW * 2 * kSlabFloats * 4);
   static constexpr int kSmemBytes = STAGES * kStageBytes + kResidentBytes + kEpiBytes + kScaleBytes + 1024;  // + alignment slack
@@ -1130,6 +1137,12 @@ static int launch_qgemm(const int8_t* a, const void* b, bool b_packed, float* y,
   }
   // Deep K: operand loads bound the tile, so the ring gets the shared memory and four warps run
   // the (short) epilogue.  Shallow K: the epilogue bounds the tile and gets more warps.
+  // Float kind: a tile's MMA time is four times that of the 8-bit kind for the same epilogue, so
+  // eight epilogue warps keep up and the shared memory they free buys the fourth ring stage
+  // (measured 2-10 % faster than three stages / sixteen warps and than four stages / four warps:
+  // 59.8 vs 62.4 us at 12 800 x 2048 x 512 Swish, 362 vs 398 us at 65 536 x 2048 x 1024 GLU).  The
+  // 8-bit kind loses with it wherever the epilogue evaluates an activation or M is small.
+  if (bn == 256 && f32) return launch_qgemm_cfg<256, 4, 8, false, false>(a, b, y, ldy, p, st);
   if (bn == 256) return deep_k ? launch_qgemm_cfg<256, 4, 4, false, false>(a, b, y, ldy, p, st) : launch_qgemm_cfg<256, 3, 16, false, false>(a, b, y, ldy, p, st);
   // every epilogue warp needs at least one 32-column chunk: a GLU tile of width 128 has only
   // 64 output columns, i.e. two chunks per lane quadrant
