@@ -77,3 +77,28 @@ def test_argument_errors_are_reported_before_any_cuda_call():
     assert mm(128, 256, 128, 8, 4, 0) == -4               # int4 weights need workspace
     assert mm(128, 256, 128, 8, 4, 0, ws=vp(256), wsb=100) == -4
     assert mm(1 << 31, 256, 128, 8, 8, 0) == -3
+
+
+def test_argument_errors_of_the_float_entry_points_need_no_device():
+    """The weight-only layer and the backward report bad arguments before any CUDA call too."""
+    L = ctypes.CDLL(aqt_build.build())
+    i64, vp, f = ctypes.c_int64, ctypes.c_void_p, ctypes.c_float(1.0)
+    one = vp(256)
+
+    def wo(M, N, K, bits_w=8, prec=0, act=0, ldx=None, ws=one, wsb=1 << 40):
+        return L.aqt_linear_fwd_weight_only(one, i64(K if ldx is None else ldx), one, one, None, None, i64(0), f, i64(M), i64(N), i64(K),
+                                            bits_w, prec, act, one, i64(N), ws, ctypes.c_size_t(wsb), None)
+    assert wo(128, 256, 130) == -1 and wo(128, 250, 128) == -1 and wo(128, 256, 128, bits_w=3) == -1
+    assert wo(128, 256, 128, prec=7) == -1 and wo(128, 256, 128, act=9) == -1
+    assert wo(128, 256, 128, ldx=130) == -2 and wo(128, 256, 128, ws=None) == -4 and wo(0, 256, 128) == 0
+
+    def bwd(M, N, K, kind=0, lddy=None, ws=one, wsb=1 << 40, xq=one):
+        return L.aqt_linear_bwd(one, i64(N if lddy is None else lddy), xq, one, kind, 8, one, one, 4, i64(M), i64(N), i64(K), one, i64(K),
+                                one, i64(K), None, ws, ctypes.c_size_t(wsb), None)
+    assert bwd(128, 256, 130) == -1 and bwd(128, 250, 128) == -1 and bwd(128, 256, 128, kind=2) == -1
+    assert bwd(128, 256, 128, lddy=258) == -2 and bwd(128, 256, 128, xq=None) == -1
+    assert bwd(128, 256, 128, ws=None) == -4 and bwd(128, 256, 128, wsb=10) == -4 and bwd(0, 256, 128) == 0
+    L.aqt_workspace_bytes.restype = ctypes.c_size_t
+    assert L.aqt_workspace_bytes(4, i64(128), i64(256), i64(128), 0, 4) == 4 * 256 * 128
+    assert L.aqt_workspace_bytes(5, i64(128), i64(256), i64(128), 0, 4) == 8 * 256 * 128 + 8 * 128 * 128
+    assert L.aqt_workspace_bytes(6, i64(12800), i64(2048), i64(512), 0, 0) > 4 * (512 * 2048 + (2048 + 512) * 12800)
