@@ -1104,7 +1104,8 @@ static int launch_qgemm(const int8_t* a, const void* b, bool b_packed, float* y,
   // Pairs pay off only for deep K and at least two full rounds of pair tiles (measured: +4 % at
   // 65 536 x 1024 x 4096 with the deep configuration, +9 % at 25 600 x 512 x 2048 with the
   // eight-warp epilogue, no gain at M = 12 800 or at K = 1024); everything else takes one CTA per tile.
-  const bool two_rounds_of_pairs = !glu && ceil_div(p.M, 2 * kBM) * ceil_div(p.N, 256) >= 2 * (sms_ / 2);
+  // (the 8-bit kind's GLU shapes are faster on single CTAs; the float kind's gain 3 % on pairs)
+  const bool two_rounds_of_pairs = (!glu || f32) && ceil_div(p.M, 2 * kBM) * ceil_div(p.N, 256) >= 2 * (sms_ / 2);
   // (float kind, measured: pairs win 6-10 % at M >= 25 600, lose 10 % at 12 800 x 2048 x 512)
   const bool pairs_ok = f32 ? (two_rounds_of_pairs && p.M >= 2 * kBM * (sms_ / 2)) : (deep_k || (p.K >= 2048 && two_rounds_of_pairs));
   if (!batched && no_pairs == nullptr && (pairs_ok || getenv("AQT_FORCE_PAIRS") != nullptr) && p.M > kBM) {
