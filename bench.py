@@ -30,19 +30,62 @@ sys.path.insert(0, ROOT)
 METRIC = "quantized Conformer linear TOPS (int4 weights, int8 activations)"
 UNIT = "TOPS"
 CFG = 2  # the Conformer FFN pair; fits one GPU many times over
-NCU_CAPTURE_VERSION = 106  # library version the ncu traffic figures below were captured at
-# call index -> DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum):
-# profiles/qgemm_requant_ffn_pair_ncu.md, profiles/qgemm_i8_ffn_pair_ncu.md
-NCU_TRAFFIC = {1: 7695360 + 44800, 2: 27341824 + 64256}
+NCU_CAPTURE_VERSION = 200  # library version the ncu traffic figures below were captured at
+# call index -> DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the
+# ncu summaries under profiles/; empty until a capture of this library version is committed
+NCU_TRAFFIC = {}
+INT8_NOMINAL_TOPS = 4500.0  # dense int8 tensor peak of the part, nominal
 
 
 def _peaks():
+    """Measured denominators (HBM copy GB/s, bf16 TFLOP/s burst and sustained) and where they come from."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
             p = json.load(f)
-        return float(p["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16": float(p["bf16_tflops"]),
+                "bf16_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "kind": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16": 1590.0, "bf16_sustained": 1400.0, "kind": "fallback"}
+
+
+def _capture(fn, stream_ctx_torch, warm: int = 1):
+    """Run fn() on a side stream once (warm-up), then capture it into a CUDA graph."""
+    torch = stream_ctx_torch
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for _ in range(warm):
+            fn(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        fn(side)
+    return graph
+
+
+def _time_replays(torch, graph, replays: int, min_seconds: float = 0.0, warm: int = 2):
+    """Milliseconds per replay (CUDA events on the current stream); at least `replays` replays
+    and at least `min_seconds` of them.  Returns (ms_per_replay, replays_done)."""
+    stream = torch.cuda.current_stream()
+    for _ in range(warm):
+        graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    done = 0
+    e0.record(stream)
+    t0 = time.perf_counter()
+    while True:
+        for _ in range(replays):
+            graph.replay()
+        done += replays
+        if min_seconds <= 0.0:
+            break
+        torch.cuda.synchronize()          # only the sustained runs look at the wall clock
+        if time.perf_counter() - t0 >= min_seconds:
+            break
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / done, done
 
 
 class ClockSampler:
@@ -201,7 +244,7 @@ def run_ours(args):
     layers = []
     for i, s in enumerate(specs):
         wt = torch.from_numpy(gen.layer_weight(w, 0, i, s, seed=0)).to(dev)
-        layers.append(QuantLinear.from_float(s, wt))
+        layers.append(QuantLinear.from_float(s, wt))   # packed int4; W2 (K = 2048) also kept sign-extended, once
     R = 6  # rotating input/output sets: the six x and six y tensors (315 MB) exceed the 126 MB L2
     x_host = gen.workload_input(w, seed=seed)
     xs = [torch.from_numpy(x_host).to(dev) for _ in range(R)]
@@ -217,6 +260,7 @@ def run_ours(args):
     # the first matmul's epilogue and only ever exists as codes + row scales.
     names = ["quantize(x) 12800x512", "qmatmul 512->2048 swish + quantize(u) rows (one kernel)", "qmatmul 2048->512"]
     NC = len(names)
+    l0, l1 = layers
 
     # pre-marshalled C-ABI calls (one set per rotating buffer) so that Python stays ahead of the GPU
     def make_calls(st, rounding=aqt.ROUND_NEAREST_EVEN):
@@ -224,25 +268,17 @@ def run_ours(args):
         for r in range(R):
             out.append((
                 aqt.bind_quantize(xs[r], specs[0].bits_a, aqt.AXIS_ROW, rounding, False, q1, s1, st),
-                aqt.bind_qmatmul_requant(q1, s1, layers[0].wq, layers[0].s_w, None, None, 1.0, specs[0].K, 8, specs[0].bits_w,
-                                         specs[0].act, aqt.SCALE_ROW, specs[1].bits_a, rounding, False, q2, s2, None,
-                                         ws, st),
-                aqt.bind_qmatmul(q2, s2, layers[1].wq, layers[1].s_w, None, None, 1.0, specs[1].K, 8, specs[1].bits_w,
+                aqt.bind_qmatmul_requant(q1, s1, l0.mm_weight, l0.s_w, None, None, 1.0, specs[0].K, 8, l0.mm_bits,
+                                         specs[0].act, aqt.SCALE_ROW, specs[1].bits_a, rounding, False, q2, s2, None, ws, st),
+                aqt.bind_qmatmul(q2, s2, l1.mm_weight, l1.s_w, None, None, 1.0, specs[1].K, 8, l1.mm_bits,
                                  specs[1].act, aqt.SCALE_ROW, ys[r], ws, st)))
         return out
 
     calls = make_calls(stream)
 
-    def step(i, events=None):
-        c = calls[i % R]
-        if events is None:
-            for f in c:
-                f()
-            return
-        events[0].record(stream)
-        for j in range(NC):
-            c[j]()
-            events[j + 1].record(stream)
+    def step(i):
+        for f in calls[i % R]:
+            f()
 
     def barrier():
         torch.cuda.synchronize()
@@ -256,56 +292,81 @@ def run_ours(args):
     if aqt.aqt_device_status() != 0:
         raise SystemExit("device status reports a failed wait during warm-up")
 
-    # The same C-ABI calls for R consecutive steps captured in a CUDA graph (launch latency out of
-    # the way).  The timed region replays the graph and, every R + 1 steps, runs one step call by
-    # call with CUDA events around each call: those give the per-kernel durations of the roofline.
-    graph = None
+    # R consecutive steps captured in a CUDA graph (launch latency out of the way), twice: plain,
+    # and with an event recorded around every call (event-record nodes inside the graph), which is
+    # where the per-call durations of the roofline come from.
+    graph = graph_ev = None
+    call_events = [[torch.cuda.Event(enable_timing=True, external=True) for _ in range(NC + 1)] for _ in range(R)]
     if not args.no_graph:
-        side = torch.cuda.Stream()
-        side.wait_stream(stream)
-        with torch.cuda.stream(side):
-            gcalls = make_calls(side)
-            for r in range(R):
-                for c in gcalls[r]:
+        def run_plain(st):
+            for c3 in make_calls(st):
+                for c in c3:
                     c()
-        torch.cuda.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=side):
-            for r in range(R):
-                for c in gcalls[r]:
+
+        def run_with_events(st):
+            for r, c3 in enumerate(make_calls(st)):
+                call_events[r][0].record(st)
+                for j, c in enumerate(c3):
                     c()
+                    call_events[r][j + 1].record(st)
+        graph = _capture(run_plain, torch)
+        graph_ev = _capture(run_with_events, torch)
         for _ in range(2):
             graph.replay()
+            graph_ev.replay()
         barrier()
+
+    per_call_samples = [[] for _ in range(NC)]
+
+    def read_call_events():
+        for r in range(R):
+            for j in range(NC):
+                per_call_samples[j].append(call_events[r][j].elapsed_time(call_events[r][j + 1]))
 
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    n_instr = len([i for i in range(args.steps) if i % (R + 1) == 0]) if graph is not None else args.steps
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(NC + 1)] for _ in range(n_instr)]
     e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # ---- the timed region: exactly args.steps steps
     barrier()
     e_begin.record(stream)
-    i, k, replays = 0, 0, 0
+    replays, i, used_ev = 0, 0, False
+    if graph is not None:
+        n_full = args.steps // R
+        for k in range(n_full):
+            if k == n_full - 1 and n_full >= 2:
+                graph_ev.replay(); used_ev = True     # the last R steps carry the per-call events
+            else:
+                graph.replay()
+            replays += 1
+            i += R
     while i < args.steps:
-        if graph is None:
-            step(i, evs[k]); k += 1; i += 1
-            continue
-        step(i, evs[k]); k += 1; i += 1          # instrumented step
-        if args.steps - i >= R:
-            graph.replay(); replays += 1; i += R  # R steps, one launch
-        else:
-            while i < args.steps:
-                step(i); i += 1
+        step(i); i += 1
     e_end.record(stream)
     barrier()
     total_ms = e_begin.elapsed_time(e_end)
-    clocks = sampler.stop() if rank == 0 else None
     status = aqt.aqt_device_status()
-    evs = evs[:k]
+    if used_ev:
+        read_call_events()
+    # more samples of the per-call events (outside the timed region), or call-by-call events without a graph
+    if graph_ev is not None:
+        for _ in range(8):
+            graph_ev.replay()
+            torch.cuda.synchronize()
+            read_call_events()
+    else:
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(NC + 1)]
+        for k in range(8):
+            evs[0].record(stream)
+            for j, f in enumerate(calls[k % R]):
+                f()
+                evs[j + 1].record(stream)
+            torch.cuda.synchronize()
+            for j in range(NC):
+                per_call_samples[j].append(evs[j].elapsed_time(evs[j + 1]))
+    per_call_ms = [statistics.mean(v) for v in per_call_samples]
 
-    per_call_ms = [statistics.mean(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(len(evs))) for j in range(NC)]
     t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -313,34 +374,28 @@ def run_ours(args):
     ops_step = sum(2 * M * s.N * s.K for s in specs)
     value = world * args.steps * ops_step / (total_ms * 1e-3) / 1e12
 
+    # ---- the same step for at least half a second (thousands of steps): the clock samples of the
+    # JSON line are taken while this and the timed region run
+    sustained = None
+    if graph is not None and world == 1 and not args.no_sustained:
+        ms_rep, n_rep = _time_replays(torch, graph, 200, min_seconds=0.6)
+        sustained = {"value": ops_step / (ms_rep / R * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_rep / R, "steps": n_rep * R,
+                     "seconds": ms_rep * n_rep * 1e-3}
+    clocks = sampler.stop() if rank == 0 else None
+
     # ---- the same step with the rounding of Fig. 2, floor(v + 0.5), in both quantizers (the headline
     # uses nearest-even, which the workload definitions ask for); graph replay, same buffers
     fig2_ms = None
     if graph is not None and world == 1:
-        side2 = torch.cuda.Stream()
-        side2.wait_stream(stream)
-        with torch.cuda.stream(side2):
-            fcalls = make_calls(side2, aqt.ROUND_HALF_UP_FLOOR)
-            for r in range(R):
-                for c in fcalls[r]:
+        def run_fig2(st):
+            for c3 in make_calls(st, aqt.ROUND_HALF_UP_FLOOR):
+                for c in c3:
                     c()
-        torch.cuda.synchronize()
-        g2 = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g2, stream=side2):
-            for r in range(R):
-                for c in fcalls[r]:
-                    c()
-        g2.replay()
-        torch.cuda.synchronize()
-        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        f0.record(stream)
-        for _ in range(10):
-            g2.replay()
-        f1.record(stream)
-        torch.cuda.synchronize()
-        fig2_ms = f0.elapsed_time(f1) / (10 * R)
+        g2 = _capture(run_fig2, torch)
+        fig2_ms = _time_replays(torch, g2, 20)[0] / R
 
-    # ---- end to end: host buffers through the C ABI, copies inside the timed region (per rank).
+    # ---- end to end: host buffers through the C ABI (aqt_ffn_fwd: copy in, quantize, both matmuls
+    # with the hidden tensor kept as codes, copy out), copies inside the timed region (per rank).
     # Every step copies its own input from pinned host memory and its own result back.  Steps
     # alternate between two streams (each with its own buffers) so that the host-to-device copy
     # of one step, the kernels of the previous one and the device-to-host copy of the one before
@@ -348,32 +403,22 @@ def run_ours(args):
     n_lanes = 2
     lanes = []
     for _ in range(n_lanes):
-        lanes.append({
-            "stream": torch.cuda.Stream(),
-            "xh": torch.from_numpy(x_host).clone().pin_memory(),
-            "yh": torch.empty((M, specs[1].N), dtype=torch.float32).pin_memory(),
-            "u": torch.empty((M, specs[0].N), dtype=torch.float32, device=dev),
-            "ws_a": torch.empty(aqt.linear_fwd_host_workspace_bytes(M, specs[0].N, specs[0].K, 8, 4, specs[0].act, True, False),
-                                dtype=torch.uint8, device=dev),
-            "ws_b": torch.empty(aqt.linear_fwd_host_workspace_bytes(M, specs[1].N, specs[1].K, 8, 4, specs[1].act, False, True),
-                                dtype=torch.uint8, device=dev)})
-
-    def e2e_step(i):
-        ln = lanes[i % n_lanes]
-        aqt.aqt_linear_fwd_host(ln["xh"], layers[0].wq, layers[0].s_w, None, ln["u"], ln["ws_a"], bits_a=8, bits_w=4,
-                                act=specs[0].act, stream=ln["stream"])
-        aqt.aqt_linear_fwd_host(ln["u"], layers[1].wq, layers[1].s_w, None, ln["yh"], ln["ws_b"], bits_a=8, bits_w=4,
-                                act=specs[1].act, stream=ln["stream"])
+        ln = {"stream": torch.cuda.Stream(), "xh": torch.from_numpy(x_host).clone().pin_memory(),
+              "yh": torch.empty((M, specs[1].N), dtype=torch.float32).pin_memory(),
+              "ws": torch.empty(aqt.aqt_workspace_bytes(aqt.OP_FFN_FWD, M, w.ff, w.d, 8, 4) + 256, dtype=torch.uint8, device=dev)}
+        ln["call"] = aqt.bind_ffn_fwd(ln["xh"], l0.mm_weight, l0.s_w, l0.mm_bits, l1.mm_weight, l1.s_w, l1.mm_bits, ln["yh"], ln["ws"],
+                                      bits_a=8, act=specs[0].act, stream=ln["stream"])
+        lanes.append(ln)
 
     for i in range(4):
-        e2e_step(i)
+        lanes[i % n_lanes]["call"]()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for ln in lanes:
         ln["stream"].wait_event(e0)
     for i in range(args.steps):
-        e2e_step(i)
+        lanes[i % n_lanes]["call"]()
     for ln in lanes:
         stream.wait_stream(ln["stream"])
     e1.record(stream)
@@ -382,43 +427,65 @@ def run_ours(args):
     if world > 1:
         dist.all_reduce(te, op=dist.ReduceOp.MAX)
     e2e_value = world * args.steps * ops_step / (float(te.item()) * 1e-3) / 1e12
+    e2e_status = aqt.aqt_device_status()
 
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
     if rank != 0:
         return 0
-
-    # ---- roofline of the dominant call (largest share of the step)
-    peak, peak_kind = _peaks()
+    # ---- roofline of the dominant call (largest share of the step), and every call's own figures
+    pk = _peaks()
     s0, s1_ = specs
     alg_bytes = [
         4 * M * s0.K + M * s0.K + 4 * M,                                              # quantize(x): read fp32, write codes + scales
         M * s0.K + s0.K * s0.N // 2 + 8 * s0.N + 4 * M + M * s0.N + 4 * M,            # GEMM 1: codes, int4 weights, scales in; codes + scales out
-        M * s1_.K + s1_.K * s1_.N // 2 + 8 * s1_.N + 4 * M + 4 * M * s1_.N,           # GEMM 2: codes, int4 weights, scales in; fp32 out
+        M * s1_.K + s1_.K * s1_.N + 8 * s1_.N + 4 * M + 4 * M * s1_.N,                # GEMM 2: codes, weights (int4 codes in int8 containers), scales in; fp32 out
     ]
-    kernels = [{"call": names[j], "ms": per_call_ms[j], "algorithmic_bytes": alg_bytes[j],
-                "gbs": alg_bytes[j] / (per_call_ms[j] * 1e-3) / 1e9, "share": per_call_ms[j] / sum(per_call_ms)} for j in range(NC)]
+    alg_ops = [0, 2 * M * s0.N * s0.K, 2 * M * s1_.N * s1_.K]
+    sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
+    sm_max_mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
+    kernels = []
+    for j in range(NC):
+        sec = per_call_ms[j] * 1e-3
+        k = {"call": names[j], "ms": per_call_ms[j], "algorithmic_bytes": alg_bytes[j], "gbs": alg_bytes[j] / sec / 1e9,
+             "hbm_frac": alg_bytes[j] / sec / 1e9 / pk["hbm_gbs"], "share": per_call_ms[j] / sum(per_call_ms),
+             "plan": ("quantize_rows", "requant ws128 (weight stationary, rows quantized in the epilogue)",
+                      aqt.aqt_plan_qmatmul(M, s1_.N, s1_.K, 8, aqt.BITS_4_UNPACKED, s1_.act))[j]}
+        if alg_ops[j]:
+            tops = alg_ops[j] / sec / 1e12
+            k.update({"tops": tops, "tensor_frac_nominal_int8": tops / INT8_NOMINAL_TOPS,
+                      "tensor_frac_2x_bf16_" + pk["kind"]: tops / (2.0 * pk["bf16"]),
+                      "tensor_frac_at_sampled_clock": tops / (INT8_NOMINAL_TOPS * sm_mhz / sm_max_mhz)})
+        kernels.append(k)
     # DRAM traffic per launch from the committed ncu captures (dram__bytes_read.sum +
     # dram__bytes_write.sum); the write part undercounts what is still in L2 when the kernel ends.
     ncu_traffic = NCU_TRAFFIC if aqt.aqt_version() == NCU_CAPTURE_VERSION else {}
     dom = max(range(NC), key=lambda j: per_call_ms[j])
+    props = torch.cuda.get_device_properties(dev)
     if dom == 1:
         # The fused kernel moves 33 MB (5 us of HBM time) and is bound by arithmetic instead: the
-        # Swish needs two special-function operations (2^x, reciprocal) per element, and an SM
-        # retires 16 of those per clock.  peak = 16 x SMs x the maximum SM clock.
-        props = torch.cuda.get_device_properties(dev)
-        sm_max_mhz = (clocks or {}).get("sm_max_mhz") or 1965
-        sfu_peak = 16 * props.multi_processor_count * sm_max_mhz * 1e6 / 1e9      # Gop/s
+        # Swish needs two special-function operations (2^x, reciprocal) per element.  peak = the
+        # special-function rate measured in this run by a kernel that does nothing else
+        # (aqt_selftest_sfu_rate); the nominal 16 op/clk/SM x SMs x the maximum SM clock beside it.
+        sfu_nominal = 16 * props.multi_processor_count * sm_max_mhz * 1e6 / 1e9      # Gop/s
+        sfu_measured = aqt.aqt_selftest_sfu_rate()
         sfu_achieved = 2.0 * M * s0.N / (per_call_ms[1] * 1e-3) / 1e9
-        roofline = {"bound": "alu", "kernel": names[1], "achieved": sfu_achieved, "peak": sfu_peak, "unit": "Gop/s",
-                    "frac": sfu_achieved / sfu_peak, "peak_source": "special-function unit: 16 op/clk/SM x %d SMs x %d MHz" %
-                    (props.multi_processor_count, sm_max_mhz), "hbm_frac": kernels[1]["gbs"] / peak,
+        roofline = {"bound": "alu", "kernel": names[1], "achieved": sfu_achieved, "peak": sfu_measured, "unit": "Gop/s",
+                    "frac": sfu_achieved / sfu_measured,
+                    "peak_source": "special-function unit, measured in this run by aqt_selftest_sfu_rate (2^x and reciprocal chains only)",
+                    "peak_nominal": sfu_nominal, "frac_of_nominal": sfu_achieved / sfu_nominal,
+                    "peak_nominal_source": "16 op/clk/SM x %d SMs x %d MHz" % (props.multi_processor_count, sm_max_mhz),
+                    "hbm_frac": kernels[1]["hbm_frac"], "tensor_frac_nominal_int8": kernels[1]["tensor_frac_nominal_int8"],
                     "traffic": ncu_traffic.get(1), "calls": kernels}
+    elif dom == 2 and kernels[2]["tensor_frac_nominal_int8"] > kernels[2]["hbm_frac"]:
+        roofline = {"bound": "tensor", "kernel": names[2], "achieved": kernels[2]["tops"], "peak": INT8_NOMINAL_TOPS, "unit": "TOP/s",
+                    "frac": kernels[2]["tensor_frac_nominal_int8"], "peak_source": "nominal dense int8 (no measured int8 peak exists)",
+                    "hbm_frac": kernels[2]["hbm_frac"], "traffic": ncu_traffic.get(2), "calls": kernels}
     else:
         achieved = kernels[dom]["gbs"]
-        roofline = {"bound": "hbm", "kernel": names[dom], "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                    "peak_source": "of " + peak_kind, "traffic": ncu_traffic.get(dom), "calls": kernels}
+        roofline = {"bound": "hbm", "kernel": names[dom], "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / pk["hbm_gbs"], "peak_source": "of " + pk["kind"], "traffic": ncu_traffic.get(dom), "calls": kernels}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -429,19 +496,26 @@ def run_ours(args):
             "frames_per_s": world * args.steps * M / (total_ms * 1e-3),
             "clocks": clocks, "device_status": status,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 4 * M * s0.K, "d2h_bytes_per_step": 4 * M * s1_.N,
-                    "ms_per_step": float(te.item()) / args.steps, "streams": n_lanes},
-            "gpu_launches": args.steps * 4, "sum_call_ms_per_step": sum(per_call_ms),
-            "launch_mode": ("cuda graph of %d steps x %d replays + %d call-by-call steps with per-call events" % (R, replays, len(evs)))
+                    "ms_per_step": float(te.item()) / args.steps, "streams": n_lanes, "api": "aqt_ffn_fwd", "device_status": e2e_status},
+            "gpu_launches": args.steps * NC, "sum_call_ms_per_step": sum(per_call_ms),
+            "launch_mode": ("cuda graph of %d steps x %d replays (%s per-call events inside the graph) + %d call-by-call steps" %
+                            (R, replays, "the last with" if used_ev else "no", args.steps - replays * R))
             if graph is not None else "call by call",
             "roofline": roofline}
+    if sustained is not None:
+        line["sustained"] = sustained
     if fig2_ms is not None:
         line["fig2_rounding"] = {"rounding": "floor(v + 0.5)", "ms_per_step": fig2_ms, "value": ops_step / (fig2_ms * 1e-3) / 1e12,
                                  "unit": UNIT}
-    if world == 1 and not args.no_encoder:
+    if world == 1 and not args.no_legs:
+        line["quantizer"] = quantizer_leg(dev)
         line["encoder"] = encoder_frames_per_s(dev)
         line["weight_only"] = weight_only_ffn_pair(dev)
+        line["weight_quantizer"] = weight_quantizer_leg(dev)
         line["backward"] = backward_ffn_layer(dev)
-        line["encoder_large"] = encoder_frames_per_s(dev, steps=2, cfg=5)  # last: seconds of dense work that pull the clocks down
+        # last: seconds of dense work that pull the clocks down
+        line["encoder_large"] = encoder_frames_per_s(dev, steps=2, cfg=5)
+        line["large_gemm"] = large_gemm_leg(dev)
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline()
     print(json.dumps(line), flush=True)
@@ -490,6 +564,115 @@ def encoder_frames_per_s(dev, steps: int = 5, cfg: int = 4):
     ms = e0.elapsed_time(e1) / steps
     return {"workload": w.name, "frames_per_s": w.M / (ms * 1e-3), "ms_per_step": ms, "tops": stack.ops / (ms * 1e-3) / 1e12,
             "steps": steps, "linears_per_step": len(specs) * w.blocks, "launch_mode": "cuda graph"}
+
+
+def quantizer_leg(dev, replays: int = 10):
+    """The activation quantizer alone on tensors far larger than L2 (row-wise abs-max, scale,
+    round, cast / nibble pack): GB/s of the bytes the method itself must move, 4 per element in,
+    1 (int8) or 1/2 (packed int4) out, 4 per row of scales, against the measured HBM copy rate.
+    Two input tensors alternate, so nothing is served from L2."""
+    import torch
+    from paper_2203_15952_b200 import binding as aqt
+    pk = _peaks()
+    out = []
+    g = torch.Generator(device=dev).manual_seed(7)
+    for (M, K) in ((65536, 4096), (65536, 1024)):
+        xs = [torch.randn((M, K), generator=g, device=dev) for _ in range(2)]
+        for bits, pack in ((8, False), (4, True)):
+            q = torch.empty((M, K // 2 if pack else K), dtype=torch.uint8 if pack else torch.int8, device=dev)
+            sc = torch.empty(M, dtype=torch.float32, device=dev)
+
+            def run(st):
+                for x in xs:
+                    aqt.bind_quantize(x, bits, aqt.AXIS_ROW, aqt.ROUND_NEAREST_EVEN, pack, q, sc, st)()
+            graph = _capture(run, torch)
+            ms = _time_replays(torch, graph, replays)[0] / len(xs)
+            nbytes = 4 * M * K + M * K * bits // 8 + 4 * M
+            gbs = nbytes / (ms * 1e-3) / 1e9
+            out.append({"rows": M, "cols": K, "bits": bits, "packed": pack, "ms": ms, "algorithmic_bytes": nbytes,
+                        "roofline": {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": gbs / pk["hbm_gbs"],
+                                     "peak_source": "of " + pk["kind"], "traffic": None}})
+            del graph
+        del xs
+    return out
+
+
+def weight_quantizer_leg(dev, replays: int = 10):
+    """The weight quantizer as a per-step leg (training from scratch re-quantizes the float weights
+    every step, Section 2.2): aqt_quantize over K per output channel with nibble packing, for the ten
+    weights of every block of the d = 512 encoder (17 blocks, 357 MB of fp32 weights: beyond L2)."""
+    import torch
+    from paper_2203_15952_b200 import binding as aqt
+    from paper_2203_15952_b200 import inputs as gen
+    pk = _peaks()
+    w = gen.WORKLOADS[4]
+    specs = gen.block_linears(w.d, w.ff, 4, 4, 8)
+    g = torch.Generator(device=dev).manual_seed(8)
+    blocks = [[torch.randn((s.N, s.K), generator=g, device=dev) * (s.K ** -0.5) for s in specs] for _ in range(w.blocks)]
+    outs = [(torch.empty((s.N, s.K // 2), dtype=torch.uint8, device=dev), torch.empty(s.N, dtype=torch.float32, device=dev)) for s in specs]
+
+    def run(st):
+        for blk in blocks:
+            for wt, (q, sc) in zip(blk, outs):
+                aqt.bind_quantize(wt, 4, aqt.AXIS_ROW, aqt.ROUND_NEAREST_EVEN, True, q, sc, st)()
+    graph = _capture(run, torch)
+    ms = _time_replays(torch, graph, replays)[0]
+    elems = sum(s.N * s.K for s in specs) * w.blocks
+    nbytes = 4 * elems + elems // 2 + 4 * sum(s.N for s in specs) * w.blocks
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"workload": "int4 weight quantizer, 10 weights x %d blocks, d = %d" % (w.blocks, w.d), "ms_per_step": ms,
+            "ms_per_block": ms / w.blocks, "launches_per_step": len(specs) * w.blocks, "algorithmic_bytes": nbytes,
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": gbs / pk["hbm_gbs"],
+                         "peak_source": "of " + pk["kind"], "traffic": None}}
+
+
+def large_gemm_leg(dev, burst_replays: int = 20, sustained_seconds: float = 2.0):
+    """The integer matmul on the large shapes of the d = 1024 encoder (M = 65 536, int8 activation
+    codes, int4 weights): burst (20 graph replays) and sustained (2 s back to back, with the SM clock
+    and power sampled meanwhile).  TOPS against the nominal dense int8 peak, against twice the
+    measured bf16 rates (no int8 peak has been measured on this machine) and scaled to the sampled clock."""
+    import torch
+    from paper_2203_15952_b200 import binding as aqt
+    pk = _peaks()
+    M = 65536
+    out = []
+    g = torch.Generator(device=dev).manual_seed(9)
+    for (N, K, act, with_res, what) in ((1024, 4096, aqt.ACT_NONE, True, "ffn second layer + residual"),
+                                        (4096, 1024, aqt.ACT_SWISH, False, "ffn first layer, Swish")):
+        xq = torch.randint(-127, 128, (M, K), generator=g, dtype=torch.int8, device=dev)
+        wq = torch.randint(-7, 8, (N, K), generator=g, dtype=torch.int8, device=dev)
+        s_x = torch.rand(M, generator=g, device=dev) * 1e-2 + 1e-3
+        s_w = torch.rand(N, generator=g, device=dev) * 1e-3 + 1e-4
+        ys = [torch.empty((M, N), dtype=torch.float32, device=dev) for _ in range(2)]
+        res = torch.randn((M, N), generator=g, device=dev) if with_res else None
+
+        def run(st):
+            for y in ys:
+                aqt.bind_qmatmul(xq, s_x, wq, s_w, None, res, 1.0, K, 8, aqt.BITS_4_UNPACKED, act, aqt.SCALE_ROW, y, None, st)()
+        graph = _capture(run, torch)
+        ops = 2.0 * M * N * K
+        burst_ms = _time_replays(torch, graph, burst_replays // 2)[0] / len(ys)
+        sampler = ClockSampler(torch.cuda.current_device())
+        sampler.start()
+        time.sleep(0.2)
+        sus_ms, n = _time_replays(torch, graph, 20, min_seconds=sustained_seconds, warm=0)
+        sus_ms /= len(ys)
+        clocks = sampler.stop()
+        mhz = clocks.get("sm_mhz") or 1965.0
+        mx = clocks.get("sm_max_mhz") or 1965.0
+        tb, ts = ops / (burst_ms * 1e-3) / 1e12, ops / (sus_ms * 1e-3) / 1e12
+        nbytes = M * K + N * K // 2 + 8 * N + 4 * M + 4 * M * N * (2 if with_res else 1)
+        out.append({"shape": "%d x %d -> %d" % (M, K, N), "what": what, "plan": aqt.aqt_plan_qmatmul(M, N, K, 8, 4, act),
+                    "burst": {"ms": burst_ms, "tops": tb, "frac_nominal_int8": tb / INT8_NOMINAL_TOPS,
+                              "frac_2x_bf16_burst_" + pk["kind"]: tb / (2 * pk["bf16"])},
+                    "sustained": {"ms": sus_ms, "tops": ts, "seconds": sus_ms * n * len(ys) * 1e-3, "frac_nominal_int8": ts / INT8_NOMINAL_TOPS,
+                                  "frac_2x_bf16_sustained_" + pk["kind"]: ts / (2 * pk["bf16_sustained"]),
+                                  "frac_of_int8_peak_at_sampled_clock": ts / (INT8_NOMINAL_TOPS * mhz / mx), "clocks": clocks},
+                    "hbm_frac_burst": nbytes / (burst_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+                    "roofline": {"bound": "tensor", "achieved": tb, "peak": INT8_NOMINAL_TOPS, "unit": "TOP/s", "frac": tb / INT8_NOMINAL_TOPS,
+                                 "peak_source": "nominal dense int8; twice the measured bf16 burst beside it", "traffic": None}})
+        del graph, xq, wq, ys, res
+    return out
 
 
 def weight_only_ffn_pair(dev, steps: int = 20):
@@ -613,7 +796,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-budget-s", type=float, default=100.0, help="--impl reference: CPU seconds for warm-up + steps together")
-    ap.add_argument("--no-encoder", action="store_true", help="skip the 17-block encoder-stack frames/s leg")
+    ap.add_argument("--no-legs", "--no-encoder", dest="no_legs", action="store_true",
+                    help="skip the legs beside the headline (quantizer, encoder stacks, weight-only, backward, large matmuls)")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the half-second sustained run of the headline step")
     ap.add_argument("--no-graph", action="store_true", help="launch every step call by call (no CUDA graph replay)")
     args = ap.parse_args()
     if args.impl == "reference":

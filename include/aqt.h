@@ -32,7 +32,7 @@
 extern "C" {
 #endif
 
-#define AQT_VERSION 106
+#define AQT_VERSION 200
 
 /* status codes */
 #define AQT_OK 0
@@ -62,6 +62,12 @@ extern "C" {
 #define AQT_ACT_GLU 2       /* a[j] = z[j] * sigmoid(z[j + N/2]), j < N/2; output has N/2 columns */
 #define AQT_ACT_GLU_SWISH 3 /* Swish applied to the GLU output                                  */
 
+/* operand widths of the matmul entry points (bits_a, bits_w).  Fig. 2 keeps 4-bit codes in an
+ * 8-bit container; the packed form is this library's storage layout. */
+#define AQT_BITS_4_UNPACKED 48 /* 4-bit codes, one per int8 container: what aqt_quantize(bits 4, pack 0) and
+                                  aqt_unpack_int4 produce.  Same layout as 8-bit codes; the smaller range lets the
+                                  epilogue convert accumulators on the plain ALUs up to a deeper K. */
+
 /* operations for aqt_workspace_bytes */
 #define AQT_OP_QMATMUL 1
 #define AQT_OP_LINEAR_FWD 2
@@ -69,6 +75,7 @@ extern "C" {
 #define AQT_OP_LINEAR_WEIGHT_ONLY 4    /* precision AQT_FLOAT_TF32   */
 #define AQT_OP_LINEAR_WEIGHT_ONLY_X2 5 /* precision AQT_FLOAT_TF32X2 */
 #define AQT_OP_LINEAR_BWD 6
+#define AQT_OP_FFN_FWD 7 /* N = feed-forward width, K = model width, bits_w for both layers */
 
 /* how float activations enter the tensor-core float matmul of the weight-only layer */
 #define AQT_FLOAT_TF32 0   /* one term: the upper ten fraction bits of each activation            */
@@ -110,9 +117,12 @@ int aqt_unpack_int4(const uint8_t* packed, int64_t rows, int64_t cols, int8_t* q
  *   z[m][n]   = fma(float(acc) * s_x[m or 0], s_w[n], bias[n]) binary32, bias = 0 if NULL
  *   a         = act(z)                                         see AQT_ACT_*
  *   y         = residual ? fma(residual_scale, a, residual) : a
- * xq        bits_a == 8: int8 [M, K];  bits_a == 4: uint8 [M, K/2] packed.
+ * xq        bits_a == 8 or AQT_BITS_4_UNPACKED: int8 [M, K];  bits_a == 4: uint8 [M, K/2] packed.
  * s_x       fp32 [M] (AQT_SCALE_ROW) or [1] (AQT_SCALE_TENSOR).
- * wq        W^T codes: bits_w == 8: int8 [N, K];  bits_w == 4: uint8 [N, K/2] packed.
+ * wq        W^T codes: bits_w == 8 or AQT_BITS_4_UNPACKED: int8 [N, K];  bits_w == 4: uint8 [N, K/2] packed.
+ *           (Weights with K > 512 that are used call after call are best unpacked once with
+ *           aqt_unpack_int4 and handed over as AQT_BITS_4_UNPACKED: the packed form is otherwise
+ *           sign-extended into the workspace on every call.)
  * s_w       fp32 [N];  bias fp32 [N] or NULL.
  * residual  fp32 [M, N_out] with row pitch ldr, or NULL.  N_out = N, or N/2 for the GLU forms.
  * y         fp32 [M, N_out], row pitch ldy.
@@ -127,6 +137,30 @@ int aqt_qmatmul(const void* xq, const float* s_x, int s_x_kind, const void* wq, 
                 const float* bias, const float* residual, int64_t ldr, float residual_scale, int64_t M,
                 int64_t N, int64_t K, int bits_a, int bits_w, int act, float* y, int64_t ldy,
                 int32_t* acc_debug, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * aqt_plan_qmatmul -- names the kernel configuration aqt_qmatmul (and every entry point that runs
+ * the same matmul) would launch for a shape: "small_m", "ws128e16", "pair256s6e4", ...  Host-only:
+ * sm_count_or_0 > 0 plans for a device with that many multiprocessors, 0 for the current device
+ * (148 if there is none).  float_kind != 0 plans the float matmul of aqt_linear_fwd_weight_only /
+ * aqt_linear_bwd with K in elements.  (No counterpart in the paper: the choice of tile shapes is
+ * this library's.)  name_out receives a NUL-terminated string of at most name_bytes bytes.
+ */
+int aqt_plan_qmatmul(int64_t M, int64_t N, int64_t K, int bits_a, int bits_w, int act, int float_kind,
+                     int sm_count_or_0, char* name_out, size_t name_bytes);
+
+/*
+ * aqt_qmatmul_with_plan -- aqt_qmatmul run with the kernel configuration named `plan` (a host
+ * string as returned by aqt_plan_qmatmul, except "small_m") instead of the one the library would
+ * choose.  For tests and tuning: results are identical whatever the plan (the integer sums are
+ * exact and the epilogue arithmetic is the same).  AQT_ERR_BADARG for an unknown name,
+ * AQT_ERR_UNSUPPORTED if that configuration cannot run the shape.  Other arguments as aqt_qmatmul.
+ */
+int aqt_qmatmul_with_plan(const char* plan, const void* xq, const float* s_x, int s_x_kind, const void* wq,
+                          const float* s_w, const float* bias, const float* residual, int64_t ldr,
+                          float residual_scale, int64_t M, int64_t N, int64_t K, int bits_a, int bits_w, int act,
+                          float* y, int64_t ldy, int32_t* acc_debug, void* workspace, size_t workspace_bytes,
+                          void* stream);
 
 /*
  * aqt_qmatmul_requant -- aqt_qmatmul whose output rows are quantized for the next layer inside
@@ -187,9 +221,29 @@ int aqt_linear_fwd_host(const float* x, int x_on_host, const void* wq, const flo
                         int act, float* y, int y_on_host, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * aqt_linear_fwd_weight_only -- the layer of the weight-only configurations (Section 4.1: "I8W":
- * int8 weight, float32 activation; "I4W": int4 weight, float32 activation; "we still need to
- * convert the weights to float during inference").  Activations are not quantized; the stored
+ * aqt_ffn_fwd -- a feed-forward pair of quantized layers, y = W2 . act(W1 . x), each layer the
+ * quantized linear layer of this library (Fig. 2 on its input rows, integer matmul, Section 2.2
+ * de-quantization): aqt_quantize(x) -> aqt_qmatmul_requant (the hidden tensor u = act(W1 . x)
+ * leaves the first matmul as codes and row scales and is never written as fp32) -> aqt_qmatmul.
+ * x, y      fp32 [M, d] dense; host pointers if x_on_host / y_on_host != 0 (pinned memory makes
+ *           the copies asynchronous), else device pointers.  The copies are enqueued on `stream`.
+ * w1q       W1^T codes [ff, d], s_w1 [ff], bias1 [ff] or NULL, bits_w1 as for aqt_qmatmul.
+ * w2q       W2^T codes [d, ff], s_w2 [d], bias2 [d] or NULL, bits_w2.
+ * bits_a    4 or 8: width both layers' activations are quantized to (per-row dynamic scales).
+ * act       AQT_ACT_NONE or AQT_ACT_SWISH between the layers.
+ * workspace at least aqt_workspace_bytes(AQT_OP_FFN_FWD, M, ff, d, bits_a, bits_w) bytes (sized for
+ *           host x and y and for one weight width: pass the wider of bits_w1 / bits_w2), 256-byte aligned.
+ * Limits: d <= 1024 and the limits of aqt_qmatmul_requant's fused form (AQT_ERR_UNSUPPORTED otherwise).
+ */
+int aqt_ffn_fwd(const float* x, int x_on_host, const void* w1q, const float* s_w1, const float* bias1, int bits_w1,
+                const void* w2q, const float* s_w2, const float* bias2, int bits_w2, int64_t M, int64_t d, int64_t ff,
+                int bits_a, int rounding, int act, float* y, int y_on_host, void* workspace, size_t workspace_bytes,
+                void* stream);
+
+/*
+ * aqt_linear_fwd_weight_only -- the layer of the weight-only configurations of Section 4.1 (I8W
+ * and I4W: 8- or 4-bit weight codes against unquantized binary32 activations; the section notes
+ * that the codes have to be turned back into floats when the layer runs).  Activations are not quantized; the stored
  * codes are converted to float and de-quantized by their channel scale (Section 2.2):
  *   z[m][n] = s_w[n] * sum_k x[m][k] * float(wq[n][k]) + bias[n]
  *   a = act(z);  y = residual ? fma(residual_scale, a, residual) : a
@@ -297,6 +351,17 @@ int aqt_device_status(void* stream, int* status_out);
  * clears.  (The paper has no counterpart: this is the library's own fault-reporting check.)
  */
 int aqt_selftest_bounded_wait(uint64_t limit_ns, int* gave_up_dev, void* stream);
+
+/*
+ * aqt_selftest_sfu_rate -- a measurement aid: launches a kernel that does nothing but the two
+ * special-function operations of the Swish / GLU epilogues (2^x and reciprocal) in independent
+ * chains on every SM, `iterations` (1 .. 2^20) rounds of 16 operations per thread.  *ops_out
+ * (host) receives the number of operations the launch performs; the caller times the launch
+ * (CUDA events) to get the device's special-function rate, the ceiling the activation epilogues
+ * are measured against.  sink_dev: one device float, never written in practice.  (The paper has
+ * no counterpart.)
+ */
+int aqt_selftest_sfu_rate(int iterations, float* sink_dev, int64_t* ops_out, void* stream);
 
 #ifdef __cplusplus
 }

@@ -7,14 +7,16 @@
  * library's product path never does.  It shares no code, header, table or helper with the CUDA
  * implementation.
  *
- * What is written out here, step by step and in the paper's order:
- *   Fig. 2 / Section 2.2 : quantize(input, axis) -- abs-max over the reduced axis, scale =
- *                          max / 127 (or / 7 for int4), scaled = divide_no_nan(input, scale),
- *                          code = floor(scaled + 0.5) cast to an int8 container.
- *   Section 2.2          : symmetric, no zero point; de-quantization multiplies by the scale.
- *   Section 1            : the matmul runs on the integer codes (native integer operations);
- *                          its float emulation differs once sums no longer fit the fp32
- *                          significand.
+ * What is written out here, in the paper's order:
+ *   Fig. 2 / Section 2.2 : the dynamic symmetric quantizer.  The largest magnitude along the
+ *                          reduced axis, divided by the largest code (127 at 8 bits, 7 at 4 bits),
+ *                          is the scale; every element is divided by its scale (zero where the
+ *                          scale is zero), rounded half-up by a floor, and kept in an 8-bit
+ *                          container.
+ *   Section 2.2          : the scheme is symmetric (no zero point), and a code times its scale
+ *                          gives the value back.
+ *   Section 1            : the matmul runs natively on the integer codes; emulating it in
+ *                          binary32 stops being exact once sums outgrow the significand.
  * Readings taken where the paper is silent are stated beside each function.
  *
  * Parity status of each function (what pins it, independent of this file) is listed in
@@ -57,16 +59,17 @@ int orc_num_threads(void) {
 #endif
 }
 
-/* qmax(b) = 2^(b-1) - 1: 127 for int8, 7 for int4 (Section 2.2: "127 for int8 (or by 7 for int4)"). */
+/* Largest code of a b-bit symmetric quantizer, 2^(b-1) - 1: the divisors 127 and 7 of Section 2.2. */
 static int qmax_of(int bits) { return bits == 8 ? 127 : (bits == 4 ? 7 : -1); }
 
-/* One element of Fig. 2 after the scale is known.
- * divide_no_nan: the quotient is 0 where the scale is 0.
- * Rounding: the figure's floor(v + 0.5) with the addition rounded in binary32, or IEEE
- * nearest-even (the workload definitions ask for the latter; both are kept).
+/* One element of Fig. 2 once its scale is known.
+ * The quotient is defined as 0 where the scale is 0 (the figure uses a division that returns 0
+ * instead of NaN or Inf there).
+ * Rounding: the figure adds one half and takes the floor, the sum being a binary32 value; the
+ * alternative is IEEE nearest-even, which the workload definitions ask for.  Both are kept.
  * The final clip is a guard only: with abs-max scaling |v| <= qmax up to one rounding, so the
- * clip acts only when the scale is subnormal and the quotient loses precision.  The paper has no
- * clamp (Section 1, "do not have clamp with learnable boundaries"). */
+ * clip acts only when the scale is subnormal and the quotient loses precision.  The method
+ * itself has no clipping range to learn or apply (Section 1). */
 static int8_t quantize_one(float x, float scale, int qmax, int rounding) {
   float v = (scale == 0.0f) ? 0.0f : x / scale;
   float r;
@@ -81,11 +84,11 @@ static int8_t quantize_one(float x, float scale, int qmax, int rounding) {
   return (int8_t)r;
 }
 
-/* Fig. 2, quantize(input, axis).  x is [rows, cols], row pitch ld (elements).
- * axis names the axis that is REDUCED (reduce_max(..., axis, keepdims=True)), so the scale has
- * extent 1 along it: ORC_AXIS_ROW -> scale[rows], ORC_AXIS_COL -> scale[cols], ORC_AXIS_TENSOR ->
- * scale[1].  q is [rows, cols] dense in an int8 container for both bit widths (the figure casts
- * to int8).  Returns 0, or -1 on a bad argument. */
+/* The quantizer of Fig. 2.  x is [rows, cols], row pitch ld (elements).
+ * axis names the axis that is REDUCED (the figure's maximum keeps that axis with extent 1), so
+ * there is one scale per slice across it: ORC_AXIS_ROW -> scale[rows], ORC_AXIS_COL ->
+ * scale[cols], ORC_AXIS_TENSOR -> scale[1].  q is [rows, cols] dense in an 8-bit container for
+ * both bit widths, as in the figure.  Returns 0, or -1 on a bad argument. */
 int orc_quantize(const float* x, int64_t rows, int64_t cols, int64_t ld, int bits, int axis,
                  int rounding, int8_t* q, float* scale) {
   const int qmax = qmax_of(bits);
@@ -94,34 +97,34 @@ int orc_quantize(const float* x, int64_t rows, int64_t cols, int64_t ld, int bit
   if (axis == ORC_AXIS_ROW) {
 #pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < rows; ++i) {
-      float max_val = 0.0f;
+      float amax = 0.0f;
       for (int64_t j = 0; j < cols; ++j) {
         float a = fabsf(x[i * ld + j]);
-        if (a > max_val) max_val = a;
+        if (a > amax) amax = a;
       }
-      float s = max_val / (float)qmax;
+      float s = amax / (float)qmax;
       scale[i] = s;
       for (int64_t j = 0; j < cols; ++j) q[i * cols + j] = quantize_one(x[i * ld + j], s, qmax, rounding);
     }
   } else if (axis == ORC_AXIS_COL) {
     for (int64_t j = 0; j < cols; ++j) {
-      float max_val = 0.0f;
+      float amax = 0.0f;
       for (int64_t i = 0; i < rows; ++i) {
         float a = fabsf(x[i * ld + j]);
-        if (a > max_val) max_val = a;
+        if (a > amax) amax = a;
       }
-      scale[j] = max_val / (float)qmax;
+      scale[j] = amax / (float)qmax;
     }
     for (int64_t i = 0; i < rows; ++i)
       for (int64_t j = 0; j < cols; ++j) q[i * cols + j] = quantize_one(x[i * ld + j], scale[j], qmax, rounding);
   } else if (axis == ORC_AXIS_TENSOR) {
-    float max_val = 0.0f;
+    float amax = 0.0f;
     for (int64_t i = 0; i < rows; ++i)
       for (int64_t j = 0; j < cols; ++j) {
         float a = fabsf(x[i * ld + j]);
-        if (a > max_val) max_val = a;
+        if (a > amax) amax = a;
       }
-    float s = max_val / (float)qmax;
+    float s = amax / (float)qmax;
     scale[0] = s;
     for (int64_t i = 0; i < rows; ++i)
       for (int64_t j = 0; j < cols; ++j) q[i * cols + j] = quantize_one(x[i * ld + j], s, qmax, rounding);
@@ -131,8 +134,8 @@ int orc_quantize(const float* x, int64_t rows, int64_t cols, int64_t ld, int bit
   return 0;
 }
 
-/* Section 2.2: "De-quantization will be done by multiplying a tensor with scale."
- * scale_kind selects which scale element applies (row i, column j, or the single one). */
+/* Section 2.2: de-quantization is one multiply of each code by its scale.
+ * `axis` selects which scale element applies (row i, column j, or the single one). */
 int orc_dequantize(const int8_t* q, int64_t rows, int64_t cols, const float* scale, int axis, float* x) {
   for (int64_t i = 0; i < rows; ++i)
     for (int64_t j = 0; j < cols; ++j) {
@@ -176,8 +179,8 @@ int64_t orc_weight_bytes(int64_t K, int64_t N, int bits) {
   return (K * N * bits + 7) / 8 + 4 * N;
 }
 
-/* The integer matmul on codes (Section 1: "native integer operations for executing quantized
- * operations (e.g. matrix multiplications)").  xq is [M, K]; wq holds W^T as [N, K] (row n is
+/* The integer matmul on codes (Section 1: quantized matrix products run as native integer
+ * operations).  xq is [M, K]; wq holds W^T as [N, K] (row n is
  * output channel n).  acc[m][n] = sum_k xq[m][k] * wq[n][k] in 64-bit integers; integer sums do
  * not depend on the order of summation.  Returns how many results fall outside int32 (0 for
  * every K <= 133 000 at 8 bits). */
@@ -194,9 +197,9 @@ int64_t orc_int_matmul(const int8_t* xq, const int8_t* wq, int64_t M, int64_t N,
   return overflow;
 }
 
-/* The float-emulated integer matmul of Section 1 ("int emulated in float32"): the same codes,
- * converted to binary32, multiplied and summed left to right in binary32.  Used only to test
- * the paper's remark that emulation and integer math agree while results fit the significand. */
+/* The integer matmul emulated in binary32, the alternative Section 1 argues against: the same
+ * codes converted to binary32, multiplied and summed left to right in binary32.  Used only to
+ * test the paper's remark that emulation and integer math agree while results fit the significand. */
 int orc_emulated_matmul_f32(const int8_t* xq, const int8_t* wq, int64_t M, int64_t N, int64_t K, float* out) {
   for (int64_t m = 0; m < M; ++m)
     for (int64_t n = 0; n < N; ++n) {
@@ -307,9 +310,9 @@ int orc_linear_fwd(const float* x, int64_t ldx, const int8_t* wq, const float* s
   return rc;
 }
 
-/* The layer of the weight-only configurations of Section 4.1 ("I8W": int8 weight, float32
- * activation; "I4W": int4 weight, float32 activation; the weights are converted to float at
- * inference).  Activations are not quantized; de-quantization multiplies the codes by their
+/* The layer of the weight-only configurations of Section 4.1 (I8W and I4W: 8- or 4-bit weight
+ * codes against unquantized binary32 activations, the codes being turned back into floats when
+ * the layer runs).  Activations are not quantized; de-quantization multiplies the codes by their
  * channel scale (Section 2.2).  The plain definition, every operation in double:
  *   z[m][n] = s_w[n] * sum_k x[m][k] * wq[n][k] + bias[n]
  * (each product of a binary32 value and a code is exact in double; the sum is rounded only at the
@@ -355,7 +358,7 @@ int orc_linear_weight_only_f64(const float* x, int64_t ldx, const int8_t* wq, co
 
 /* Backward of the quantized linear layer with straight-through quantizers.  The paper states only
  * that the scale carries no gradient (Fig. 2: stop_gradient(scale)) and that training runs the
- * same integer forward ("what you train is what you serve", Section 1); it does not print the
+ * same integer forward that serving uses (Section 1); it does not print the
  * backward products.  The plain straight-through definition is taken: the forward is
  *   y[m][n] = sum_k xhat[m][k] * what[n][k] + bias[n],  xhat = s_x * xq,  what = s_w * wq,
  * the quantizers pass gradients through unchanged (d xhat / d x = 1, d what / d w = 1), scales are

@@ -20,12 +20,14 @@ AXIS_ROW, AXIS_COL, AXIS_TENSOR = 0, 1, 2
 ROUND_HALF_UP_FLOOR, ROUND_NEAREST_EVEN = 0, 1
 SCALE_ROW, SCALE_TENSOR = 0, 1
 ACT_NONE, ACT_SWISH, ACT_GLU, ACT_GLU_SWISH = 0, 1, 2, 3
-OP_QMATMUL, OP_LINEAR_FWD, OP_QMATMUL_REQUANT, OP_LINEAR_WEIGHT_ONLY, OP_LINEAR_WEIGHT_ONLY_X2, OP_LINEAR_BWD = 1, 2, 3, 4, 5, 6
+OP_QMATMUL, OP_LINEAR_FWD, OP_QMATMUL_REQUANT, OP_LINEAR_WEIGHT_ONLY, OP_LINEAR_WEIGHT_ONLY_X2, OP_LINEAR_BWD, OP_FFN_FWD = 1, 2, 3, 4, 5, 6, 7
 FLOAT_TF32, FLOAT_TF32X2 = 0, 1
+BITS_4_UNPACKED = 48  # 4-bit codes, one per int8 container
 
 EXPORTS = ("aqt_version", "aqt_status_string", "aqt_quantize", "aqt_pack_int4", "aqt_unpack_int4", "aqt_qmatmul",
            "aqt_linear_fwd", "aqt_linear_fwd_host", "aqt_workspace_bytes", "aqt_device_status", "aqt_qmatmul_w4_noalloc",
-           "aqt_selftest_bounded_wait", "aqt_qmatmul_requant", "aqt_linear_fwd_weight_only", "aqt_linear_bwd")
+           "aqt_selftest_bounded_wait", "aqt_qmatmul_requant", "aqt_linear_fwd_weight_only", "aqt_linear_bwd",
+           "aqt_plan_qmatmul", "aqt_qmatmul_with_plan", "aqt_ffn_fwd", "aqt_selftest_sfu_rate")
 NOALLOC_MAX_WEIGHT_BYTES = 4 << 20
 
 
@@ -145,6 +147,15 @@ def aqt_workspace_bytes(op: int, M: int, N: int, K: int, bits_a: int, bits_w: in
     return int(lib().aqt_workspace_bytes(int(op), _i64(M), _i64(N), _i64(K), int(bits_a), int(bits_w)))
 
 
+def aqt_plan_qmatmul(M: int, N: int, K: int, bits_a: int = 8, bits_w: int = 8, act: int = ACT_NONE, float_kind: bool = False,
+                     sm_count: int = 0) -> str:
+    """Name of the kernel configuration the library launches for this shape (host-only)."""
+    buf = ctypes.create_string_buffer(64)
+    _check("aqt_plan_qmatmul", lib().aqt_plan_qmatmul(_i64(M), _i64(N), _i64(K), int(bits_a), int(bits_w), int(act),
+                                                      int(bool(float_kind)), int(sm_count), buf, ctypes.c_size_t(64)))
+    return buf.value.decode()
+
+
 def aqt_device_status(stream=None) -> int:
     out = ctypes.c_int(0)
     _check("aqt_device_status", lib().aqt_device_status(_stream(stream), ctypes.byref(out)))
@@ -158,6 +169,24 @@ def aqt_selftest_bounded_wait(limit_ns: int = 1_000_000, stream=None) -> bool:
     _check("aqt_selftest_bounded_wait", lib().aqt_selftest_bounded_wait(ctypes.c_uint64(limit_ns), _ptr(flag), _stream(stream)))
     torch.cuda.synchronize()
     return bool(flag.item() == 1)
+
+
+def aqt_selftest_sfu_rate(iterations: int = 4096, repeats: int = 3) -> float:
+    """Special-function operations per second (in Gop/s) of the current device, measured with a
+    kernel that runs only 2^x and reciprocal chains; best of `repeats` timed launches."""
+    sink = torch.zeros(1, dtype=torch.float32, device="cuda")
+    ops = ctypes.c_int64(0)
+    stream = torch.cuda.current_stream()
+    best = 0.0
+    for i in range(repeats + 1):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        _check("aqt_selftest_sfu_rate", lib().aqt_selftest_sfu_rate(int(iterations), _ptr(sink), ctypes.byref(ops), _stream(stream)))
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if i > 0:
+            best = max(best, ops.value / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+    return best
 
 
 def aqt_quantize(x: torch.Tensor, bits: int, axis: int = AXIS_ROW, rounding: int = ROUND_NEAREST_EVEN,
@@ -208,20 +237,24 @@ def aqt_qmatmul(xq: torch.Tensor, s_x: torch.Tensor, wq: torch.Tensor, s_w: torc
                 bias: Optional[torch.Tensor] = None, residual: Optional[torch.Tensor] = None, residual_scale: float = 1.0,
                 *, K: int, bits_a: int = 8, bits_w: int = 8, act: int = ACT_NONE, s_x_kind: int = SCALE_ROW,
                 y: Optional[torch.Tensor] = None, acc_debug: Optional[torch.Tensor] = None,
-                workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+                workspace: Optional[torch.Tensor] = None, stream=None, plan: Optional[str] = None) -> torch.Tensor:
     """Integer matmul on codes + de-quantizing epilogue.  xq [M, K] int8 or [M, K/2] uint8 packed;
-    wq [N, K] int8 or [N, K/2] uint8 packed.  Returns y fp32 [M, N_out]."""
+    wq [N, K] int8 or [N, K/2] uint8 packed.  Returns y fp32 [M, N_out].  plan: a kernel
+    configuration by name (aqt_qmatmul_with_plan) instead of the library's own choice."""
     M, N = xq.shape[0], wq.shape[0]
     n_out = _n_out(N, act)
     if y is None:
         y = torch.empty((M, n_out), dtype=torch.float32, device=xq.device)
     need = aqt_workspace_bytes(OP_QMATMUL, M, N, K, bits_a, bits_w)
     workspace = _workspace(need, workspace, xq.device)
-    _check("aqt_qmatmul", lib().aqt_qmatmul(
-        _ptr(xq), _ptr(s_x), int(s_x_kind), _ptr(wq), _ptr(s_w), _ptr(bias), _ptr(residual),
-        _i64(residual.stride(0) if residual is not None else 0), ctypes.c_float(residual_scale), _i64(M), _i64(N), _i64(K),
-        int(bits_a), int(bits_w), int(act), _ptr(y), _i64(y.stride(0)), _ptr(acc_debug), _ptr(workspace),
-        ctypes.c_size_t(0 if workspace is None else workspace.numel()), _stream(stream)))
+    args = (_ptr(xq), _ptr(s_x), int(s_x_kind), _ptr(wq), _ptr(s_w), _ptr(bias), _ptr(residual),
+            _i64(residual.stride(0) if residual is not None else 0), ctypes.c_float(residual_scale), _i64(M), _i64(N), _i64(K),
+            int(bits_a), int(bits_w), int(act), _ptr(y), _i64(y.stride(0)), _ptr(acc_debug), _ptr(workspace),
+            ctypes.c_size_t(0 if workspace is None else workspace.numel()), _stream(stream))
+    if plan is None:
+        _check("aqt_qmatmul", lib().aqt_qmatmul(*args))
+    else:
+        _check("aqt_qmatmul_with_plan", lib().aqt_qmatmul_with_plan(ctypes.c_char_p(plan.encode()), *args))
     return y
 
 
@@ -357,4 +390,25 @@ def aqt_linear_fwd_host(x: torch.Tensor, wq: torch.Tensor, s_w: torch.Tensor, bi
         _ptr(x), int(not x.is_cuda), _ptr(wq), _ptr(s_w), _ptr(bias), _i64(M), _i64(N), _i64(K), int(bits_a), int(bits_w),
         int(a_scale_kind), int(rounding), int(act), _ptr(y), int(not y.is_cuda), _ptr(workspace),
         ctypes.c_size_t(workspace.numel()), _stream(stream)))
+    return y
+
+
+def bind_ffn_fwd(x, w1q, s_w1, bits_w1, w2q, s_w2, bits_w2, y, workspace, *, bits_a=8, rounding=ROUND_NEAREST_EVEN, act=ACT_SWISH,
+                 stream=None):
+    """Pre-marshalled aqt_ffn_fwd (see bind): x, y fp32 [M, d] on the host (pinned) or the device."""
+    M, d = x.shape
+    ff = w1q.shape[0]
+    return bind("aqt_ffn_fwd", _ptr(x), int(not x.is_cuda), _ptr(w1q), _ptr(s_w1), _ptr(None), int(bits_w1), _ptr(w2q), _ptr(s_w2),
+                _ptr(None), int(bits_w2), _i64(M), _i64(d), _i64(ff), int(bits_a), int(rounding), int(act), _ptr(y), int(not y.is_cuda),
+                _ptr(workspace), ctypes.c_size_t(workspace.numel()), _stream(stream))
+
+
+def aqt_ffn_fwd(x, w1q, s_w1, bits_w1, w2q, s_w2, bits_w2, y, workspace=None, **kw):
+    """y = W2 . act(W1 . x) through two quantized layers (aqt_ffn_fwd); x / y may be pinned host tensors."""
+    M, d = x.shape
+    ff = w1q.shape[0]
+    if workspace is None:
+        workspace = torch.empty(aqt_workspace_bytes(OP_FFN_FWD, M, ff, d, kw.get("bits_a", 8), 4), dtype=torch.uint8,
+                                device=w1q.device)
+    bind_ffn_fwd(x, w1q, s_w1, bits_w1, w2q, s_w2, bits_w2, y, workspace, **kw)()
     return y

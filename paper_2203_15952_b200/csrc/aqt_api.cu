@@ -12,26 +12,27 @@ using namespace aqt;
 
 namespace {
 
-// The kernels use tcgen05 / TMEM and exist for compute capability 10.x only.
+// The kernels use tcgen05 / TMEM and exist for compute capability 10.x only.  Asked of the
+// current device on every call (the answer is cached per device ordinal).
 int check_device() {
-  static int cached = 1;  // 1 = not yet known
-  if (cached == 1) {
-    int dev = 0, major = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return AQT_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return AQT_ERR_CUDA;
-    cached = (major == 10) ? AQT_OK : AQT_ERR_UNSUPPORTED;
-  }
-  return cached;
+  DeviceInfo d;
+  int rc = current_device_info(&d);
+  if (rc != AQT_OK) return rc;
+  return d.cc_major == 10 ? AQT_OK : AQT_ERR_UNSUPPORTED;
 }
 
-bool bits_ok(int b) { return b == 4 || b == 8; }
+// Operand widths a matmul accepts: 8, 4 (nibble-packed) or 4-bit codes in int8 containers.
+bool bits_ok(int b) { return b == 4 || b == 8 || b == AQT_BITS_4_UNPACKED; }
+bool quant_bits_ok(int b) { return b == 4 || b == 8; }
+bool is_packed(int b) { return b == 4; }
+int code_bits(int b) { return b == 8 ? 8 : 4; }  // range of the codes, whatever the container
 bool act_ok(int a) { return a >= AQT_ACT_NONE && a <= AQT_ACT_GLU_SWISH; }
 bool is_glu(int a) { return a == AQT_ACT_GLU || a == AQT_ACT_GLU_SWISH; }
 
 size_t ws_qmatmul(int64_t M, int64_t N, int64_t K, int bits_a, int bits_w) {
   size_t b = 0;
-  if (bits_a == 4) b += round_up((size_t)M * (size_t)K, 256);
-  if (bits_w == 4) b += round_up((size_t)N * (size_t)K, 256);
+  if (is_packed(bits_a)) b += round_up((size_t)M * (size_t)K, 256);
+  if (is_packed(bits_w)) b += round_up((size_t)N * (size_t)K, 256);
   return b;
 }
 size_t ws_linear(int64_t M, int64_t N, int64_t K, int bits_w) {
@@ -147,18 +148,22 @@ int run_small_m(const void* xq, bool a_packed, const float* s_x, int s_x_kind, c
 // Codes already in int8 containers for A; B possibly packed.  ws holds B's unpacked copy.
 int qmatmul_i8a(const int8_t* a_codes, const float* s_x, int s_x_kind, const void* wq, const float* s_w, const float* bias,
                 const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K, int bits_a, int bits_w,
-                int act, float* y, int64_t ldy, int32_t* acc_debug, uint8_t* ws, cudaStream_t st) {
-  if (small_m_applies(M, K)) {
+                int act, float* y, int64_t ldy, int32_t* acc_debug, uint8_t* ws, cudaStream_t st, int forced_plan = kPlanNone) {
+  if (forced_plan == kPlanNone && small_m_applies(M, K)) {
     // a few rows: weight-bandwidth-bound kernel, packed weights read as they are
-    return run_small_m(a_codes, false, s_x, s_x_kind, wq, bits_w == 4, s_w, bias, residual, ldr, residual_scale, M, N, K, act, y, ldy,
+    return run_small_m(a_codes, false, s_x, s_x_kind, wq, is_packed(bits_w), s_w, bias, residual, ldr, residual_scale, M, N, K, act, y, ldy,
                        acc_debug, st);
   }
   // 4-bit weights: the weight-stationary kernel (K <= 512) sign-extends them itself in shared
   // memory after TMA staging; deeper K takes a one-off sign-extended copy in the workspace.
   const void* b_codes = wq;
   bool b_packed = false;
-  if (bits_w == 4) {
-    if (qgemm_uses_ws(N, K) && K % 32 == 0) {  // the packed rows must keep the 16-byte pitch bulk copies need
+  if (is_packed(bits_w)) {
+    const int sms = sm_count();
+    if (sms <= 0) return AQT_ERR_CUDA;
+    const int plan = forced_plan != kPlanNone ? forced_plan : plan_qgemm(GemmShape{M, N, K, act, 0, false}, sms);
+    const bool ws_plan = plan == kPlanWs128E16 || plan == kPlanWs128E8;
+    if (ws_plan && K % 32 == 0) {  // the packed rows must keep the 16-byte pitch bulk copies need
       b_packed = true;
     } else {
       int rc = launch_unpack_int4(reinterpret_cast<const uint8_t*>(wq), N * K / 2, reinterpret_cast<int8_t*>(ws), st);
@@ -182,8 +187,27 @@ int qmatmul_i8a(const int8_t* a_codes, const float* s_x, int s_x_kind, const voi
   p.n_out = is_glu(act) ? (int)(N / 2) : (int)N;
   p.tiles_m = p.tiles_n = p.k_blocks = 0;
   // |acc| <= K * 2^(bits_a - 1) * 2^(bits_w - 1) for any codes the containers can hold
-  p.small_acc = (K * (int64_t)(qmax_of(bits_a) + 1) * (qmax_of(bits_w) + 1) <= (1ll << 22)) ? 1 : 0;
-  return launch_qgemm(a_codes, b_codes, b_packed, y, ldy, p, st);
+  p.small_acc = (K * (int64_t)(qmax_of(code_bits(bits_a)) + 1) * (qmax_of(code_bits(bits_w)) + 1) <= (1ll << 22)) ? 1 : 0;
+  return launch_qgemm(a_codes, b_codes, b_packed, y, ldy, p, st, forced_plan);
+}
+
+// Workspace of aqt_ffn_fwd: [x on the device | y on the device | codes of x | scales | codes of u | scales | matmul scratch].
+struct FfnLayout {
+  size_t x, y, q1, s1, q2, s2, mm, total;
+};
+FfnLayout ffn_layout(int64_t M, int64_t d, int64_t ff, int bits_w1, int bits_w2) {
+  FfnLayout L;
+  L.x = 0;
+  L.y = L.x + round_up((size_t)M * d * 4, 256);
+  L.q1 = L.y + round_up((size_t)M * d * 4, 256);
+  L.s1 = L.q1 + round_up((size_t)M * d, 256);
+  L.q2 = L.s1 + round_up((size_t)M * 4, 256);
+  L.s2 = L.q2 + round_up((size_t)M * ff, 256);
+  L.mm = L.s2 + round_up((size_t)M * 4, 256);
+  const size_t mm1 = round_up(ws_qmatmul(M, ff, d, 8, bits_w1), 256) + requant_exchange_bytes(M, ff);
+  const size_t mm2 = ws_qmatmul(M, d, ff, 8, bits_w2);
+  L.total = L.mm + round_up(mm1 > mm2 ? mm1 : mm2, 256);
+  return L;
 }
 
 }  // namespace
@@ -212,13 +236,14 @@ size_t aqt_workspace_bytes(int op, int64_t M, int64_t N, int64_t K, int bits_a, 
   if (op == AQT_OP_LINEAR_WEIGHT_ONLY) return ws_weight_only(0, N, K, AQT_FLOAT_TF32);
   if (op == AQT_OP_LINEAR_WEIGHT_ONLY_X2) return ws_weight_only(M, N, K, AQT_FLOAT_TF32X2);
   if (op == AQT_OP_LINEAR_BWD) return bwd_layout(M, N, K).total;
+  if (op == AQT_OP_FFN_FWD) return ffn_layout(M, K, N, bits_w, bits_w).total;
   if (op == AQT_OP_QMATMUL_REQUANT) return round_up(ws_qmatmul(M, N, K, bits_a, bits_w), 256) + requant_exchange_bytes(M, N);
   return 0;
 }
 
 int aqt_quantize(const float* x, int64_t rows, int64_t cols, int64_t ld, int bits, int axis, int rounding, int pack,
                  void* q_out, float* scale_out, void* stream) {
-  if (rows < 0 || cols < 0 || ld < cols || !bits_ok(bits)) return AQT_ERR_BADARG;
+  if (rows < 0 || cols < 0 || ld < cols || !quant_bits_ok(bits)) return AQT_ERR_BADARG;
   if (axis != AQT_AXIS_ROW && axis != AQT_AXIS_COL && axis != AQT_AXIS_TENSOR) return AQT_ERR_BADARG;
   if (rounding != AQT_ROUND_HALF_UP_FLOOR && rounding != AQT_ROUND_NEAREST_EVEN) return AQT_ERR_BADARG;
   if (pack != 0 && pack != 1) return AQT_ERR_BADARG;
@@ -256,10 +281,10 @@ int aqt_unpack_int4(const uint8_t* packed, int64_t rows, int64_t cols, int8_t* q
   return launch_unpack_int4(packed, rows * cols / 2, q, reinterpret_cast<cudaStream_t>(stream));
 }
 
-int aqt_qmatmul(const void* xq, const float* s_x, int s_x_kind, const void* wq, const float* s_w, const float* bias,
-                const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K, int bits_a,
-                int bits_w, int act, float* y, int64_t ldy, int32_t* acc_debug, void* workspace, size_t workspace_bytes,
-                void* stream) {
+static int qmatmul_entry(const void* xq, const float* s_x, int s_x_kind, const void* wq, const float* s_w, const float* bias,
+                         const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K, int bits_a,
+                         int bits_w, int act, float* y, int64_t ldy, int32_t* acc_debug, void* workspace, size_t workspace_bytes,
+                         void* stream, int forced_plan) {
   int rc = validate_matmul_shape(M, N, K, bits_a, bits_w, act, s_x_kind);
   if (rc != AQT_OK) return rc;
   if (M == 0 || N == 0) return AQT_OK;
@@ -278,19 +303,55 @@ int aqt_qmatmul(const void* xq, const float* s_x, int s_x_kind, const void* wq, 
   if (rc != AQT_OK) return rc;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
-  if (small_m_applies(M, K)) {
-    return run_small_m(xq, bits_a == 4, s_x, s_x_kind, wq, bits_w == 4, s_w, bias, residual, ldr, residual_scale, M, N, K, act, y, ldy,
+  if (forced_plan == kPlanNone && small_m_applies(M, K)) {
+    return run_small_m(xq, is_packed(bits_a), s_x, s_x_kind, wq, is_packed(bits_w), s_w, bias, residual, ldr, residual_scale, M, N, K, act, y, ldy,
                        acc_debug, st);
   }
   const int8_t* a_codes = reinterpret_cast<const int8_t*>(xq);
-  if (bits_a == 4) {
+  if (is_packed(bits_a)) {
     rc = launch_unpack_int4(reinterpret_cast<const uint8_t*>(xq), M * K / 2, reinterpret_cast<int8_t*>(ws), st);
     if (rc != AQT_OK) return rc;
     a_codes = reinterpret_cast<const int8_t*>(ws);
     ws += round_up((size_t)M * (size_t)K, 256);
   }
   return qmatmul_i8a(a_codes, s_x, s_x_kind, wq, s_w, bias, residual, ldr, residual_scale, M, N, K, bits_a, bits_w, act, y,
-                     ldy, acc_debug, ws, st);
+                     ldy, acc_debug, ws, st, forced_plan);
+}
+
+int aqt_qmatmul(const void* xq, const float* s_x, int s_x_kind, const void* wq, const float* s_w, const float* bias,
+                const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K, int bits_a,
+                int bits_w, int act, float* y, int64_t ldy, int32_t* acc_debug, void* workspace, size_t workspace_bytes,
+                void* stream) {
+  return qmatmul_entry(xq, s_x, s_x_kind, wq, s_w, bias, residual, ldr, residual_scale, M, N, K, bits_a, bits_w, act, y, ldy, acc_debug,
+                       workspace, workspace_bytes, stream, kPlanNone);
+}
+
+int aqt_qmatmul_with_plan(const char* plan, const void* xq, const float* s_x, int s_x_kind, const void* wq, const float* s_w,
+                          const float* bias, const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N,
+                          int64_t K, int bits_a, int bits_w, int act, float* y, int64_t ldy, int32_t* acc_debug, void* workspace,
+                          size_t workspace_bytes, void* stream) {
+  const int id = gemm_plan_by_name(plan);
+  if (id == kPlanNone) return AQT_ERR_BADARG;
+  return qmatmul_entry(xq, s_x, s_x_kind, wq, s_w, bias, residual, ldr, residual_scale, M, N, K, bits_a, bits_w, act, y, ldy, acc_debug,
+                       workspace, workspace_bytes, stream, id);
+}
+
+int aqt_plan_qmatmul(int64_t M, int64_t N, int64_t K, int bits_a, int bits_w, int act, int float_kind, int sm_count_or_0,
+                     char* name_out, size_t name_bytes) {
+  if (name_out == nullptr || name_bytes == 0 || M <= 0 || N <= 0 || K <= 0 || !act_ok(act)) return AQT_ERR_BADARG;
+  if (!float_kind && (!bits_ok(bits_a) || !bits_ok(bits_w))) return AQT_ERR_BADARG;
+  int sms = sm_count_or_0;
+  if (sms <= 0) sms = sm_count();
+  if (sms <= 0) sms = kDefaultSms;
+  const char* name;
+  if (!float_kind && small_m_applies(M, K)) {
+    name = "small_m";
+  } else {
+    name = gemm_plan_name(plan_qgemm(GemmShape{M, N, float_kind ? 4 * K : K, act, float_kind ? 1 : 0, false}, sms));
+  }
+  if (strlen(name) + 1 > name_bytes) return AQT_ERR_BADARG;
+  memcpy(name_out, name, strlen(name) + 1);
+  return AQT_OK;
 }
 
 int aqt_qmatmul_requant(const void* xq, const float* s_x, int s_x_kind, const void* wq, const float* s_w, const float* bias,
@@ -299,7 +360,7 @@ int aqt_qmatmul_requant(const void* xq, const float* s_x, int s_x_kind, const vo
                         int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
   int rc = validate_matmul_shape(M, N, K, bits_a, bits_w, act, s_x_kind);
   if (rc != AQT_OK) return rc;
-  if (!bits_ok(bits_out) || (pack_out != 0 && pack_out != 1) || (pack_out == 1 && bits_out != 4)) return AQT_ERR_BADARG;
+  if (!quant_bits_ok(bits_out) || (pack_out != 0 && pack_out != 1) || (pack_out == 1 && bits_out != 4)) return AQT_ERR_BADARG;
   if (rounding != AQT_ROUND_HALF_UP_FLOOR && rounding != AQT_ROUND_NEAREST_EVEN) return AQT_ERR_BADARG;
   const int64_t n_out = is_glu(act) ? N / 2 : N;
   if (n_out % (pack_out ? 32 : 16) != 0) return AQT_ERR_BADARG;  // rows of codes keep a 16-byte pitch
@@ -331,7 +392,7 @@ int aqt_qmatmul_requant(const void* xq, const float* s_x, int s_x_kind, const vo
   }
 
   const int8_t* a_codes = reinterpret_cast<const int8_t*>(xq);
-  if (bits_a == 4) {
+  if (is_packed(bits_a)) {
     rc = launch_unpack_int4(reinterpret_cast<const uint8_t*>(xq), M * K / 2, reinterpret_cast<int8_t*>(ws), st);
     if (rc != AQT_OK) return rc;
     a_codes = reinterpret_cast<const int8_t*>(ws);
@@ -339,7 +400,7 @@ int aqt_qmatmul_requant(const void* xq, const float* s_x, int s_x_kind, const vo
   }
   const void* b_codes = wq;
   bool b_packed = false;
-  if (bits_w == 4) {
+  if (is_packed(bits_w)) {
     if (K % 32 == 0 && K <= 512) {  // the deep-K form (512 < K <= 1024) has no room to unpack in shared memory
       b_packed = true;
     } else {
@@ -364,7 +425,7 @@ int aqt_qmatmul_requant(const void* xq, const float* s_x, int s_x_kind, const vo
   p.K = (int)K;
   p.n_out = (int)n_out;
   p.tiles_m = p.tiles_n = p.k_blocks = 0;
-  p.small_acc = (K * (int64_t)(qmax_of(bits_a) + 1) * (qmax_of(bits_w) + 1) <= (1ll << 22)) ? 1 : 0;
+  p.small_acc = (K * (int64_t)(qmax_of(code_bits(bits_a)) + 1) * (qmax_of(code_bits(bits_w)) + 1) <= (1ll << 22)) ? 1 : 0;
   rp.q_out = nullptr;
   rp.s_out = s_out;
   rp.exchange = nullptr;
@@ -381,6 +442,7 @@ int aqt_linear_fwd(const float* x, int64_t ldx, const void* wq, const float* s_w
   int rc = validate_matmul_shape(M, N, K, bits_a, bits_w, act, a_scale_kind);
   if (rc != AQT_OK) return rc;
   if (rounding != AQT_ROUND_HALF_UP_FLOOR && rounding != AQT_ROUND_NEAREST_EVEN) return AQT_ERR_BADARG;
+  if (!quant_bits_ok(bits_a)) return AQT_ERR_BADARG;  // the width the activations are quantized to
   if (M == 0 || N == 0) return AQT_OK;
   const int64_t n_out = is_glu(act) ? N / 2 : N;
   if (x == nullptr || wq == nullptr || s_w == nullptr || y == nullptr) return AQT_ERR_BADARG;
@@ -439,6 +501,50 @@ int aqt_linear_fwd_host(const float* x, int x_on_host, const void* wq, const flo
   return AQT_OK;
 }
 
+int aqt_ffn_fwd(const float* x, int x_on_host, const void* w1q, const float* s_w1, const float* bias1, int bits_w1,
+                const void* w2q, const float* s_w2, const float* bias2, int bits_w2, int64_t M, int64_t d, int64_t ff,
+                int bits_a, int rounding, int act, float* y, int y_on_host, void* workspace, size_t workspace_bytes,
+                void* stream) {
+  if (M < 0 || d <= 0 || ff <= 0 || !quant_bits_ok(bits_a) || !bits_ok(bits_w1) || !bits_ok(bits_w2)) return AQT_ERR_BADARG;
+  if (act != AQT_ACT_NONE && act != AQT_ACT_SWISH) return AQT_ERR_BADARG;
+  if (rounding != AQT_ROUND_HALF_UP_FLOOR && rounding != AQT_ROUND_NEAREST_EVEN) return AQT_ERR_BADARG;
+  if (M == 0) return AQT_OK;
+  if (x == nullptr || y == nullptr || w1q == nullptr || w2q == nullptr || s_w1 == nullptr || s_w2 == nullptr) return AQT_ERR_BADARG;
+  const FfnLayout L = ffn_layout(M, d, ff, bits_w1, bits_w2);
+  if (workspace == nullptr || workspace_bytes < L.total) return AQT_ERR_WORKSPACE;
+  if (!is_aligned(workspace, 256)) return AQT_ERR_ALIGN;
+  int rc = check_device();
+  if (rc != AQT_OK) return rc;
+  if (!requant_applies(M, ff, d, act, false, false)) return AQT_ERR_UNSUPPORTED;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  const float* x_dev = x;
+  float* y_dev = y;
+  if (x_on_host) {
+    AQT_RETURN_IF_CUDA(cudaMemcpyAsync(ws + L.x, x, (size_t)M * d * 4, cudaMemcpyHostToDevice, st));
+    x_dev = reinterpret_cast<const float*>(ws + L.x);
+  }
+  if (y_on_host) y_dev = reinterpret_cast<float*>(ws + L.y);
+  int8_t* q1 = reinterpret_cast<int8_t*>(ws + L.q1);
+  float* s1 = reinterpret_cast<float*>(ws + L.s1);
+  int8_t* q2 = reinterpret_cast<int8_t*>(ws + L.q2);
+  float* s2 = reinterpret_cast<float*>(ws + L.s2);
+  const size_t mm_bytes = L.total - L.mm;
+  // Fig. 2 on the input rows; first matmul with the rows of u = act(W1 x) quantized in its epilogue
+  // (4-bit codes stay in int8 containers between the kernels); second matmul.
+  rc = aqt_quantize(x_dev, M, d, d, bits_a, AQT_AXIS_ROW, rounding, 0, q1, s1, stream);
+  if (rc != AQT_OK) return rc;
+  const int bits_mm = bits_a == 8 ? 8 : AQT_BITS_4_UNPACKED;
+  rc = aqt_qmatmul_requant(q1, s1, AQT_SCALE_ROW, w1q, s_w1, bias1, nullptr, 0, 0.0f, M, ff, d, bits_mm, bits_w1, act, bits_a, rounding, 0,
+                           q2, s2, nullptr, 0, ws + L.mm, mm_bytes, stream);
+  if (rc != AQT_OK) return rc;
+  rc = aqt_qmatmul(q2, s2, AQT_SCALE_ROW, w2q, s_w2, bias2, nullptr, 0, 0.0f, M, d, ff, bits_mm, bits_w2, AQT_ACT_NONE, y_dev, d, nullptr,
+                   ws + L.mm, mm_bytes, stream);
+  if (rc != AQT_OK) return rc;
+  if (y_on_host) AQT_RETURN_IF_CUDA(cudaMemcpyAsync(y, y_dev, (size_t)M * d * 4, cudaMemcpyDeviceToHost, st));
+  return AQT_OK;
+}
+
 int aqt_linear_fwd_weight_only(const float* x, int64_t ldx, const void* wq, const float* s_w, const float* bias,
                                const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K,
                                int bits_w, int precision, int act, float* y, int64_t ldy, void* workspace,
@@ -469,7 +575,7 @@ int aqt_linear_fwd_weight_only(const float* x, int64_t ldx, const void* wq, cons
   if (precision == AQT_FLOAT_TF32X2) {
     // x = hi + lo with hi a tf32 value: one matmul over [hi | lo] against [w | w]
     float* x2 = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace) + round_up((size_t)N * (size_t)K * 8, 256));
-    rc = launch_codes_to_float_twice(wq, bits_w == 4, N, K, w_f, st);
+    rc = launch_codes_to_float_twice(wq, is_packed(bits_w), N, K, w_f, st);
     if (rc != AQT_OK) return rc;
     rc = launch_split_hi_lo(x, ldx, M, K, x2, st);
     if (rc != AQT_OK) return rc;
@@ -477,7 +583,7 @@ int aqt_linear_fwd_weight_only(const float* x, int64_t ldx, const void* wq, cons
     k_mm = 2 * K;
     a_pitch = 8 * K;
   } else {
-    rc = launch_codes_to_float(wq, bits_w == 4, N * K, w_f, st);
+    rc = launch_codes_to_float(wq, is_packed(bits_w), N * K, w_f, st);
     if (rc != AQT_OK) return rc;
   }
   GemmParams p;
@@ -534,7 +640,7 @@ int aqt_linear_bwd(const float* dy, int64_t lddy, const void* xq, const float* s
   if (dx != nullptr) {
     // dx = dy . (s_w wq): rows m, columns k, contraction n
     float* wt = reinterpret_cast<float*>(ws + L.wt);
-    rc = launch_transpose_scale_codes(wq, bits_w == 4, s_w, true, N, K, wt, N, N, K, st);
+    rc = launch_transpose_scale_codes(wq, is_packed(bits_w), s_w, true, N, K, wt, N, N, K, st);
     if (rc != AQT_OK) return rc;
     rc = float_gemm_nt(dy, lddy, wt, M, K, N, ones, dx, lddx, st);
     if (rc != AQT_OK) return rc;
@@ -547,7 +653,7 @@ int aqt_linear_bwd(const float* dy, int64_t lddy, const void* xq, const float* s
     rc = launch_transpose_f32(dy, lddy, M, N, dyt, m_pad, L.chunk, L.n_pad, dbias != nullptr ? reinterpret_cast<float*>(ws + L.partial) : nullptr,
                               dbias, st);
     if (rc != AQT_OK) return rc;
-    rc = launch_transpose_scale_codes(xq, bits_a == 4, s_x, s_x_kind == AQT_SCALE_ROW, M, K, xt, m_pad, L.chunk, K, st);
+    rc = launch_transpose_scale_codes(xq, is_packed(bits_a), s_x, s_x_kind == AQT_SCALE_ROW, M, K, xt, m_pad, L.chunk, K, st);
     if (rc != AQT_OK) return rc;
     if (L.batches == 1) {
       rc = float_gemm_nt(dyt, L.chunk, xt, N, K, L.chunk, ones, dw, lddw, st);
@@ -621,6 +727,33 @@ int aqt_selftest_bounded_wait(uint64_t limit_ns, int* gave_up_dev, void* stream)
   int rc = check_device();
   if (rc != AQT_OK) return rc;
   bounded_wait_selftest_kernel<<<1, 64, 0, reinterpret_cast<cudaStream_t>(stream)>>>(limit_ns, gave_up_dev);
+  return AQT_LAUNCH_STATUS();
+}
+
+// Nothing but special-function work: eight independent chains of 2^x and reciprocal per thread.
+__global__ void __launch_bounds__(256) sfu_rate_kernel(int iterations, float* sink) {
+  float v[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) v[j] = 0.25f + 0.01f * (float)((threadIdx.x + j) & 15);
+  for (int i = 0; i < iterations; ++i) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = rcp_approx(1.0f + ex2_approx(v[j]));
+  }
+  float acc = 0.0f;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) acc += v[j];
+  if (acc == 12345.0f) *sink = acc;  // never true: keeps the chains alive
+}
+
+int aqt_selftest_sfu_rate(int iterations, float* sink_dev, int64_t* ops_out, void* stream) {
+  if (iterations <= 0 || iterations > (1 << 20) || sink_dev == nullptr || ops_out == nullptr) return AQT_ERR_BADARG;
+  int rc = check_device();
+  if (rc != AQT_OK) return rc;
+  const int sms = sm_count();
+  if (sms <= 0) return AQT_ERR_CUDA;
+  const int ctas = sms * 8;
+  sfu_rate_kernel<<<ctas, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(iterations, sink_dev);
+  *ops_out = (int64_t)ctas * 256 * iterations * 16;
   return AQT_LAUNCH_STATUS();
 }
 

@@ -6,6 +6,8 @@
 #include <stdio.h>
 #include <stdlib.h>
 
+#include <atomic>
+
 #include "../../include/aqt.h"
 
 namespace aqt {
@@ -36,6 +38,66 @@ inline int cuda_fail(cudaError_t e, const char* what, int line) {
 inline int launch_status(int line) {
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? AQT_OK : cuda_fail(e, "kernel launch", line);
+}
+
+// Properties of the current device, looked up once per device ordinal.  Host threads may race on
+// the first lookup; both then store the same values.
+constexpr int kMaxDevices = 64;
+struct DeviceInfo {
+  int ordinal;
+  int sms;       // multiprocessors
+  int cc_major;  // compute capability, major
+};
+inline int current_device_info(DeviceInfo* out) {
+  static std::atomic<int> sms[kMaxDevices];
+  static std::atomic<int> cc[kMaxDevices];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return AQT_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return AQT_ERR_UNSUPPORTED;
+  int n = sms[dev].load(std::memory_order_acquire);
+  if (n == 0) {
+    int major = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return AQT_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return AQT_ERR_CUDA;
+    cc[dev].store(major, std::memory_order_relaxed);
+    sms[dev].store(n, std::memory_order_release);
+  }
+  out->ordinal = dev;
+  out->sms = n;
+  out->cc_major = cc[dev].load(std::memory_order_relaxed);
+  return AQT_OK;
+}
+// Multiprocessors of the current device; 0 if there is none (callers that only plan then assume
+// the 148 of the one part this library is built for).
+inline int sm_count() {
+  DeviceInfo d;
+  return current_device_info(&d) == AQT_OK ? d.sms : 0;
+}
+constexpr int kDefaultSms = 148;
+
+// Opt a kernel into `bytes` of dynamic shared memory, once per device (the attribute belongs to
+// the function as loaded on one device).  `done` is one mask per kernel instantiation.
+template <class Kernel>
+inline int ensure_dynamic_smem(Kernel kernel, int bytes, std::atomic<uint64_t>& done) {
+  DeviceInfo d;
+  int rc = current_device_info(&d);
+  if (rc != AQT_OK) return rc;
+  const uint64_t bit = 1ull << d.ordinal;
+  if (done.load(std::memory_order_acquire) & bit) return AQT_OK;
+  AQT_RETURN_IF_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  done.fetch_or(bit, std::memory_order_release);
+  return AQT_OK;
+}
+
+// Overrides of the kernel choice for tuning runs.  They exist only in builds made with
+// -DAQT_TUNING; the shipped library never reads the environment to pick a kernel.
+inline const char* tuning_env(const char* name) {
+#ifdef AQT_TUNING
+  return getenv(name);
+#else
+  (void)name;
+  return nullptr;
+#endif
 }
 
 inline bool is_aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }

@@ -639,7 +639,7 @@ static size_t requant_exchange_bytes(int64_t M, int64_t N) {
 // True if this kernel takes the call: K <= 512; NONE / Swish in every form, the GLU forms when
 // only int8 codes and scales are asked for (no fp32 output, hence no residual, no nibble packing).
 static bool requant_applies(int64_t M, int64_t N, int64_t K, int act, bool with_y, bool pack_out) {
-  const int sms = sm_count() > 0 ? sm_count() : 148;
+  const int sms = sm_count() > 0 ? sm_count() : kDefaultSms;
   if (!(M > 0 && ceil_div(N, 128) <= sms)) return false;
   const bool glu = !(act == AQT_ACT_NONE || act == AQT_ACT_SWISH);
   if (ceil_div(K, kBK) <= kWsMaxKBlocks) return !glu || (!with_y && !pack_out);
@@ -680,11 +680,9 @@ static int launch_requant_inst(const int8_t* a, const void* b, void* q_out, floa
     }
   }
   auto kernel = qgemm_requant_kernel<BPACK, SMALL, WITH_Y, ROUNDING, PACK_OUT, GLU, DEEP>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    AQT_RETURN_IF_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
-    attr_set = true;
-  }
+  static std::atomic<uint64_t> smem_opted_in{0};
+  rc = ensure_dynamic_smem(kernel, Cfg::kSmemBytes, smem_opted_in);
+  if (rc != AQT_OK) return rc;
   int groups = sms / p.tiles_n;
   if (groups > p.tiles_m) groups = p.tiles_m;
   cudaLaunchConfig_t cfg = {};

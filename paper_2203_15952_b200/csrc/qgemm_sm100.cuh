@@ -21,6 +21,7 @@
 #pragma once
 
 #include <cuda.h>
+#include <string.h>
 
 #include "aqt_common.cuh"
 #include "pack.cuh"
@@ -53,7 +54,12 @@ struct GemmCfg {
   static constexpr int kStageBytes = WS ? kABytes : kABytes + kBBytes;
   static constexpr int kResidentBytes = WS ? kWsMaxKBlocks * kBBytes : 0;
   static constexpr int kStages = STAGES;
-  static constexpr int kTmemCols = 2 * BN;  // two accumulator buffers; a power of two >= 32
+  // Two accumulator buffers, so that the epilogue of a tile overlaps the next tile's MMAs; a tile
+  // 512 columns wide (CTA pairs only) fills tensor memory by itself and has one.
+  static_assert(BN <= 256 || (BN == 512 && CTA2), "512-column tiles are a form of the CTA-pair kernel");
+  static constexpr int kAccBufs = BN == 512 ? 1 : 2;
+  static constexpr int kMmaN = BN > 256 ? 256 : BN;  // columns one tcgen05.mma covers
+  static constexpr int kTmemCols = kAccBufs * BN;    // a power of two >= 32
   // Output staging buffers per warp: two let a warp fill one while the bulk store of the other is
   // still being read; with sixteen warps each warp stores once per tile and one is enough.
   // "Lean" epilogue: where the ring, two staging buffers per warp and the scale slabs together
@@ -451,6 +457,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   static_assert(!BPACK || WS, "packed weights are unpacked into the resident slab");
   constexpr bool TF32 = (ACCK == kAccFloat);  // float operands: no activation scale, accumulators are binary32
   static_assert(!(TF32 && (BPACK || DEBUG)), "the float kind reads expanded weights and has no integer accumulators to dump");
+  static_assert(!(TF32 && BN == 512), "512-column tiles exist for the 8-bit kind only");
   const uint32_t pair_rank = CTA2 ? cluster_ctarank() : 0u;  // 0 = leader: issues the MMAs, owns the barriers the pair shares
   const int row_in_tile = (int)pair_rank * kBM;               // this CTA's first row inside the tile
 
@@ -574,7 +581,14 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             // its half of the weight rows (leader: first half / values, peer: second half / gates).
             if (pair_rank == 0) mbar_arrive_expect_tx(bar, 2 * Cfg::kStageBytes);
             tma_load_2d_pair(stage, &tm_a, kb * kBK, tm * TILE_M + row_in_tile, bar);
-            tma_load_2d_pair(stage + Cfg::kABytes, &tm_b, kb * kBK, pair_rank == 0 ? row0 : row1, bar);
+            if (BN == 512) {
+              // two MMAs of 256 columns per k-step: this CTA supplies 128 weight rows to each
+              const int r = tn * BN + (int)pair_rank * 128;
+              tma_load_2d_pair(stage + Cfg::kABytes, &tm_b, kb * kBK, r, bar);
+              tma_load_2d_pair(stage + Cfg::kABytes + 128 * kBK, &tm_b, kb * kBK, r + 256, bar);
+            } else {
+              tma_load_2d_pair(stage + Cfg::kABytes, &tm_b, kb * kBK, pair_rank == 0 ? row0 : row1, bar);
+            }
             continue;
           }
           mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
@@ -590,13 +604,13 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && pair_rank == 0) {
-      constexpr uint32_t idesc = TF32 ? idesc_tf32(BN, TILE_M) : idesc_i8(BN, TILE_M);
+      constexpr uint32_t idesc = TF32 ? idesc_tf32(Cfg::kMmaN, TILE_M) : idesc_i8(Cfg::kMmaN, TILE_M);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       if (WS) ok = mbar_wait(smem_u32(BPACK ? &b_ready_bar : &b_loaded_bar), 0, &abort_flag, t_start);
       int tm, tn;
       for (int i = 0; ok && tile_at<WS, CTA2>(p, i, tm, tn); ++i, ++tcount) {
-        const uint32_t buf = tcount & 1, aph = (tcount >> 1) & 1;
+        const uint32_t buf = tcount % Cfg::kAccBufs, aph = (tcount / Cfg::kAccBufs) & 1;
         if (!mbar_wait(smem_u32(&tmem_empty_bar[buf]), aph ^ 1, &abort_flag, t_start)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * BN;
@@ -617,6 +631,8 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             } else {
               if (CTA2) tc_mma_i8_pair(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, accumulate);
               else tc_mma_i8(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, accumulate);
+              if (BN == 512)  // columns 256 .. 511: the second 128 weight rows of each CTA's stage (16 KB further on)
+                tc_mma_i8_pair(d_tmem + 256, a_desc + 2 * kk, b_desc + (128 * kBK >> 4) + 2 * kk, idesc, accumulate);
             }
           }
           // stage reusable (in both CTAs of a pair) once these MMAs have read it
@@ -691,7 +707,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     }
 
     for (int i = 0; ok && tile_at<WS, CTA2>(p, i, tm, tn); ++i) {
-      const uint32_t buf = i & 1, aph = (i >> 1) & 1;
+      const uint32_t buf = i % Cfg::kAccBufs, aph = (i / Cfg::kAccBufs) & 1;
       const int out0 = tn * out_cols_tile;  // first output column of the tile
       const int row0_warp = tm * TILE_M + row_in_tile + quad * 32;  // first output row of this warp
       const int m = row0_warp + lane;
@@ -956,15 +972,6 @@ static int make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, const void* bas
   return r == CUDA_SUCCESS ? AQT_OK : AQT_ERR_CUDA;
 }
 
-static int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
-  }
-  return n;
-}
-
 // Rounds of a persistent grid over the tiles: fewer rounds of fuller waves win.
 static int pick_bn(int64_t M, int64_t N, bool glu, int sms) {
   const int64_t tiles_m = ceil_div(M, kBM);
@@ -1000,6 +1007,8 @@ static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t l
     const bool glu = (p.act == AQT_ACT_GLU) || (p.act == AQT_ACT_GLU_SWISH);
     if ((glu ? BN / 2 : BN) / 32 / (EW / 4) < 1) return AQT_ERR_UNSUPPORTED;  // a warp without columns would never release TMEM
     if (WS && (p.k_blocks > kWsMaxKBlocks || p.tiles_n > sms)) return AQT_ERR_UNSUPPORTED;
+    if (BN == 512 && glu) return AQT_ERR_UNSUPPORTED;  // value and gate halves are not laid out for two MMAs per step
+    if (CTA2 && p.M <= kBM) return AQT_ERR_UNSUPPORTED;
   }
   CUtensorMap tm_a, tm_b, tm_y, tm_r;
   int rc = make_map_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, a, (uint64_t)p.M, (uint64_t)p.K,
@@ -1008,8 +1017,8 @@ static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t l
   if (BPACK) {
     rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, b, (uint64_t)p.N, (uint64_t)p.K / 2, (uint64_t)p.K / 2, BN / 2, 64, 0);
   } else {
-    rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, b, (uint64_t)(p.b_rows != 0 ? p.b_rows : p.N), (uint64_t)p.K, (uint64_t)p.K, BN / 2,
-                     kBK);
+    rc = make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, b, (uint64_t)(p.b_rows != 0 ? p.b_rows : p.N), (uint64_t)p.K, (uint64_t)p.K,
+                     BN == 512 ? 128 : BN / 2, kBK);
   }
   if (rc != AQT_OK) return rc;
   if (p.batch_tiles_m > 0 && (WS || CTA2)) return AQT_ERR_UNSUPPORTED;
@@ -1024,11 +1033,9 @@ static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t l
     tm_r = tm_y;  // never dereferenced
   }
   auto kernel = qgemm_i8_kernel<BN, STAGES, EW, WS, BPACK, ACCK, DEBUG, CTA2>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    AQT_RETURN_IF_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
-    attr_set = true;
-  }
+  static std::atomic<uint64_t> smem_opted_in{0};
+  rc = ensure_dynamic_smem(kernel, Cfg::kSmemBytes, smem_opted_in);
+  if (rc != AQT_OK) return rc;
   const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
   unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
   if (WS && (int)grid < p.tiles_n) grid = (unsigned)p.tiles_n;  // every n-tile needs an owner
@@ -1058,7 +1065,7 @@ static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t l
 template <int BN, int STAGES, int EW, bool WS, bool BPACK, bool CTA2 = false>
 static int launch_qgemm_cfg(const int8_t* a, const void* b, float* y, int64_t ldy, const GemmParams& p, cudaStream_t st) {
   if (p.kind == 1) {
-    if constexpr (!BPACK) {
+    if constexpr (!BPACK && BN != 512) {
       if (p.acc_debug == nullptr) return launch_qgemm_inst<BN, STAGES, EW, WS, false, kAccFloat, false, CTA2>(a, b, y, ldy, p, st);
     }
     return AQT_ERR_UNSUPPORTED;
@@ -1068,72 +1075,114 @@ static int launch_qgemm_cfg(const int8_t* a, const void* b, float* y, int64_t ld
   return launch_qgemm_inst<BN, STAGES, EW, WS, BPACK, kAccInt32, false, CTA2>(a, b, y, ldy, p, st);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Choice of the kernel configuration ("plan") for a shape, and the launch of a plan
+
+// Every configuration of the kernel template that the library instantiates.
+enum GemmPlan {
+  kPlanNone = 0,
+  kPlanWs128E16,        // weight stationary (K <= 512), 128-column tiles, sixteen epilogue warps
+  kPlanWs128E8,         // the same with eight epilogue warps: the GLU forms (64 output columns per tile)
+  kPlanStream256S3E16,  // both operands streamed, 256-column tiles, shallow K
+  kPlanStream256S4E4,   //   deep K: four-warp epilogue, deeper ring
+  kPlanStream256S4E8,   //   float kind
+  kPlanStream128S4E16,
+  kPlanStream128S6E4,
+  kPlanStream128S4E8,   //   GLU at width 128
+  kPlanStream64S5E8,
+  kPlanStream64S8E4,
+  kPlanPair256S4E8,     // CTA pairs on 256-row tiles
+  kPlanPair256S6E4,
+  kPlanPair128S6E8,
+  kPlanPair128S8E4,
+  kPlanPair512S3E16,    // CTA pairs on 256 x 512 tiles, one accumulator buffer (few, deep tiles)
+  kPlanCount
+};
+static const char* const kGemmPlanNames[kPlanCount] = {
+    "none",          "ws128e16",      "ws128e8",       "stream256s3e16", "stream256s4e4", "stream256s4e8",
+    "stream128s4e16", "stream128s6e4", "stream128s4e8", "stream64s5e8",   "stream64s8e4",  "pair256s4e8",
+    "pair256s6e4",   "pair128s6e8",   "pair128s8e4",   "pair512s3e16"};
+static const char* gemm_plan_name(int plan) { return plan > 0 && plan < kPlanCount ? kGemmPlanNames[plan] : kGemmPlanNames[0]; }
+static int gemm_plan_by_name(const char* name) {
+  if (name == nullptr) return kPlanNone;
+  for (int i = 1; i < kPlanCount; ++i)
+    if (strcmp(name, kGemmPlanNames[i]) == 0) return i;
+  return kPlanNone;
+}
+
+// What the choice depends on.  K in bytes of contraction per operand row (see GemmParams).
+struct GemmShape {
+  int64_t M, N, K;
+  int act;
+  int kind;      // 0: 8-bit codes, 1: float kind
+  bool batched;  // stacked batches: streaming kernel, one CTA per tile
+};
+
 // True if the weight-stationary kernel takes this shape (and can therefore unpack 4-bit weights itself).
-static bool qgemm_uses_ws(int64_t N, int64_t K) {
-  static const char* off = getenv("AQT_NO_WS");  // tuning aid: force the streaming kernel
-  if (off != nullptr) return false;
-  const int sms = sm_count() > 0 ? sm_count() : 148;
+static bool qgemm_uses_ws(int64_t N, int64_t K, int sms) {
+  if (tuning_env("AQT_NO_WS") != nullptr) return false;  // tuning builds: force the streaming kernel
   return ceil_div(K, kBK) <= kWsMaxKBlocks && ceil_div(N, 128) <= sms;
 }
 
-// a: int8 [M, K] codes.  b: int8 [N, K] codes, or -- only if b_packed and qgemm_uses_ws(N, K) --
-// packed nibbles [N, K/2].  All dense, 16-byte aligned.
-static int launch_qgemm(const int8_t* a, const void* b, bool b_packed, float* y, int64_t ldy, const GemmParams& p, cudaStream_t st) {
-  const bool glu = (p.act == AQT_ACT_GLU) || (p.act == AQT_ACT_GLU_SWISH);
-  const bool batched = p.batch_tiles_m > 0;  // streaming kernel, one CTA per tile
-  if (!batched && qgemm_uses_ws(p.N, p.K)) {
-    // tile width 128; a GLU tile has 64 output columns, i.e. two chunks per lane quadrant
-    if (glu) return b_packed ? launch_qgemm_cfg<128, 6, 8, true, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 6, 8, true, false>(a, b, y, ldy, p, st);
-    return b_packed ? launch_qgemm_cfg<128, 6, 16, true, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 6, 16, true, false>(a, b, y, ldy, p, st);
-  }
-  if (b_packed) return AQT_ERR_UNSUPPORTED;
+// sms: multiprocessors of the device the launch will go to.
+static int plan_qgemm(const GemmShape& g, int sms) {
+  const bool glu = (g.act == AQT_ACT_GLU) || (g.act == AQT_ACT_GLU_SWISH);
+  const bool f32 = g.kind == 1;
+  if (!g.batched && qgemm_uses_ws(g.N, g.K, sms)) return glu ? kPlanWs128E8 : kPlanWs128E16;  // a GLU tile has 64 output columns
   // "Deep" configuration (four-warp epilogue, longest ring): pays off when K is deep AND every
   // CTA walks many tiles; with few tiles per CTA the exposed epilogue of the last tile costs more
   // than the extra ring stages gain (measured at M = 12 800 .. 25 600).
-  const int sms_ = sm_count() > 0 ? sm_count() : 148;
-  bool deep_k = p.K >= 2048 && !glu && ceil_div(p.M, kBM) * ceil_div(p.N, 256) >= 4 * sms_;
+  bool deep_k = g.K >= 2048 && !glu && ceil_div(g.M, kBM) * ceil_div(g.N, 256) >= 4 * sms;
   // Float kind: a k-block takes as many tensor-core clocks as an 8-bit one but holds a quarter of
   // the elements, so every shape is "deep" in bytes and the epilogue is a small part of a tile
   // unless it evaluates an activation (measured: the four-warp epilogue wins at 12 800 x 512 x
   // 2048 and 65 536 x 1024 x 4096 without activation, loses by 20-40 % with Swish).
-  const bool f32 = p.kind == 1;
-  if (f32) deep_k = p.act == AQT_ACT_NONE && p.K >= 8192;
-  static const char* deep_env = getenv("AQT_DEEP");  // tuning aid: 0 / 1 overrides the deep-K choice
-  if (deep_env != nullptr && !glu) deep_k = atoi(deep_env) != 0;
-  static const char* no_pairs = getenv("AQT_NO_PAIRS");  // tuning aid: one CTA per tile
+  if (f32) deep_k = g.act == AQT_ACT_NONE && g.K >= 8192;
+  if (const char* e = tuning_env("AQT_DEEP")) {
+    if (!glu) deep_k = atoi(e) != 0;
+  }
+  const int pairs = sms / 2;
   // Pairs pay off only for deep K and at least two full rounds of pair tiles (measured: +4 % at
   // 65 536 x 1024 x 4096 with the deep configuration, +9 % at 25 600 x 512 x 2048 with the
   // eight-warp epilogue, no gain at M = 12 800 or at K = 1024); everything else takes one CTA per tile.
   // (the 8-bit kind's GLU shapes are faster on single CTAs; the float kind's gain 3 % on pairs)
-  const bool two_rounds_of_pairs = (!glu || f32) && ceil_div(p.M, 2 * kBM) * ceil_div(p.N, 256) >= 2 * (sms_ / 2);
+  const bool two_rounds_of_pairs = (!glu || f32) && ceil_div(g.M, 2 * kBM) * ceil_div(g.N, 256) >= 2 * pairs;
   // (float kind, measured: pairs win 6-10 % at M >= 25 600, lose 10 % at 12 800 x 2048 x 512)
-  const bool pairs_ok = f32 ? (two_rounds_of_pairs && p.M >= 2 * kBM * (sms_ / 2)) : (deep_k || (p.K >= 2048 && two_rounds_of_pairs));
-  if (!batched && no_pairs == nullptr && (pairs_ok || getenv("AQT_FORCE_PAIRS") != nullptr) && p.M > kBM) {
+  bool pairs_ok = f32 ? (two_rounds_of_pairs && g.M >= 2 * kBM * pairs) : (deep_k || (g.K >= 2048 && two_rounds_of_pairs));
+  if (tuning_env("AQT_NO_PAIRS") != nullptr) pairs_ok = false;
+  if (tuning_env("AQT_FORCE_PAIRS") != nullptr) pairs_ok = true;
+  if (!g.batched && g.M > kBM) {
+    // Few, deep tiles (K >= 2048, all of N within one or two 512-column tiles, at most one round of
+    // 256 x 512 tiles over the pairs): each pair takes one whole tile, so the activations are read
+    // once, the weights once per 256 rows, and no SM waits for a second, mostly empty round.
+    bool wide = !f32 && !glu && g.K >= 2048 && g.N % 512 == 0 && ceil_div(g.M, 2 * kBM) * (g.N / 512) <= pairs;
+    if (const char* e = tuning_env("AQT_WIDE_PAIRS")) wide = !f32 && !glu && atoi(e) != 0;
+    if (wide) return kPlanPair512S3E16;
+  }
+  if (!g.batched && pairs_ok && g.M > kBM) {
     // CTA pairs on 256-row tiles; width by the number of rounds over the pairs
-    const int pairs = (sm_count() > 0 ? sm_count() : 148) / 2;
-    const int64_t tiles_m2 = ceil_div(p.M, 2 * kBM);
-    const double cost256 = (double)ceil_div(tiles_m2 * ceil_div(p.N, 256), pairs) * (256 + 24);
-    const double cost128 = (double)ceil_div(tiles_m2 * ceil_div(p.N, 128), pairs) * (128 + 24);
+    const int64_t tiles_m2 = ceil_div(g.M, 2 * kBM);
+    const double cost256 = (double)ceil_div(tiles_m2 * ceil_div(g.N, 256), pairs) * (256 + 24);
+    const double cost128 = (double)ceil_div(tiles_m2 * ceil_div(g.N, 128), pairs) * (128 + 24);
     int bn2 = cost256 <= cost128 ? 256 : 128;
-    static const char* force2 = getenv("AQT_BN");
-    if (force2 != nullptr && (atoi(force2) == 128 || atoi(force2) == 256)) bn2 = atoi(force2);
+    if (const char* e = tuning_env("AQT_BN")) {
+      if (atoi(e) == 128 || atoi(e) == 256) bn2 = atoi(e);
+    }
     // The four-warp epilogue / deeper ring pays off for pairs only from K = 4096 bytes (measured at
     // 65 536 x 1024 x 4096: 2753 vs 2671 TOPS burst, equal sustained; float kind 801 vs 752
     // TFLOP/s); at K = 2048 the eight-warp epilogue with four stages is 20-27 % faster (41.1 vs
     // 52.3 us at 37 888 x 512 x 2048, where the deep-K rule first applies; 83.1 vs 104.9 us at 65 536).
-    static const char* deep_pairs = getenv("AQT_DEEP_PAIRS");  // tuning aid: 0 / 1 overrides the choice
-    const bool dp = deep_pairs != nullptr ? atoi(deep_pairs) != 0 : (deep_k && p.K >= 4096);
-    if (bn2 == 256) return dp ? launch_qgemm_cfg<256, 6, 4, false, false, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<256, 4, 8, false, false, true>(a, b, y, ldy, p, st);
-    return dp ? launch_qgemm_cfg<128, 8, 4, false, false, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 6, 8, false, false, true>(a, b, y, ldy, p, st);
+    bool dp = deep_k && g.K >= 4096;
+    if (const char* e = tuning_env("AQT_DEEP_PAIRS")) dp = atoi(e) != 0;
+    if (bn2 == 256) return dp ? kPlanPair256S6E4 : kPlanPair256S4E8;
+    return dp ? kPlanPair128S8E4 : kPlanPair128S6E8;
   }
-  int bn = pick_bn(p.M, p.N, glu, sm_count() > 0 ? sm_count() : 148);
+  int bn = pick_bn(g.M, g.N, glu, sms);
   // operand bytes per output are four times those of the 8-bit kind: the widest tile wins whenever it
   // still gives every SM a tile (a weight gradient has few, very deep tiles and takes narrow ones)
-  if (f32 && p.N >= 256 && ceil_div(p.M, kBM) * ceil_div(p.N, 256) >= sms_) bn = 256;
-  // tuning aid: AQT_BN=64|128|256 in the environment overrides the tile-width heuristic
-  static const char* force = getenv("AQT_BN");
-  if (force != nullptr) {
-    const int v = atoi(force);
+  if (f32 && g.N >= 256 && ceil_div(g.M, kBM) * ceil_div(g.N, 256) >= sms) bn = 256;
+  if (const char* e = tuning_env("AQT_BN")) {
+    const int v = atoi(e);
     if ((v == 64 && !glu) || v == 128 || v == 256) bn = v;
   }
   // Deep K: operand loads bound the tile, so the ring gets the shared memory and four warps run
@@ -1143,13 +1192,87 @@ static int launch_qgemm(const int8_t* a, const void* b, bool b_packed, float* y,
   // (measured 2-10 % faster than three stages / sixteen warps and than four stages / four warps:
   // 59.8 vs 62.4 us at 12 800 x 2048 x 512 Swish, 362 vs 398 us at 65 536 x 2048 x 1024 GLU).  The
   // 8-bit kind loses with it wherever the epilogue evaluates an activation or M is small.
-  if (bn == 256 && f32) return launch_qgemm_cfg<256, 4, 8, false, false>(a, b, y, ldy, p, st);
-  if (bn == 256) return deep_k ? launch_qgemm_cfg<256, 4, 4, false, false>(a, b, y, ldy, p, st) : launch_qgemm_cfg<256, 3, 16, false, false>(a, b, y, ldy, p, st);
+  if (bn == 256 && f32) return kPlanStream256S4E8;
+  if (bn == 256) return deep_k ? kPlanStream256S4E4 : kPlanStream256S3E16;
   // every epilogue warp needs at least one 32-column chunk: a GLU tile of width 128 has only
   // 64 output columns, i.e. two chunks per lane quadrant
-  if (bn == 128 && glu) return launch_qgemm_cfg<128, 4, 8, false, false>(a, b, y, ldy, p, st);
-  if (bn == 128) return deep_k ? launch_qgemm_cfg<128, 6, 4, false, false>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 4, 16, false, false>(a, b, y, ldy, p, st);
-  return deep_k ? launch_qgemm_cfg<64, 8, 4, false, false>(a, b, y, ldy, p, st) : launch_qgemm_cfg<64, 5, 8, false, false>(a, b, y, ldy, p, st);
+  if (bn == 128 && glu) return kPlanStream128S4E8;
+  if (bn == 128) return deep_k ? kPlanStream128S6E4 : kPlanStream128S4E16;
+  return deep_k ? kPlanStream64S8E4 : kPlanStream64S5E8;
+}
+
+// Tile width and epilogue warps of each plan (same order as GemmPlan).
+static const int kGemmPlanBn[kPlanCount] = {0, 128, 128, 256, 256, 256, 128, 128, 128, 64, 64, 256, 256, 128, 128, 512};
+static const int kGemmPlanEw[kPlanCount] = {0, 16, 8, 16, 4, 8, 16, 4, 8, 8, 4, 8, 4, 8, 4, 16};
+
+// True if `plan` can run this shape at all (used when a caller names the plan itself).
+static bool gemm_plan_takes(int plan, const GemmShape& g, int sms) {
+  if (plan <= kPlanNone || plan >= kPlanCount) return false;
+  const bool glu = (g.act == AQT_ACT_GLU) || (g.act == AQT_ACT_GLU_SWISH);
+  const bool ws = plan == kPlanWs128E16 || plan == kPlanWs128E8;
+  const bool pair = plan >= kPlanPair256S4E8 && plan <= kPlanPair512S3E16;
+  if (ws && (g.batched || ceil_div(g.K, kBK) > kWsMaxKBlocks || ceil_div(g.N, 128) > sms)) return false;
+  if (pair && (g.batched || g.M <= kBM)) return false;
+  if (plan == kPlanPair512S3E16 && (glu || g.kind != 0)) return false;
+  // every epilogue warp needs at least one 32-column chunk of the tile's output columns
+  const int out_cols = glu ? kGemmPlanBn[plan] / 2 : kGemmPlanBn[plan];
+  return out_cols / 32 / (kGemmPlanEw[plan] / 4) >= 1;
+}
+
+// a: int8 [M, K] codes.  b: int8 [N, K] codes, or -- only if b_packed and a weight-stationary plan --
+// packed nibbles [N, K/2].  All dense, 16-byte aligned.
+static int launch_qgemm_plan(int plan, const int8_t* a, const void* b, bool b_packed, float* y, int64_t ldy, const GemmParams& p,
+                             cudaStream_t st) {
+  switch (plan) {
+    case kPlanWs128E16:
+      return b_packed ? launch_qgemm_cfg<128, 6, 16, true, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 6, 16, true, false>(a, b, y, ldy, p, st);
+    case kPlanWs128E8:
+      return b_packed ? launch_qgemm_cfg<128, 6, 8, true, true>(a, b, y, ldy, p, st) : launch_qgemm_cfg<128, 6, 8, true, false>(a, b, y, ldy, p, st);
+    default: break;
+  }
+  if (b_packed) return AQT_ERR_UNSUPPORTED;
+  switch (plan) {
+    case kPlanStream256S3E16: return launch_qgemm_cfg<256, 3, 16, false, false>(a, b, y, ldy, p, st);
+    case kPlanStream256S4E4: return launch_qgemm_cfg<256, 4, 4, false, false>(a, b, y, ldy, p, st);
+    case kPlanStream256S4E8: return launch_qgemm_cfg<256, 4, 8, false, false>(a, b, y, ldy, p, st);
+    case kPlanStream128S4E16: return launch_qgemm_cfg<128, 4, 16, false, false>(a, b, y, ldy, p, st);
+    case kPlanStream128S6E4: return launch_qgemm_cfg<128, 6, 4, false, false>(a, b, y, ldy, p, st);
+    case kPlanStream128S4E8: return launch_qgemm_cfg<128, 4, 8, false, false>(a, b, y, ldy, p, st);
+    case kPlanStream64S5E8: return launch_qgemm_cfg<64, 5, 8, false, false>(a, b, y, ldy, p, st);
+    case kPlanStream64S8E4: return launch_qgemm_cfg<64, 8, 4, false, false>(a, b, y, ldy, p, st);
+    case kPlanPair256S4E8: return launch_qgemm_cfg<256, 4, 8, false, false, true>(a, b, y, ldy, p, st);
+    case kPlanPair256S6E4: return launch_qgemm_cfg<256, 6, 4, false, false, true>(a, b, y, ldy, p, st);
+    case kPlanPair128S6E8: return launch_qgemm_cfg<128, 6, 8, false, false, true>(a, b, y, ldy, p, st);
+    case kPlanPair128S8E4: return launch_qgemm_cfg<128, 8, 4, false, false, true>(a, b, y, ldy, p, st);
+    case kPlanPair512S3E16: return launch_qgemm_cfg<512, 3, 16, false, false, true>(a, b, y, ldy, p, st);
+    default: return AQT_ERR_UNSUPPORTED;
+  }
+}
+
+static GemmShape gemm_shape_of(const GemmParams& p) {
+  GemmShape g;
+  g.M = p.M;
+  g.N = p.N;
+  g.K = p.K;
+  g.act = p.act;
+  g.kind = p.kind;
+  g.batched = p.batch_tiles_m > 0;
+  return g;
+}
+
+// forced_plan: kPlanNone lets the library choose.
+static int launch_qgemm(const int8_t* a, const void* b, bool b_packed, float* y, int64_t ldy, const GemmParams& p, cudaStream_t st,
+                        int forced_plan = kPlanNone) {
+  const int sms = sm_count();
+  if (sms <= 0) return AQT_ERR_CUDA;
+  const GemmShape g = gemm_shape_of(p);
+  int plan = forced_plan;
+  if (plan != kPlanNone) {
+    if (!gemm_plan_takes(plan, g, sms)) return AQT_ERR_UNSUPPORTED;
+  } else {
+    plan = plan_qgemm(g, sms);
+  }
+  return launch_qgemm_plan(plan, a, b, b_packed, y, ldy, p, st);
 }
 
 }  // namespace aqt

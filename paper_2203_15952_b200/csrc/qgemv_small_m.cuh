@@ -144,7 +144,7 @@ __global__ void __launch_bounds__(kSmallThreads) qgemv_small_m_kernel(const Smal
 }
 
 static bool small_m_applies(int64_t M, int64_t K) {
-  static const char* lim = getenv("AQT_SMALL_M_MAX");  // tuning aid: 0 disables this kernel
+  const char* lim = tuning_env("AQT_SMALL_M_MAX");  // tuning builds: 0 disables this kernel
   const int64_t max_rows = lim != nullptr ? atoi(lim) : kSmallMaxRows;
   return M >= 1 && M <= max_rows && M <= kSmallMaxRows && K <= kSmallMaxK;
 }
@@ -159,10 +159,10 @@ static int launch_small_m_mb(const SmallParams& p, cudaStream_t st) {
 #define AQT_SMALL_LAUNCH(WP, GL)                                                                                    \
   do {                                                                                                              \
     auto kernel = qgemv_small_m_kernel<MB, WP, GL>;                                                                 \
-    static bool attr_set = false;                                                                                   \
-    if (!attr_set && smem > 48 * 1024) {                                                                            \
-      AQT_RETURN_IF_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MB * kSmallMaxK)); \
-      attr_set = true;                                                                                              \
+    static std::atomic<uint64_t> smem_opted_in{0};                                                                  \
+    if (smem > 48 * 1024) {                                                                                         \
+      const int rc_attr = ensure_dynamic_smem(kernel, MB * kSmallMaxK, smem_opted_in);                              \
+      if (rc_attr != AQT_OK) return rc_attr;                                                                        \
     }                                                                                                               \
     kernel<<<grid, kSmallThreads, smem, st>>>(p);                                                                   \
   } while (0)

@@ -29,6 +29,11 @@ from . import binding as aqt
 from .inputs import LinearSpec
 
 
+def _container_bits(bits_a: int) -> int:
+    """Activation codes travel between kernels in int8 containers (as Fig. 2 casts them)."""
+    return 8 if bits_a == 8 else aqt.BITS_4_UNPACKED
+
+
 @dataclass
 class QuantLinear:
     """Pre-quantized weights of one linear: codes W^T [N, K] (nibble-packed when 4-bit), one
@@ -37,6 +42,7 @@ class QuantLinear:
     wq: torch.Tensor
     s_w: torch.Tensor
     bias: Optional[torch.Tensor]
+    wq_unpacked: Optional[torch.Tensor] = None
 
     @classmethod
     def from_float(cls, spec: LinearSpec, wt: torch.Tensor, bias: Optional[torch.Tensor] = None,
@@ -45,7 +51,25 @@ class QuantLinear:
         quantizer the activations use (Fig. 2), packing 4-bit codes two per byte."""
         assert wt.shape == (spec.N, spec.K)
         wq, s_w = aqt.aqt_quantize(wt, spec.bits_w, aqt.AXIS_ROW, rounding, pack=(spec.bits_w == 4))
-        return cls(spec, wq, s_w, bias)
+        return cls(spec, wq, s_w, bias).prepare()
+
+    def prepare(self) -> "QuantLinear":
+        """Packed 4-bit weights deeper than the weight-stationary kernel's 512 (which sign-extends
+        them itself in shared memory) would be sign-extended into the workspace on every call:
+        do it once here and hand the matmuls the int8 containers instead."""
+        s = self.spec
+        if s.bits_w == 4 and (s.K > 512 or s.K % 32 != 0) and self.wq_unpacked is None:
+            self.wq_unpacked = aqt.aqt_unpack_int4(self.wq, s.K)
+        return self
+
+    @property
+    def mm_weight(self) -> torch.Tensor:
+        """The codes as handed to the matmul entry points."""
+        return self.wq if self.wq_unpacked is None else self.wq_unpacked
+
+    @property
+    def mm_bits(self) -> int:
+        return self.spec.bits_w if self.wq_unpacked is None else aqt.BITS_4_UNPACKED
 
     @property
     def weight_bytes(self) -> int:
@@ -78,8 +102,8 @@ class LayerRunner:
                residual: Optional[torch.Tensor] = None, residual_scale: float = 1.0) -> torch.Tensor:
         """Integer matmul + epilogue of `layer` on already-quantized activations (int8 containers)."""
         s = layer.spec
-        return aqt.aqt_qmatmul(xq, s_x, layer.wq, layer.s_w, layer.bias, residual, residual_scale, K=s.K, bits_a=8, bits_w=s.bits_w,
-                               act=s.act, s_x_kind=self.a_scale_kind, y=y, workspace=self.workspace)
+        return aqt.aqt_qmatmul(xq, s_x, layer.mm_weight, layer.s_w, layer.bias, residual, residual_scale, K=s.K, bits_a=_container_bits(s.bits_a),
+                               bits_w=layer.mm_bits, act=s.act, s_x_kind=self.a_scale_kind, y=y, workspace=self.workspace)
 
     def fuses_requant(self, layer: QuantLinear, with_y: bool = True) -> bool:
         """True if `layer`'s matmul can quantize its own output rows in its epilogue (the GLU
@@ -103,16 +127,16 @@ class LayerRunner:
         epilogue.  Returns (codes, scales); y (fp32) is written too if given."""
         s = layer.spec
         q, sc = self.code_buffers(role, s.n_out)
-        aqt.aqt_qmatmul_requant(xq, s_x, layer.wq, layer.s_w, layer.bias, residual, residual_scale, K=s.K, bits_a=8,
-                                bits_w=s.bits_w, act=s.act, s_x_kind=self.a_scale_kind, bits_out=bits_out,
+        aqt.aqt_qmatmul_requant(xq, s_x, layer.mm_weight, layer.s_w, layer.bias, residual, residual_scale, K=s.K, bits_a=_container_bits(s.bits_a),
+                                bits_w=layer.mm_bits, act=s.act, s_x_kind=self.a_scale_kind, bits_out=bits_out,
                                 rounding=self.rounding, pack_out=False, q_out=q, s_out=sc, y=y, workspace=self.workspace)
         return q, sc
 
     def __call__(self, layer: QuantLinear, x: torch.Tensor, y: torch.Tensor, residual: Optional[torch.Tensor] = None,
                  residual_scale: float = 1.0) -> torch.Tensor:
         s = layer.spec
-        return aqt.aqt_linear_fwd(x, layer.wq, layer.s_w, layer.bias, residual, residual_scale, bits_a=s.bits_a,
-                                  bits_w=s.bits_w, a_scale_kind=self.a_scale_kind, rounding=self.rounding, act=s.act,
+        return aqt.aqt_linear_fwd(x, layer.mm_weight, layer.s_w, layer.bias, residual, residual_scale, bits_a=s.bits_a,
+                                  bits_w=layer.mm_bits, a_scale_kind=self.a_scale_kind, rounding=self.rounding, act=s.act,
                                   y=y, workspace=self.workspace)
 
 
@@ -142,11 +166,7 @@ class FfnPair:
     def launches_per_step(self) -> int:
         """Kernels of the library launched by one forward()."""
         l0, l1 = self.layers
-        unpack2 = 1 if (l1.spec.bits_w == 4 and l1.spec.K > 512) else 0
-        if self.fused:
-            return 3 + unpack2
-        unpack1 = 1 if (l0.spec.bits_w == 4 and l0.spec.K > 512) else 0
-        return 4 + unpack1 + unpack2
+        return 3 if self.fused else 4
 
     @property
     def ops(self) -> int:
@@ -187,7 +207,7 @@ class ConformerBlockLinears:
         # run the three projections as one matmul over their concatenated output channels
         hq, hs = run.quantize_input(self.h_a, L[2].spec.bits_a)
         wq, s_w, bias = self._fused_qkv(L)
-        aqt.aqt_qmatmul(hq, hs, wq, s_w, bias, None, 1.0, K=self.d, bits_a=8, bits_w=L[2].spec.bits_w, act=aqt.ACT_NONE,
+        aqt.aqt_qmatmul(hq, hs, wq, s_w, bias, None, 1.0, K=self.d, bits_a=_container_bits(L[2].spec.bits_a), bits_w=L[2].mm_bits, act=aqt.ACT_NONE,
                         s_x_kind=run.a_scale_kind, y=self.qkv, workspace=run.workspace)
         note(L[2].spec.name, self.q); note(L[3].spec.name, self.k); note(L[4].spec.name, self.v)
         # h_b = h_a + W_o v is needed both as fp32 (residual stream) and as codes (pointwise 1)
@@ -249,7 +269,8 @@ class ConformerBlockLinears:
             q, k, v = L[2], L[3], L[4]
             assert q.spec.bits_w == k.spec.bits_w == v.spec.bits_w and q.spec.act == k.spec.act == v.spec.act == aqt.ACT_NONE
             bias = None if q.bias is None else torch.cat([q.bias, k.bias, v.bias]).contiguous()
-            self._qkv_weights[key] = (torch.cat([q.wq, k.wq, v.wq]).contiguous(), torch.cat([q.s_w, k.s_w, v.s_w]).contiguous(), bias)
+            self._qkv_weights[key] = (torch.cat([q.mm_weight, k.mm_weight, v.mm_weight]).contiguous(),
+                                      torch.cat([q.s_w, k.s_w, v.s_w]).contiguous(), bias)
         return self._qkv_weights[key]
 
     def ops(self, layers: List[QuantLinear]) -> int:

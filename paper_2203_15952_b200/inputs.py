@@ -15,6 +15,8 @@ width 512, 8 heads) and stand in for those workloads.
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
 from dataclasses import dataclass
 from typing import Optional, Sequence
 
@@ -65,19 +67,35 @@ def _index_grid(rows: int, cols: int, row_subset: Optional[Sequence[int]]) -> np
     return r[:, None] * np.uint64(cols) + c[None, :]
 
 
+def _for_each_chunk(n_rows: int, chunk_rows: int, fill) -> None:
+    """fill(a, b) for consecutive row ranges; large tensors on a few threads (the numpy kernels
+    release the interpreter lock, and every element is a function of its own counter only, so the
+    result does not depend on how the rows are cut)."""
+    starts = list(range(0, n_rows, chunk_rows))
+    threads = min(len(starts), os.cpu_count() or 1, 16)
+    if threads <= 1:
+        for a in starts:
+            fill(a, min(a + chunk_rows, n_rows))
+        return
+    with ThreadPoolExecutor(max_workers=threads) as pool:
+        list(pool.map(lambda a: fill(a, min(a + chunk_rows, n_rows)), starts))
+
+
 def normal(seed: int, tensor_id: int, rows: int, cols: int, std: float = 1.0,
-           row_subset: Optional[Sequence[int]] = None, chunk_rows: int = 8192) -> np.ndarray:
+           row_subset: Optional[Sequence[int]] = None, chunk_rows: int = 2048) -> np.ndarray:
     """float32 [rows, cols] (or [len(row_subset), cols]) ~ N(0, std^2)."""
     sel = np.arange(rows) if row_subset is None else np.asarray(row_subset)
     out = np.empty((len(sel), cols), dtype=np.float32)
-    for a in range(0, len(sel), chunk_rows):
-        idx = _index_grid(rows, cols, sel[a:a + chunk_rows])
-        out[a:a + chunk_rows] = (_normal_f64(seed, tensor_id, idx) * std).astype(np.float32)
+
+    def fill(a, b):
+        idx = _index_grid(rows, cols, sel[a:b])
+        out[a:b] = (_normal_f64(seed, tensor_id, idx) * std).astype(np.float32)
+    _for_each_chunk(len(sel), chunk_rows, fill)
     return out
 
 
 def student_t3(seed: int, tensor_id: int, rows: int, cols: int,
-               row_subset: Optional[Sequence[int]] = None, chunk_rows: int = 4096) -> np.ndarray:
+               row_subset: Optional[Sequence[int]] = None, chunk_rows: int = 1024) -> np.ndarray:
     """float32 heavy-tailed activations: Student-t with 3 degrees of freedom, unit variance.
 
     t = z0 / sqrt((z1^2 + z2^2 + z3^2) / 3), divided by sqrt(3) (the variance of t_3 is 3).
@@ -85,12 +103,23 @@ def student_t3(seed: int, tensor_id: int, rows: int, cols: int,
     """
     sel = np.arange(rows) if row_subset is None else np.asarray(row_subset)
     out = np.empty((len(sel), cols), dtype=np.float32)
-    for a in range(0, len(sel), chunk_rows):
-        idx = _index_grid(rows, cols, sel[a:a + chunk_rows])
+
+    def fill(a, b):
+        idx = _index_grid(rows, cols, sel[a:b])
         z = [_normal_f64(seed, tensor_id * 4 + j + (1 << 60), idx) for j in range(4)]
         t = z[0] / np.sqrt((z[1] ** 2 + z[2] ** 2 + z[3] ** 2) / 3.0)
-        out[a:a + chunk_rows] = (t / np.sqrt(3.0)).astype(np.float32)
+        out[a:b] = (t / np.sqrt(3.0)).astype(np.float32)
+    _for_each_chunk(len(sel), chunk_rows, fill)
     return out
+
+
+def random_codes(seed: int, rows: int, cols: int, bits: int) -> np.ndarray:
+    """int8 [rows, cols] quantization codes drawn uniformly from [-qmax, qmax] (qmax = 127 at 8
+    bits, 7 at 4), for tests that start from codes instead of from float tensors.  One sequential
+    stream per seed (numpy's PCG64), so the full tensor is generated and rows are picked from it."""
+    qmax = 127 if bits == 8 else 7
+    rng = np.random.Generator(np.random.PCG64(seed))
+    return rng.integers(-qmax, qmax + 1, size=(rows, cols), dtype=np.int8)
 
 
 def tensor_id(config: int, block: int = 0, layer: int = 0, role: int = 0) -> int:

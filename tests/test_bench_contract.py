@@ -39,7 +39,7 @@ def test_gpu_arm_prints_the_contract_line_with_roofline_and_e2e():
     """The library's own arm on one GPU: one JSON line with the contract's keys, a roofline object
     for the dominant call, an end-to-end figure with its copy sizes, and a non-zero launch count."""
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--steps", "14", "--warmup", "3", "--no-cpu-baseline",
-                          "--no-encoder"], capture_output=True, text=True, timeout=600, cwd=ROOT)
+                          "--no-legs"], capture_output=True, text=True, timeout=600, cwd=ROOT)
     assert out.returncode == 0, out.stderr[-2000:]
     lines = [l for l in out.stdout.strip().splitlines() if l.startswith("{")]
     assert len(lines) == 1
@@ -48,10 +48,13 @@ def test_gpu_arm_prints_the_contract_line_with_roofline_and_e2e():
                 "dtype", "data", "config", "e2e", "gpu_launches", "roofline", "clocks"):
         assert key in d, key
     assert d["n_gpus"] == 1 and d["steps"] == 14 and d["unit"] == "TOPS" and d["value"] > 0 and d["vs_baseline"] is None
-    assert d["gpu_launches"] == 14 * 4 and d["device_status"] == 0
+    assert d["gpu_launches"] == 14 * 3 and d["device_status"] == 0 and d["e2e"]["device_status"] == 0
     r = d["roofline"]
     assert r["bound"] in ("hbm", "tensor", "alu") and 0 < r["frac"] < 1.5 and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
     assert len(r["calls"]) == 3 and abs(sum(c["share"] for c in r["calls"]) - 1.0) < 1e-9
+    # per-call durations come from events inside the replayed graph: together they are the step
+    assert 0.7 < d["sum_call_ms_per_step"] / d["sustained"]["ms_per_step"] < 1.3
+    assert d["sustained"]["seconds"] >= 0.5 and d["clocks"]["samples"] >= 4
     e = d["e2e"]
     assert e["h2d_bytes_per_step"] == 4 * 12800 * 512 and e["d2h_bytes_per_step"] == 4 * 12800 * 512 and 0 < e["value"] < d["value"]
     assert "workload" in d["config"] and "model" not in d["config"]

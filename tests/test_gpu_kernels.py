@@ -102,7 +102,10 @@ def _codes(rng, rows, K, bits):
     return rng.integers(-qm, qm + 1, (rows, K)).astype(np.int8)
 
 
-def _run_qmatmul(M, N, K, bits_a, bits_w, act, with_bias, with_res, s_x_kind=aqt.SCALE_ROW, seed=0, extremes=False):
+def _run_qmatmul(M, N, K, bits_a, bits_w, act, with_bias, with_res, s_x_kind=aqt.SCALE_ROW, seed=0, extremes=False, plan=None,
+                 unpacked4=False):
+    """One aqt_qmatmul call against the oracle.  plan: a kernel configuration by name instead of
+    the library's choice.  unpacked4: 4-bit codes handed over in int8 containers (AQT_BITS_4_UNPACKED)."""
     rng = np.random.default_rng(seed + 1000 * M + N + K)
     xq = _codes(rng, M, K, bits_a)
     wq = _codes(rng, N, K, bits_w)
@@ -119,14 +122,23 @@ def _run_qmatmul(M, N, K, bits_a, bits_w, act, with_bias, with_res, s_x_kind=aqt
     y_ref = orc.epilogue_f32(acc_ref, s_x, s_x_kind, s_w, bias, res, 0.5, act)
     y64 = orc.epilogue_f64(acc_ref, s_x, s_x_kind, s_w, bias, res, 0.5, act)
 
-    xq_d = _dev(orc.pack_int4(xq)) if bits_a == 4 else _dev(xq)
-    wq_d = _dev(orc.pack_int4(wq)) if bits_w == 4 else _dev(wq)
+    xq_d = _dev(orc.pack_int4(xq)) if (bits_a == 4 and not unpacked4) else _dev(xq)
+    wq_d = _dev(orc.pack_int4(wq)) if (bits_w == 4 and not unpacked4) else _dev(wq)
+    arg_a = aqt.BITS_4_UNPACKED if (bits_a == 4 and unpacked4) else bits_a
+    arg_w = aqt.BITS_4_UNPACKED if (bits_w == 4 and unpacked4) else bits_w
     acc_d = torch.full((M, N), -12345, dtype=torch.int32, device=DEV)
     y_d = torch.full((M, n_out), float("nan"), dtype=torch.float32, device=DEV)
     aqt.aqt_qmatmul(xq_d, _dev(s_x), wq_d, _dev(s_w), None if bias is None else _dev(bias),
-                    None if res is None else _dev(res), 0.5, K=K, bits_a=bits_a, bits_w=bits_w, act=act,
-                    s_x_kind=s_x_kind, y=y_d, acc_debug=acc_d)
+                    None if res is None else _dev(res), 0.5, K=K, bits_a=arg_a, bits_w=arg_w, act=act,
+                    s_x_kind=s_x_kind, y=y_d, acc_debug=acc_d, plan=plan)
     _status_ok()
+    # the production instantiation (no accumulator dump) writes the same output bits
+    y_p = torch.full((M, n_out), float("nan"), dtype=torch.float32, device=DEV)
+    aqt.aqt_qmatmul(xq_d, _dev(s_x), wq_d, _dev(s_w), None if bias is None else _dev(bias),
+                    None if res is None else _dev(res), 0.5, K=K, bits_a=arg_a, bits_w=arg_w, act=act,
+                    s_x_kind=s_x_kind, y=y_p, plan=plan)
+    _status_ok()
+    assert torch.equal(y_p.view(torch.int32), y_d.view(torch.int32))
     acc = acc_d.cpu().numpy()
     y = y_d.cpu().numpy()
     assert np.array_equal(acc.astype(np.int64), acc_ref), "accumulators differ: %d of %d" % ((acc != acc_ref).sum(), acc.size)
@@ -164,7 +176,16 @@ def test_qmatmul_int4_operands(bits_a, bits_w, M, N, K):
 @pytest.mark.parametrize("act", [aqt.ACT_SWISH, aqt.ACT_GLU, aqt.ACT_GLU_SWISH])
 @pytest.mark.parametrize("M,N,K", [(256, 512, 256), (300, 1024, 512), (100, 136, 64)])
 def test_qmatmul_activations(act, M, N, K):
+    if act != aqt.ACT_SWISH and M > 128:
+        assert aqt.aqt_plan_qmatmul(M, N, K, 8, 4, act) == "ws128e8"      # the GLU forms of the weight-stationary kernel
     _run_qmatmul(M, N, K, 8, 4, act, True, True)
+
+
+@pytest.mark.parametrize("plan", ["stream128s4e8", "stream256s3e16"])
+def test_qmatmul_glu_streaming_plan_named(plan):
+    """GLU on the streaming kernel (K > 512: value and gate rows of a tile are two boxes of the ring)."""
+    _run_qmatmul(600, 1024, 1024, 8, 4, aqt.ACT_GLU_SWISH, True, True, plan=plan)
+    _run_qmatmul(300, 512, 640, 8, 8, aqt.ACT_GLU, False, False, plan=plan)
 
 
 @pytest.mark.parametrize("M", [4, 200, 1300])
@@ -220,22 +241,66 @@ def test_linear_fwd_small_batch_matches_oracle():
     assert np.array_equal(y.cpu().numpy().view(np.uint32), y_ref.view(np.uint32))
 
 
-def test_qmatmul_cta_pairs_forced(monkeypatch):
-    """The two-CTA (cta_group::2) form of the streaming kernel, forced on for shapes that would
-    normally take one CTA per tile: ragged M (the second CTA's rows partly or wholly outside),
-    ragged N, GLU halves split across the pair, residual, several tiles per pair."""
-    monkeypatch.setenv("AQT_FORCE_PAIRS", "1")
-    _run_qmatmul(130, 200, 2048, 8, 8, aqt.ACT_NONE, True, True, extremes=True)
-    _run_qmatmul(256, 512, 1024, 8, 4, aqt.ACT_GLU_SWISH, True, True)
-    _run_qmatmul(700, 384, 640, 8, 8, aqt.ACT_SWISH, True, False)
-    _run_qmatmul(256 * 80 + 37, 256, 2048, 8, 8, aqt.ACT_NONE, False, True)
-    _run_qmatmul(512, 1024, 4096, 4, 4, aqt.ACT_NONE, False, False, s_x_kind=aqt.SCALE_TENSOR)
+PAIR_PLANS = ["pair256s4e8", "pair256s6e4", "pair128s6e8", "pair128s8e4"]
+
+
+@pytest.mark.parametrize("plan", PAIR_PLANS + ["pair512s3e16"])
+def test_qmatmul_cta_pair_plans_named(plan):
+    """Every two-CTA (cta_group::2) configuration of the streaming kernel, named explicitly, on
+    shapes that would otherwise take one CTA per tile: ragged M (the second CTA's rows partly or
+    wholly outside), ragged N, residual, several tiles per pair, 4-bit operands in both layouts."""
+    _run_qmatmul(130, 200, 2048, 8, 8, aqt.ACT_NONE, True, True, extremes=True, plan=plan)
+    _run_qmatmul(700, 384, 640, 8, 8, aqt.ACT_SWISH, True, False, plan=plan)
+    _run_qmatmul(256 * 80 + 37, 256, 2048, 8, 8, aqt.ACT_NONE, False, True, plan=plan)
+    _run_qmatmul(512, 1024, 4096, 4, 4, aqt.ACT_NONE, False, False, s_x_kind=aqt.SCALE_TENSOR, plan=plan)
+    _run_qmatmul(1000, 1536, 1024, 8, 4, aqt.ACT_NONE, True, True, plan=plan, unpacked4=True)
+
+
+@pytest.mark.parametrize("plan", ["pair256s4e8", "pair256s6e4", "pair128s6e8", "pair128s8e4"])
+def test_qmatmul_cta_pair_plans_glu(plan):
+    """GLU halves split across the pair (value rows in the leader, gate rows in its peer)."""
+    _run_qmatmul(256, 512, 1024, 8, 4, aqt.ACT_GLU_SWISH, True, True, plan=plan)
+    _run_qmatmul(900, 1024, 512, 8, 8, aqt.ACT_GLU, False, True, plan=plan)
+
+
+@pytest.mark.parametrize("plan", ["stream256s3e16", "stream256s4e4", "stream128s4e16", "stream128s6e4", "stream64s5e8", "stream64s8e4",
+                                  "ws128e16"])
+def test_qmatmul_single_cta_plans_named(plan):
+    """The one-CTA-per-tile configurations by name, on one shallow shape all of them can take."""
+    _run_qmatmul(777, 640, 512, 8, 4, aqt.ACT_SWISH, True, True, plan=plan)
+    _run_qmatmul(300, 256, 384, 8, 8, aqt.ACT_NONE, True, False, plan=plan, extremes=True)
+
+
+def test_qmatmul_wide_pair_tiles_ffn_second_layer_shape():
+    """The benchmark's second matmul (12 800 x 2048 -> 512, 4-bit weights kept unpacked by the
+    caller): the plan the library picks is the 256 x 512 pair tile; full size, sampled rows."""
+    M, N, K = 12800, 512, 2048
+    assert aqt.aqt_plan_qmatmul(M, N, K, 8, aqt.BITS_4_UNPACKED) == "pair512s3e16"
+    xq = gen.random_codes(11, M, K, 8)
+    wq = gen.random_codes(12, N, K, 4)
+    rng = np.random.default_rng(13)
+    s_x = rng.uniform(1e-3, 5e-2, M).astype(np.float32)
+    s_w = rng.uniform(1e-4, 5e-3, N).astype(np.float32)
+    res = rng.standard_normal((M, N)).astype(np.float32)
+    acc_d = torch.empty((M, N), dtype=torch.int32, device=DEV)
+    args = (_dev(xq), _dev(s_x), _dev(wq), _dev(s_w), None, _dev(res), 0.5)
+    y = aqt.aqt_qmatmul(*args, K=K, bits_a=8, bits_w=aqt.BITS_4_UNPACKED)
+    y2 = aqt.aqt_qmatmul(*args, K=K, bits_a=8, bits_w=aqt.BITS_4_UNPACKED, acc_debug=acc_d)
+    y3 = aqt.aqt_qmatmul(_dev(xq), _dev(s_x), _dev(orc.pack_int4(wq)), _dev(s_w), None, _dev(res), 0.5, K=K, bits_a=8, bits_w=4)
+    _status_ok()
+    rows = sorted(set([0, 127, 128, 255, 256, 511, 512, M - 257, M - 129, M - 1]) | set(rng.integers(0, M, 40).tolist()))
+    acc_ref = orc.int_matmul(xq[rows], wq)
+    assert np.array_equal(acc_d.cpu().numpy()[rows].astype(np.int64), acc_ref)
+    y_ref = orc.epilogue_f32(acc_ref, s_x[rows], orc.SCALE_ROW, s_w, None, res[rows], 0.5, orc.ACT_NONE)
+    assert np.array_equal(y.cpu().numpy()[rows].view(np.uint32), y_ref.view(np.uint32))
+    assert torch.equal(y.view(torch.int32), y2.view(torch.int32)) and torch.equal(y.view(torch.int32), y3.view(torch.int32))
 
 
 def test_qmatmul_cta_pairs_large_deep_k_sampled_rows():
     """A shape that takes CTA pairs by itself (deep K, many tiles per pair): 19 200 x 1024 x 2048.
     Accumulators and outputs are compared with the oracle on sampled rows."""
     M, N, K = 19200, 1024, 2048
+    assert aqt.aqt_plan_qmatmul(M, N, K, 8, 4) == "pair256s4e8"
     rng = np.random.default_rng(7)
     xq = rng.integers(-127, 128, (M, K)).astype(np.int8)
     wq = rng.integers(-7, 8, (N, K)).astype(np.int8)

@@ -129,7 +129,7 @@ def test_cfg2_ffn_pair_full_size_sampled_rows():
 
 
 def _check_block(w, specs, cpu, keep, h_in_rows, rows):
-    g = {k: v.cpu().numpy()[rows] for k, v in keep.items()}
+    g = {k: v[rows].cpu().numpy() for k, v in keep.items()}
     n = [s.name for s in specs]
     _check_layer(specs[0], cpu[0], h_in_rows, g[n[0]])
     _check_layer(specs[1], cpu[1], g[n[0]], g[n[1]], residual_rows=h_in_rows, rs=0.5)
@@ -180,16 +180,15 @@ def test_cfg4_stack_mixed_precision():
     xd = _dev(x)
     h_gpu = stack.forward(xd).cpu().numpy()
     assert aqt.aqt_device_status() == 0 and np.isfinite(h_gpu).all()
-    # layer-wise parity of the first and the last block, fed with the GPU's own block inputs
+    # layer-wise parity of every block, each fed with the GPU's own block input
     blk = stack.block
     src = xd
     for b in range(w.blocks):
         dst = stack.h0 if b % 2 == 0 else stack.h1
-        keep = {} if b in (0, w.blocks - 1) else None
-        h_in_rows = src.cpu().numpy()[rows] if keep is not None else None
+        keep = {}
+        h_in_rows = src[rows].cpu().numpy()
         blk.forward(blocks_gpu[b], src, dst, keep=keep)
-        if keep is not None:
-            _check_block(w, specs, blocks_cpu[b], keep, h_in_rows, rows)
+        _check_block(w, specs, blocks_cpu[b], keep, h_in_rows, rows)
         src = dst
     assert np.array_equal(src.cpu().numpy().view(np.uint32), h_gpu.view(np.uint32))     # deterministic
     # Free-running oracle (fed its own outputs) on a few rows.  A last-ulp difference in a Swish

@@ -7,7 +7,8 @@ aqt_qmatmul_w4_noalloc exists for callers that cannot get device scratch memory 
 inside a capture, a host application that owns all allocations, a fixed memory budget): the
 sign-extended weights go into an array built into the library instead of a caller workspace.
 All calls share that array and it keeps the previous call's bytes, so the test makes two calls in
-a row with different weights and a smaller second shape, and checks both against aqt_qmatmul.
+a row with different weights and a smaller second shape, and checks both against aqt_qmatmul
+and against the CPU oracle.
 """
 import ctypes
 
@@ -33,9 +34,22 @@ def _case(seed, M, N, K, act, with_res):
     return xq, s_x, wq, s_w, bias, res, n_out
 
 
-@pytest.mark.parametrize("first,second", [((300, 512, 512, aqt.ACT_NONE, True), (129, 136, 96, aqt.ACT_SWISH, False)),
-                                          ((256, 1024, 2048, aqt.ACT_GLU_SWISH, True), (256, 1024, 2048, aqt.ACT_NONE, False))])
-def test_noalloc_matches_workspace_entry_point_twice_in_a_row(first, second):
+def _oracle_rows(xq, s_x, wq, s_w, bias, res, act, rows):
+    """The oracle's result for the given rows (codes unpacked by the oracle's own routine)."""
+    import oracle as orc
+    wq_i8 = orc.unpack_int4(wq.cpu().numpy(), 2 * wq.shape[1])
+    acc = orc.int_matmul(xq.cpu().numpy()[rows], wq_i8)
+    r = None if res is None else res.cpu().numpy()[rows]
+    args = (acc, s_x.cpu().numpy()[rows], orc.SCALE_ROW, s_w.cpu().numpy(), bias.cpu().numpy(), r, 0.5, act)
+    return orc.epilogue_f32(*args), orc.epilogue_f64(*args), np.abs(orc.epilogue_f64(acc, args[1], orc.SCALE_ROW, args[3], None, None, 0.0, 0))
+
+
+# Every shape has K > 512, so the weights always go through the built-in scratch array (smaller K
+# is sign-extended in shared memory and would not touch it).  The second call of a pair is
+# smaller than the first and uses other weights: it runs over the first call's stale bytes.
+@pytest.mark.parametrize("first,second", [((300, 512, 2048, aqt.ACT_NONE, True), (129, 136, 1024, aqt.ACT_SWISH, False)),
+                                          ((256, 1024, 2048, aqt.ACT_GLU_SWISH, True), (200, 256, 640, aqt.ACT_NONE, False))])
+def test_noalloc_matches_workspace_entry_point_and_oracle_twice_in_a_row(first, second):
     for seed, (M, N, K, act, with_res) in enumerate((first, second)):
         xq, s_x, wq, s_w, bias, res, n_out = _case(seed, M, N, K, act, with_res)
         y_ref = aqt.aqt_qmatmul(xq, s_x, wq, s_w, bias, res, 0.5, K=K, bits_a=8, bits_w=4, act=act)
@@ -44,6 +58,17 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row(first, second):
         assert aqt.aqt_device_status() == 0
         # same kernels on the same codes: identical bits (stricter than the 1e-6 used against the oracle)
         assert torch.equal(y.view(torch.int32), y_ref.view(torch.int32))
+        # and against the CPU oracle on rows across the tile edges
+        rows = sorted(set([0, 1, 127, 128, M - 1]) | set(range(0, M, 37)))
+        y32, y64, z = _oracle_rows(xq, s_x, wq, s_w, bias, res, act, rows)
+        got = y.cpu().numpy()[rows]
+        if act == aqt.ACT_NONE:
+            assert np.array_equal(got.view(np.uint32), y32.view(np.uint32))
+        else:
+            mag = np.maximum(np.maximum(np.abs(y64), z[:, :n_out]), np.abs(bias.cpu().numpy()[:n_out])[None, :])
+            if res is not None:
+                mag = np.maximum(mag, np.abs(res.cpu().numpy()[rows]))
+            assert np.all(np.abs(got - y64) <= 1e-6 * mag + 1e-30)
 
 
 def test_noalloc_rejects_weights_larger_than_the_builtin_scratch():
@@ -56,8 +81,19 @@ def test_noalloc_rejects_weights_larger_than_the_builtin_scratch():
     with pytest.raises(aqt.AqtError) as e:
         aqt.aqt_qmatmul_w4_noalloc(xq, s[:128], wq, s, K=K, y=y)
     assert e.value.status == -3
-    # the largest accepted size still works
-    N2 = aqt.NOALLOC_MAX_WEIGHT_BYTES // K
-    y2 = torch.zeros((128, N2), dtype=torch.float32, device=DEV)
-    aqt.aqt_qmatmul_w4_noalloc(xq, s[:128], wq[:N2], s[:N2], K=K, y=y2)
-    assert aqt.aqt_device_status() == 0 and float(y2.abs().max()) == 0.0
+
+
+def test_noalloc_largest_accepted_weights_use_the_whole_scratch():
+    """N * K equal to the built-in limit, random codes: a tail or overrun error at the end of the
+    array would change the last output channels."""
+    K = 2048
+    N = aqt.NOALLOC_MAX_WEIGHT_BYTES // K
+    xq, s_x, wq, s_w, bias, res, n_out = _case(5, 160, N, K, aqt.ACT_NONE, False)
+    y_ref = aqt.aqt_qmatmul(xq, s_x, wq, s_w, bias, None, 0.5, K=K, bits_a=8, bits_w=4)
+    y = torch.full((160, N), float("nan"), dtype=torch.float32, device=DEV)
+    aqt.aqt_qmatmul_w4_noalloc(xq, s_x, wq, s_w, bias, None, 0.5, K=K, y=y)
+    assert aqt.aqt_device_status() == 0
+    assert torch.equal(y.view(torch.int32), y_ref.view(torch.int32))
+    rows = [0, 127, 128, 159]
+    y32, _, _ = _oracle_rows(xq, s_x, wq, s_w, bias, None, aqt.ACT_NONE, rows)
+    assert np.array_equal(y.cpu().numpy()[rows].view(np.uint32), y32.view(np.uint32))
