@@ -137,10 +137,8 @@ __device__ __forceinline__ void st_relaxed_gpu(uint32_t* p, uint32_t v) {
 }
 
 constexpr uint32_t kValidBit = 0x80000000u;
-// Pass 2 of a tile runs kLag tiles behind its pass 1, which is the time the exchange has to
-// complete; with four TMEM buffers that leaves the MMA one tile of lookahead.  kSlots tiles'
-// worth of shared-memory exchange state (maxima parts, arrival counts, scale constants).
-constexpr int kLag = 2;
+// One slot of shared-memory exchange state (final row maxima, hand-over barriers) per accumulator
+// buffer, i.e. per set of epilogue warps: tile i of a CTA uses buffer and slot i mod 4.
 constexpr int kSlots = 4;
 constexpr int kExchangeBatch = 16;  // exchange loads the exchange warp keeps in flight (one round trip for N <= 2048)
 
@@ -231,14 +229,9 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
   __shared__ uint64_t res_bar[EW];    // WITH_Y: residual tile landed in a warp's fp32 staging buffer
   __shared__ uint64_t b_loaded_bar;
   __shared__ uint64_t b_ready_bar;
-  __shared__ uint32_t amax_part[kSlots][4][kBM];  // row maxima per column part of the tile in pass 1 (slot = tile mod kSlots)
-  // Warps of a row quadrant that have written their part (running counts).  A warp can be in pass 1
-  // of tile j + kLag while another is still in pass 1 of tile j + 1, never further ahead (its pass 2
-  // of tile j needs this quadrant's maxima of tile j published): kSlots > kLag counters suffice.
-  __shared__ uint32_t quad_arrivals[kSlots][4];
   __shared__ __align__(16) uint32_t row_amax[kSlots][kBM];  // final row maxima (bit patterns) of a tile awaiting pass 2
   __shared__ uint64_t ctx_ready_bar[kSlots];  // the exchange warp has filled row_amax[.]
-  __shared__ uint64_t ctx_free_bar[kSlots];   // every epilogue warp has read its rows of row_amax[.]
+  __shared__ uint64_t ctx_free_bar[kSlots];   // the set's four warps have read their rows of row_amax[.]
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
@@ -270,14 +263,14 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     }
     for (int b = 0; b < 4; ++b) {
       mbar_init(smem_u32(&tmem_full_bar[b]), 1);
-      mbar_init(smem_u32(&tmem_empty_bar[b]), EW);
+      mbar_init(smem_u32(&tmem_empty_bar[b]), 4);  // the four warps of the set that owns the buffer
     }
     for (int w = 0; w < EW; ++w) mbar_init(smem_u32(&res_bar[w]), 1);
     mbar_init(smem_u32(&b_loaded_bar), 1);
     mbar_init(smem_u32(&b_ready_bar), EW);
     for (int b = 0; b < kSlots; ++b) {
       mbar_init(smem_u32(&ctx_ready_bar[b]), 1);
-      mbar_init(smem_u32(&ctx_free_bar[b]), EW);
+      mbar_init(smem_u32(&ctx_free_bar[b]), 4);
     }
     fence_barrier_init();
     fence_proxy_async_smem();
@@ -298,7 +291,6 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     asm volatile("st.shared.f32 [%0], %1;" ::"r"(smem_scale + t * 4), "f"(wv) : "memory");
     asm volatile("st.shared.f32 [%0], %1;" ::"r"(smem_scale + (BN + t) * 4), "f"(bv) : "memory");
   }
-  if (threadIdx.x < 4 * kSlots) quad_arrivals[threadIdx.x >> 2][threadIdx.x & 3] = 0u;
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -407,16 +399,22 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     }
   } else {
     // ------------------------------------------------------------------ epilogue warps
+    // Four sets of four warps, one warp of a set per TMEM lane quadrant (hence one per scheduler).
+    // Set s owns accumulator buffer s and with it every fourth tile of this CTA, all of its
+    // columns: pass 1 chunk by chunk, publication of the rows' maxima straight from registers
+    // (a thread has seen its whole row of the tile, so nothing is merged across warps), the wait
+    // for the other n-tiles' maxima, pass 2.  The four warps that share a scheduler therefore work
+    // on four different tiles in four different phases: while one is on the special-function unit
+    // (pass 1 of a Swish tile is bound by it), the others issue multiply-adds and byte permutes
+    // (pass 2), wait for the exchange, or wait for the tensor core.
     const int ew = warp - 2;
-    const int quad = warp & 3;   // TMEM lane quadrant this warp may access
-    const int cpart = ew >> 2;   // which 32 (GLU: 16) output columns of the tile
-    const int col = cpart * (GLU ? 16 : 32);
+    const int quad = warp & 3;  // TMEM lane quadrant this warp may access
+    const int set = ew >> 2;    // accumulator buffer and tile residue (mod 4) of this warp
+    constexpr int CW = GLU ? 16 : 32;  // output columns per chunk; four chunks per tile
     const int row_in_tile = quad * 32 + lane;
-      const uint32_t y_buf = smem_epi + ew * kStageBufBytes;
-    const uint32_t c_sw = smem_scale + (uint32_t)col * 4, c_bias = c_sw + BN * 4;
+    const uint32_t y_buf = smem_epi + ew * kStageBufBytes;
     const bool has_res = WITH_Y && p.residual != nullptr;
-    const int oc = tn * (GLU ? HALF : BN) + col;  // first output column of this warp
-    const bool cols_ok = oc < n_out;
+    const int oc0 = tn * (GLU ? HALF : BN);  // first output column of this CTA's tiles
     bool ok = true;
 
     if (BPACK) {
@@ -446,36 +444,41 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&b_ready_bar));
-        ok = mbar_wait(smem_u32(&b_ready_bar), 0, &abort_flag, t_start);  // staging area free for codes
+        ok = mbar_wait(smem_u32(&b_ready_bar), 0, &abort_flag, t_start);  // staging area free for the fp32 output
       }
     }
 
-    if (ok && has_res && lane == 0 && n_my > 0) {
-      const int r0 = group * kBM + quad * 32;
+    uint32_t res_count = 0;  // residual boxes this warp has consumed (phase of its barrier)
+    if (ok && has_res && lane == 0 && set < n_my) {
+      const int r0 = (group + set * groups) * kBM + quad * 32;
       mbar_arrive_expect_tx(smem_u32(&res_bar[ew]), kStageBufBytes);
-      tma_load_2d(y_buf, &tm_r, cols_ok ? oc : 0, r0 < p.M ? r0 : 0, smem_u32(&res_bar[ew]));
+      tma_load_2d(y_buf, &tm_r, oc0 < n_out ? oc0 : 0, r0 < p.M ? r0 : 0, smem_u32(&res_bar[ew]));
     }
 
-    for (int i = 0; ok && i < n_my + kLag; ++i) {
-      if (i < n_my) {
-        // -------------------------------------------------------------- pass 1 of tile i
-        const int tm = group + i * groups;
-        const uint32_t buf = i & 3, aph = (i >> 2) & 1;
-        const int row0_warp = tm * kBM + quad * 32;
-        const int m = row0_warp + lane;
-        const float sx = (p.s_x_kind == AQT_SCALE_ROW) ? (m < p.M ? __ldg(p.s_x + m) : 0.0f) : __ldg(p.s_x);
-        if (!mbar_wait(smem_u32(&tmem_full_bar[buf]), aph, &abort_flag, t_start)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t taddr = tmem_base + buf * BN + ((uint32_t)(quad * 32) << 16) + col;
-        float amax = 0.0f;
-        uint32_t acc[32];
-        float a[32];  // the non-GLU form's u, staged for the fp32 output further down
+    const uint32_t buf = (uint32_t)set;
+    const uint32_t tbase = tmem_base + buf * BN + ((uint32_t)(quad * 32) << 16);
+    for (int i = set; ok && i < n_my; i += 4) {
+      const int tm = group + i * groups;
+      const uint32_t aph = (uint32_t)(i >> 2) & 1u;
+      const int row0_warp = tm * kBM + quad * 32;
+      const int m = row0_warp + lane;
+      const float sx = (p.s_x_kind == AQT_SCALE_ROW) ? (m < p.M ? __ldg(p.s_x + m) : 0.0f) : __ldg(p.s_x);
+      if (!mbar_wait(smem_u32(&tmem_full_bar[buf]), aph, &abort_flag, t_start)) { ok = false; break; }
+      tc_fence_after();
+
+      // -------------------------------------------------------------- pass 1: u, row maxima; u back to TMEM
+      float amax = 0.0f;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        const int col = c * CW;
+        const bool cols_ok = oc0 + col < n_out;  // columns beyond N contribute nothing
+        const uint32_t c_sw = smem_scale + (uint32_t)col * 4, c_bias = c_sw + BN * 4;
         if constexpr (GLU) {
           // gates first: g = sigmoid(z_gate); then the values are scaled by it
           uint32_t accv[16], accg[16];
           float av[16], g[16];
-          tmem_ld_32x16(taddr + HALF, accg);
-          tmem_ld_32x16(taddr, accv);
+          tmem_ld_32x16(tbase + HALF + col, accg);
+          tmem_ld_32x16(tbase + col, accv);
           tmem_ld_wait();
           dequant16<SMALL>(accg, sx, c_sw + HALF * 4, c_bias + HALF * 4, g);
 #pragma unroll
@@ -484,19 +487,24 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
 #pragma unroll
           for (int j = 0; j < 16; ++j) av[j] = av[j] * g[j];
           if (p.act == AQT_ACT_GLU_SWISH) swish16(av);
+          float cmax = 0.0f;
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
-            amax = fmaxf(amax, fabsf(av[j]));
+            cmax = fmaxf(cmax, fabsf(av[j]));
             accv[j] = __float_as_uint(av[j]);
           }
-          tmem_st_32x16(taddr, accv);  // u replaces the value accumulators
+          if (cols_ok) amax = fmaxf(amax, cmax);
+          tmem_st_32x16(tbase + col, accv);  // u replaces the value accumulators
         } else {
-          tmem_ld_32x32(taddr, acc);
+          uint32_t acc[32];
+          float a[32];
+          tmem_ld_32x32(tbase + col, acc);
           tmem_ld_wait();
           dequant32<SMALL>(acc, sx, c_sw, c_bias, a);
           if (p.act == AQT_ACT_SWISH) swish32(a);
           if (has_res) {
-            if (!mbar_wait(smem_u32(&res_bar[ew]), i & 1, &abort_flag, t_start)) { ok = false; break; }
+            if (!mbar_wait(smem_u32(&res_bar[ew]), res_count & 1u, &abort_flag, t_start)) { ok = false; break; }
+            ++res_count;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
               const uint32_t src = y_buf + lane * 128 + ((j ^ (lane & 7)) << 4);
@@ -507,96 +515,88 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
               a[4 * j + 2] = __fmaf_rn(p.residual_scale, a[4 * j + 2], r2);
               a[4 * j + 3] = __fmaf_rn(p.residual_scale, a[4 * j + 3], r3);
             }
-            __syncwarp();
+            __syncwarp();  // every lane has read its residual row before the buffer is overwritten
           }
+          float cmax = 0.0f;
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            amax = fmaxf(amax, fabsf(a[j]));
+            cmax = fmaxf(cmax, fabsf(a[j]));
             acc[j] = __float_as_uint(a[j]);
           }
-          tmem_st_32x32(taddr, acc);
-        }
-        // this warp's part of the row maxima (columns beyond N contribute nothing)
-        amax_part[i % kSlots][cpart][row_in_tile] = cols_ok ? __float_as_uint(amax) : 0u;
-        __syncwarp();
-        int last = 0;
-        if (lane == 0) {
-          __threadfence_block();
-          last = (atomicAdd(&quad_arrivals[i % kSlots][quad], 1u) & 3u) == 3u ? 1 : 0;
-          __threadfence_block();
-        }
-        last = __shfl_sync(0xffffffffu, last, 0);
-        if (last) {
-          // the last of the quadrant's four warps publishes the CTA's maxima of these 32 rows
-          const uint32_t sl = i % kSlots;
-          const uint32_t v = max(max(amax_part[sl][0][row_in_tile], amax_part[sl][1][row_in_tile]),
-                                 max(amax_part[sl][2][row_in_tile], amax_part[sl][3][row_in_tile]));
-          st_relaxed_gpu(rp.exchange + ((size_t)tm * p.tiles_n + tn) * kBM + row_in_tile, v | kValidBit);
-        }
-
-        if (WITH_Y) {
-          if (!has_res) {
-            if (lane == 0) tma_store_wait_read<0>();
-            __syncwarp();
-          }
+          if (cols_ok) amax = fmaxf(amax, cmax);
+          tmem_st_32x32(tbase + col, acc);  // u replaces the accumulators it was made from
+          if (WITH_Y) {
+            if (!has_res) {
+              if (lane == 0) tma_store_wait_read<0>();  // the previous chunk's bulk store has read the buffer out
+              __syncwarp();
+            }
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const uint32_t dst = y_buf + lane * 128 + ((j ^ (lane & 7)) << 4);
-            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(a[4 * j]), "f"(a[4 * j + 1]), "f"(a[4 * j + 2]),
-                         "f"(a[4 * j + 3])
-                         : "memory");
-          }
-          fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) {
-            if (cols_ok && row0_warp < p.M) tma_store_2d(&tm_y, y_buf, oc, row0_warp);
-            tma_store_commit();
-            if (has_res) {
-              tma_store_wait_read<0>();
-              if (i + 1 < n_my) {
-                const int nr = (tm + groups) * kBM + quad * 32;
-                mbar_arrive_expect_tx(smem_u32(&res_bar[ew]), kStageBufBytes);
-                tma_load_2d(y_buf, &tm_r, cols_ok ? oc : 0, nr < p.M ? nr : 0, smem_u32(&res_bar[ew]));
+            for (int j = 0; j < 8; ++j) {
+              const uint32_t dst = y_buf + lane * 128 + ((j ^ (lane & 7)) << 4);
+              asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(a[4 * j]), "f"(a[4 * j + 1]), "f"(a[4 * j + 2]),
+                           "f"(a[4 * j + 3])
+                           : "memory");
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              if (cols_ok && row0_warp < p.M) tma_store_2d(&tm_y, y_buf, oc0 + col, row0_warp);
+              tma_store_commit();
+              if (has_res) {
+                // the next chunk's residual goes into the same buffer once this store has read it out
+                tma_store_wait_read<0>();
+                const bool more_here = c + 1 < 4;
+                if (more_here || i + 4 < n_my) {
+                  const int ncol = oc0 + (more_here ? col + CW : 0);
+                  const int nr = (more_here ? tm : tm + 4 * groups) * kBM + quad * 32;
+                  mbar_arrive_expect_tx(smem_u32(&res_bar[ew]), kStageBufBytes);
+                  tma_load_2d(y_buf, &tm_r, ncol < n_out ? ncol : 0, nr < p.M ? nr : 0, smem_u32(&res_bar[ew]));
+                }
               }
             }
           }
         }
-
       }
-      if (i >= kLag) {
-        // -------------------------------------------------------------- pass 2 of tile i - kLag
-        const int j = i - kLag;
-        const int tm = group + j * groups;
-        const uint32_t buf = j & 3;
-        const int row0_warp = tm * kBM + quad * 32;
-        const uint32_t par = j % kSlots;
-        if (!mbar_wait(smem_u32(&ctx_ready_bar[par]), (j / kSlots) & 1, &abort_flag, t_start)) { ok = false; break; }
-        const float amax = __uint_as_float(row_amax[par][row_in_tile]);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&ctx_free_bar[par]));
-        const ScaleCtx c = make_scale_ctx(amax, rp.qmax_out);
-        if (tn == 0 && cpart == 0 && row0_warp + lane < p.M) rp.s_out[row0_warp + lane] = c.s;
-        const uint32_t taddr = tmem_base + buf * BN + ((uint32_t)(quad * 32) << 16) + col;
-        const int m = row0_warp + lane;
-        tmem_st_wait();  // this warp's stores of pass 1 (long complete)
+      if (!ok) break;
+      // this CTA's maxima of the tile's rows, each tagged valid: one word per row, straight from the registers
+      st_relaxed_gpu(rp.exchange + ((size_t)tm * p.tiles_n + tn) * kBM + row_in_tile, __float_as_uint(amax) | kValidBit);
+
+      // -------------------------------------------------------------- pass 2: scale, codes
+      if (!mbar_wait(smem_u32(&ctx_ready_bar[set]), aph, &abort_flag, t_start)) { ok = false; break; }
+      const float amax_row = __uint_as_float(row_amax[set][row_in_tile]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctx_free_bar[set]));
+      const ScaleCtx sc = make_scale_ctx(amax_row, rp.qmax_out);
+      if (tn == 0 && m < p.M) rp.s_out[m] = sc.s;
+      tmem_st_wait();  // this warp's stores of pass 1
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        const int col = c * CW;
+        const int oc = oc0 + col;
+        const bool cols_ok = oc < n_out;
         if constexpr (GLU) {
           uint32_t u[16], w[4];
-          tmem_ld_32x16(taddr, u);
+          tmem_ld_32x16(tbase + col, u);
           tmem_ld_wait();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[buf]));
-          codes_of<ROUNDING, false, 16>(u, c, rp.qmax_out, w);
+          if (c == 3) {
+            // the tile has been read out by this warp: the accumulator buffer goes back to the MMA
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[buf]));
+          }
+          codes_of<ROUNDING, false, 16>(u, sc, rp.qmax_out, w);
           // 16 consecutive codes of the row: one 16-byte store
           if (m < p.M && cols_ok) *reinterpret_cast<uint4*>(rp.q_out + (size_t)m * n_out + oc) = make_uint4(w[0], w[1], w[2], w[3]);
         } else {
           uint32_t u[32], w[8];
-          tmem_ld_32x32(taddr, u);
+          tmem_ld_32x32(tbase + col, u);
           tmem_ld_wait();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[buf]));
-          codes_of<ROUNDING, PACK_OUT, 32>(u, c, rp.qmax_out, w);
+          if (c == 3) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[buf]));
+          }
+          codes_of<ROUNDING, PACK_OUT, 32>(u, sc, rp.qmax_out, w);
           // Each thread holds 32 consecutive codes of its row: one or two 16-byte stores, each a
           // whole 32-byte sector (or half of one for packed nibbles), straight to global memory.
           if (m < p.M && cols_ok) {
