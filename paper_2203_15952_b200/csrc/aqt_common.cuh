@@ -89,6 +89,33 @@ inline int ensure_dynamic_smem(Kernel kernel, int bytes, std::atomic<uint64_t>& 
   return AQT_OK;
 }
 
+// Launch with the programmatic-stream-serialization attribute (see grid_dependency_wait), optionally
+// as thread-block clusters of `cluster` CTAs.
+template <class... KArgs, class... Args>
+inline int launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, unsigned cluster, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
+  if (cluster > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = cluster;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n;
+  AQT_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
+  return launch_status(__LINE__);
+}
+
 // Overrides of the kernel choice for tuning runs.  They exist only in builds made with
 // -DAQT_TUNING; the shipped library never reads the environment to pick a kernel.
 inline const char* tuning_env(const char* name) {
@@ -145,6 +172,19 @@ __device__ __forceinline__ int quantize_elem(float x, const ScaleCtx& c, int qma
   }
   return max(-qmax, min(qmax, q));
 }
+
+// Programmatic dependent launch.  Every kernel of the library is launched so that it may start
+// while the kernel before it in the stream is still draining, and orders itself with
+//   grid_dependency_wait()     returns once the preceding kernel has completed and its memory
+//                              operations are visible; placed before the first global-memory access
+//                              that could touch anything another kernel reads or writes (set-up
+//                              that touches only this CTA's own state runs before it)
+//   grid_dependents_launch()   lets the next kernel's CTAs be scheduled once every CTA of this
+//                              kernel has executed it (or exited); always after the wait, so that
+//                              by the time a later kernel runs, the one before this kernel is complete
+// Without the launch attribute both are no-ops.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependents_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ uint64_t global_timer_ns() {
   uint64_t t;

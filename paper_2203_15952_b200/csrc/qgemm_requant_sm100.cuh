@@ -8,24 +8,26 @@
 // back (it is written too only when the caller asks for it, e.g. for a residual stream).
 //
 // A row's abs-max spans all N output columns, i.e. several CTAs.  The grid is made of groups of
-// tiles_n CTAs; the CTAs of a group own the n-tiles of the same m-tile at the same time (weight
-// stationary, K <= 512: each keeps its weight slab resident) and exchange row maxima through
-// global memory, one word per (m-tile, n-tile, row):
-//   pass 1 (tile j)   TMEM accumulators -> u (registers) -> row maxima; u goes back into the TMEM
-//                     columns it came from; the last of the four warps that share a row quadrant
-//                     merges their maxima and stores them, tagged valid in the sign bit (a
-//                     maximum is never negative), into the CTA's words of the exchange area
-//   exchange warp     for each tile in turn: reads the words of all n-tiles (128 rows per 512-byte
-//                     request, all requests in flight together), again until every one is valid,
-//                     and leaves the final maximum of each row in shared memory
-//   pass 2 (tile j-2) scale from the final maximum, u from TMEM, codes, stores; the TMEM buffer
-//                     goes back to the MMA
-// Every word carries its own validity, so no counter, fence or atomic on global memory is needed,
-// and the epilogue warps never wait on global memory.
-// Pass 2 of a tile runs after pass 1 of the tile two further on, so the exchange has two tiles'
-// worth of time to complete; four TMEM buffers of 128 columns keep the tensor core one tile ahead.
-// All CTAs must be resident at once (they wait on one another): the launch is cooperative and
-// the grid never exceeds one CTA per SM.  Every wait is bounded as in the plain GEMM.
+// tiles_n CTAs; the CTAs of a group own the n-tiles of the same m-tile at about the same time
+// (weight stationary, K <= 512 or 1024: each keeps its weight slab resident) and exchange row maxima
+// through global memory, one 64-bit word per (m-tile, n-tile, row): the maximum's bit pattern below a
+// tag that identifies this execution, so a word is its own validity and nothing is cleared,
+// counted or fenced.
+//   epilogue warps    four sets of four warps (one warp per TMEM lane quadrant); set s owns
+//                     accumulator buffer s and every fourth tile, all 128 columns of it:
+//                       pass 1  accumulators -> u (registers) -> row maxima; u goes back into the
+//                               TMEM columns it came from; the maxima are published
+//                       wait    for the group's other CTAs (the exchange warps do the polling)
+//                       pass 2  scale from the final maximum, u from TMEM, codes, stores; the TMEM
+//                               buffer goes back to the MMA
+//                     The four warps on a scheduler thus sit in four different phases of four
+//                     different tiles, which is what keeps the special-function unit (pass 1 of a
+//                     Swish tile) and the other pipes (pass 2) busy at the same time.
+//   exchange warps    two, one per half of the rows: for each tile in turn read the words of all
+//                     n-tiles (all requests in flight together), again until every one is valid,
+//                     and leave the final maximum of each row in shared memory
+// All CTAs of a group must be resident at once (they wait on one another): the grid never exceeds
+// one CTA per SM.  Every wait is bounded as in the plain GEMM.
 #pragma once
 
 #include "qgemm_sm100.cuh"
@@ -36,7 +38,10 @@ struct RequantParams {
   GemmParams g;         // act: NONE or SWISH
   uint8_t* q_out;       // codes of the output: int8 [M, N] or packed nibbles [M, N/2], dense
   float* s_out;         // [M] scales of the output rows
-  uint32_t* exchange;   // [tiles_m][tiles_n][128]: bit pattern of a CTA's row maximum | 0x80000000; zero on entry
+  uint64_t* exchange;   // [tiles_m][tiles_n][128] words: (launch tag << 32) | bit pattern of a CTA's row maximum
+  uint32_t* generation; // [groups] counters behind the words: each group of CTAs bumps its own when it has finished
+  uint32_t tag;         // tag of this call (no other call of the process uses it); a word counts once its upper half
+                        // equals this tag mixed with the group's generation, which differs on every execution of the call
   int qmax_out;         // 127 or 7
   int rounding;
   int pack_out;         // 1: two 4-bit codes per byte
@@ -53,7 +58,7 @@ struct RequantCfg {
   static constexpr int kKBlocks = DEEP ? kRequantDeepKBlocks : kWsMaxKBlocks;
   static constexpr int BN = 128;
   static constexpr int EW = 16;
-  static constexpr int kThreads = 32 * (2 + EW + 1);  // producer, MMA issuer, epilogue warps, exchange warp
+  static constexpr int kThreads = 32 * (2 + EW + 2);  // producer, MMA issuer, epilogue warps, two exchange warps
   static constexpr int kStages = (WITH_Y || DEEP) ? 5 : 7;
   static constexpr int kABytes = kBM * kBK;
   static constexpr int kBBytes = BN * kBK;
@@ -125,22 +130,31 @@ __device__ __forceinline__ void swish16(float (&a)[16]) {
   }
 }
 
+// A call's tag mixed with a generation count: distinct generations of one call give distinct values.
+__device__ __forceinline__ uint32_t mix_tag(uint32_t call_tag, uint32_t generation) {
+  uint32_t x = call_tag ^ (generation * 0x9E3779B1u);
+  x ^= x >> 16;
+  x *= 0x7FEB352Du;
+  x ^= x >> 15;
+  return x;
+}
+
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-__device__ __forceinline__ uint4 ld_relaxed_gpu_v4(const uint32_t* p) {
-  uint4 v;
-  asm volatile("ld.relaxed.gpu.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+// Two exchange words (each read as one indivisible 64-bit value).
+__device__ __forceinline__ ulonglong2 ld_relaxed_gpu_2x64(const uint64_t* p) {
+  ulonglong2 v;
+  asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v.x), "=l"(v.y) : "l"(p) : "memory");
   return v;
 }
-__device__ __forceinline__ void st_relaxed_gpu(uint32_t* p, uint32_t v) {
-  asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+__device__ __forceinline__ void st_relaxed_gpu_64(uint64_t* p, uint64_t v) {
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 
-constexpr uint32_t kValidBit = 0x80000000u;
 // One slot of shared-memory exchange state (final row maxima, hand-over barriers) per accumulator
 // buffer, i.e. per set of epilogue warps: tile i of a CTA uses buffer and slot i mod 4.
 constexpr int kSlots = 4;
-constexpr int kExchangeBatch = 16;  // exchange loads the exchange warp keeps in flight (one round trip for N <= 2048)
+constexpr int kExchangeBatch = 16;  // n-tiles whose words an exchange warp asks for at once (one 16-byte load each per lane)
 
 // Called between polls of a bounded wait: false once the CTA is aborting or the limit has passed
 // (which then sets both the CTA's abort flag and the device status word).
@@ -210,7 +224,7 @@ __device__ __forceinline__ void codes_of(const uint32_t (&u)[NV], const ScaleCtx
 // output columns u = v * sigmoid(g) (then Swish for AQT_ACT_GLU_SWISH), 16 per epilogue warp.
 // The GLU form writes codes and scales only (no fp32 output, no residual, no nibble packing).
 template <bool BPACK, bool SMALL, bool WITH_Y, int ROUNDING, bool PACK_OUT, bool GLU = false, bool DEEP = false>
-__global__ void __launch_bounds__(32 * 19, 1)
+__global__ void __launch_bounds__(32 * 20, 1)
 qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                      const __grid_constant__ CUtensorMap tm_y,
                      const __grid_constant__ CUtensorMap tm_r, const RequantParams rp) {
@@ -269,7 +283,7 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     mbar_init(smem_u32(&b_loaded_bar), 1);
     mbar_init(smem_u32(&b_ready_bar), EW);
     for (int b = 0; b < kSlots; ++b) {
-      mbar_init(smem_u32(&ctx_ready_bar[b]), 1);
+      mbar_init(smem_u32(&ctx_ready_bar[b]), 2);  // both exchange warps
       mbar_init(smem_u32(&ctx_free_bar[b]), 4);
     }
     fence_barrier_init();
@@ -279,6 +293,12 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     tmem_alloc(smem_u32(&tmem_base_slot), Cfg::kTmemCols);
     tmem_relinquish();
   }
+  // everything above touched only this CTA's own state; from here on global memory is read
+  grid_dependency_wait();
+  // Tag of this execution's exchange words.  A replayed CUDA graph repeats the call's own tag, so the
+  // group's generation counter goes into it: every CTA of the group reads it here, and the group's
+  // first CTA bumps it after its last tile, which it cannot finish before all of them have started.
+  const uint32_t tag = mix_tag(rp.tag, __ldcg(rp.generation + group));
   for (int t = threadIdx.x; t < BN; t += blockDim.x) {
     // scales and biases of the tile's weight rows: (GLU) values first, then gates
     const int n = !GLU ? tn * BN + t : (t < HALF ? tn * HALF + t : p.N / 2 + tn * HALF + (t - HALF));
@@ -328,6 +348,7 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
           tma_load_2d(smem_ring + s * Cfg::kABytes, &tm_a, kb * kBK, tm * kBM, bar);
         }
       }
+      grid_dependents_launch();  // every load of this CTA has been issued: the next kernel may be scheduled behind it
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -353,47 +374,46 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         if (ok) tc_commit(smem_u32(&tmem_full_bar[buf]));
       }
     }
-  } else if (warp == 2 + EW) {
-    // ------------------------------------------------------------------ exchange warp
-    // Lane l owns rows 4l .. 4l+3 of the tile: one 16-byte load per n-tile (the warp's request
-    // covers the n-tile's 128 words), kExchangeBatch of them in flight.
+  } else if (warp >= 2 + EW) {
+    // ------------------------------------------------------------------ exchange warps
+    // Two warps, each for one half of the tile's rows: lane l of warp h owns rows 64h + 2l and
+    // 64h + 2l + 1, i.e. one 16-byte load (two words) per n-tile, kExchangeBatch of them in flight.
+    const int xh = warp - (2 + EW);
     bool ok = true;
     for (int i = 0; ok && i < n_my; ++i) {
       const int tm = group + i * groups;
       const uint32_t par = i % kSlots, ph = (i / kSlots) & 1;
       if (!mbar_wait(smem_u32(&ctx_free_bar[par]), ph ^ 1, &abort_flag, t_start)) break;
-      const uint32_t* xt = rp.exchange + (size_t)tm * p.tiles_n * kBM + 4 * lane;
-      uint4 m4 = make_uint4(0u, 0u, 0u, 0u);
+      const uint64_t* xt = rp.exchange + (size_t)tm * p.tiles_n * kBM + 64 * xh + 2 * lane;
+      uint2 m2 = make_uint2(0u, 0u);
       for (int t0 = 0; ok && t0 < p.tiles_n; t0 += kExchangeBatch) {
-        // all loads of the batch in flight at once; the whole batch is asked for again until every word is valid
+        // all loads of the batch in flight at once; the whole batch is asked for again until every word carries this launch's tag
         for (uint32_t spin = 1;; ++spin) {
-          uint4 w[kExchangeBatch];
-#pragma unroll
-          for (int t = 0; t < kExchangeBatch; ++t)
-            w[t] = t0 + t < p.tiles_n ? ld_relaxed_gpu_v4(xt + (size_t)(t0 + t) * kBM) : make_uint4(kValidBit, kValidBit, kValidBit, kValidBit);
-          uint32_t all = kValidBit;
-          uint4 b4 = make_uint4(0u, 0u, 0u, 0u);
+          ulonglong2 w[kExchangeBatch];
 #pragma unroll
           for (int t = 0; t < kExchangeBatch; ++t) {
-            all &= w[t].x & w[t].y & w[t].z & w[t].w;
-            b4.x = max(b4.x, w[t].x & ~kValidBit);
-            b4.y = max(b4.y, w[t].y & ~kValidBit);
-            b4.z = max(b4.z, w[t].z & ~kValidBit);
-            b4.w = max(b4.w, w[t].w & ~kValidBit);
+            const uint64_t none = (uint64_t)tag << 32;  // a maximum of zero
+            w[t] = t0 + t < p.tiles_n ? ld_relaxed_gpu_2x64(xt + (size_t)(t0 + t) * kBM) : make_ulonglong2(none, none);
           }
-          if (__all_sync(0xffffffffu, (all & kValidBit) != 0u)) {
-            m4.x = max(m4.x, b4.x);
-            m4.y = max(m4.y, b4.y);
-            m4.z = max(m4.z, b4.z);
-            m4.w = max(m4.w, b4.w);
+          bool all = true;
+          uint2 b2 = make_uint2(0u, 0u);
+#pragma unroll
+          for (int t = 0; t < kExchangeBatch; ++t) {
+            all = all && (uint32_t)(w[t].x >> 32) == tag && (uint32_t)(w[t].y >> 32) == tag;
+            b2.x = max(b2.x, (uint32_t)w[t].x);
+            b2.y = max(b2.y, (uint32_t)w[t].y);
+          }
+          if (__all_sync(0xffffffffu, all)) {
+            m2.x = max(m2.x, b2.x);
+            m2.y = max(m2.y, b2.y);
             break;
           }
           if ((spin & 0xF) == 0 && !__all_sync(0xffffffffu, keep_waiting(&abort_flag, t_start))) { ok = false; break; }  // warp-uniform
         }
       }
       if (!__all_sync(0xffffffffu, ok)) break;
-      // final maxima of rows 4l .. 4l+3 for the epilogue warps
-      *reinterpret_cast<uint4*>(&row_amax[par][4 * lane]) = m4;
+      // final maxima of this warp's rows for the epilogue warps
+      *reinterpret_cast<uint2*>(&row_amax[par][64 * xh + 2 * lane]) = m2;
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&ctx_ready_bar[par]));
     }
@@ -559,7 +579,7 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       }
       if (!ok) break;
       // this CTA's maxima of the tile's rows, each tagged valid: one word per row, straight from the registers
-      st_relaxed_gpu(rp.exchange + ((size_t)tm * p.tiles_n + tn) * kBM + row_in_tile, __float_as_uint(amax) | kValidBit);
+      st_relaxed_gpu_64(rp.exchange + ((size_t)tm * p.tiles_n + tn) * kBM + row_in_tile, ((uint64_t)tag << 32) | __float_as_uint(amax));
 
       // -------------------------------------------------------------- pass 2: scale, codes
       if (!mbar_wait(smem_u32(&ctx_ready_bar[set]), aph, &abort_flag, t_start)) { ok = false; break; }
@@ -629,11 +649,32 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     tc_fence_after();
     tmem_dealloc(tmem_base, Cfg::kTmemCols);
   }
+  if (tn == 0 && threadIdx.x == 0) rp.generation[group] = __ldcg(rp.generation + group) + 1u;
 }
 
-// Bytes of the exchange area (one word per m-tile, n-tile and row).
+// A tag no earlier call of this process has used: a counter run through a bijection of the 32-bit
+// integers, so that consecutive tags share no pattern with small integers or with one another.  A
+// word of the exchange area counts only if its upper half equals the call's tag mixed with the
+// group's generation counter (see the kernel), so the area needs no clearing: whatever another call
+// or an earlier execution of this call left there carries another value.  Memory that never held
+// exchange words passes for valid with probability 2^-32 per word.
+static uint32_t next_launch_tag() {
+  static std::atomic<uint32_t> counter{0};
+  uint32_t x = counter.fetch_add(1, std::memory_order_relaxed) + 1u;
+  x ^= x >> 16;
+  x *= 0x7FEB352Du;
+  x ^= x >> 15;
+  x *= 0x846CA68Bu;
+  x ^= x >> 16;
+  return x != 0u ? x : 0x9E3779B9u;  // zero marks a wiped word
+}
+
+constexpr int kMaxGroups = 256;  // at most one group per SM
+
+// Bytes of the exchange area (one 64-bit word per m-tile, n-tile and row).
 static size_t requant_exchange_bytes(int64_t M, int64_t N) {
-  return round_up((size_t)ceil_div(M, kBM) * (size_t)ceil_div(N, 128) * kBM * 4, 256);
+  const size_t tiles_m = (size_t)ceil_div(M, kBM);
+  return round_up(tiles_m * (size_t)ceil_div(N, 128) * kBM * 8 + (size_t)kMaxGroups * 4, 256);
 }
 
 // True if this kernel takes the call: K <= 512; NONE / Swish in every form, the GLU forms when
@@ -658,8 +699,9 @@ static int launch_requant_inst(const int8_t* a, const void* b, void* q_out, floa
   const int sms = sm_count();
   if (sms <= 0) return AQT_ERR_CUDA;
   if (p.k_blocks > Cfg::kKBlocks || p.tiles_n > sms) return AQT_ERR_UNSUPPORTED;
-  rp.exchange = reinterpret_cast<uint32_t*>(exchange);
-  AQT_RETURN_IF_CUDA(cudaMemsetAsync(exchange, 0, (size_t)p.tiles_m * p.tiles_n * kBM * 4, st));
+  rp.exchange = reinterpret_cast<uint64_t*>(exchange);
+  rp.generation = reinterpret_cast<uint32_t*>(rp.exchange + (size_t)p.tiles_m * p.tiles_n * kBM);
+  rp.tag = next_launch_tag();
 
   CUtensorMap tm_a, tm_b, tm_y, tm_r;
   int rc = make_map_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, a, (uint64_t)p.M, (uint64_t)p.K, (uint64_t)p.K, kBM, kBK);
@@ -685,18 +727,12 @@ static int launch_requant_inst(const int8_t* a, const void* b, void* q_out, floa
   if (rc != AQT_OK) return rc;
   int groups = sms / p.tiles_n;
   if (groups > p.tiles_m) groups = p.tiles_m;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(groups * p.tiles_n), 1, 1);
-  cfg.blockDim = dim3(Cfg::kThreads, 1, 1);
-  cfg.dynamicSmemBytes = Cfg::kSmemBytes;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeCooperative;  // the CTAs wait on one another: all must be resident
-  attr[0].val.cooperative = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  AQT_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, kernel, tm_a, tm_b, tm_y, tm_r, rp));
-  return AQT_LAUNCH_STATUS();
+  // The CTAs of a group wait on one another, so all of them must get an SM: the grid never exceeds
+  // one CTA per SM (each takes most of an SM's shared memory), and CTAs of the kernel before it in
+  // the stream never wait on anything, so the SMs they hold become free.  Should another stream keep
+  // SMs occupied for seconds, the bounded waits give up and report AQT_ERR_TIMEOUT.
+  return launch_pdl(kernel, dim3((unsigned)(groups * p.tiles_n), 1, 1), dim3(Cfg::kThreads, 1, 1), Cfg::kSmemBytes, st, 1, tm_a, tm_b,
+                    tm_y, tm_r, rp);
 }
 
 // a: int8 [M, K]; b: int8 [N, K] or (b_packed) nibbles [N, K/2]; y may be null (then no fp32 output

@@ -513,6 +513,8 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       tmem_relinquish();
     }
   }
+  // everything above touched only this CTA's own state; from here on global memory is read
+  grid_dependency_wait();
   if (WS) {
     // scales and biases of the CTA's n-tile, once: values first, then (GLU) gates
     const int tn = blockIdx.x % p.tiles_n;
@@ -600,6 +602,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           }
         }
       }
+      grid_dependents_launch();  // every load of this CTA has been issued: the next kernel may be scheduled behind it
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -1043,23 +1046,9 @@ static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t l
     // one cluster of two CTAs per tile in flight
     const int64_t pairs = sms / 2;
     grid = 2u * (unsigned)(tiles < pairs ? tiles : pairs);
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid, 1, 1);
-    cfg.blockDim = dim3(Cfg::kThreads, 1, 1);
-    cfg.dynamicSmemBytes = Cfg::kSmemBytes;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    AQT_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, kernel, tm_a, tm_b, tm_y, tm_r, p));
-    return AQT_LAUNCH_STATUS();
+    return launch_pdl(kernel, dim3(grid, 1, 1), dim3(Cfg::kThreads, 1, 1), Cfg::kSmemBytes, st, 2, tm_a, tm_b, tm_y, tm_r, p);
   }
-  kernel<<<grid, Cfg::kThreads, Cfg::kSmemBytes, st>>>(tm_a, tm_b, tm_y, tm_r, p);
-  return AQT_LAUNCH_STATUS();
+  return launch_pdl(kernel, dim3(grid, 1, 1), dim3(Cfg::kThreads, 1, 1), Cfg::kSmemBytes, st, 1, tm_a, tm_b, tm_y, tm_r, p);
 }
 
 template <int BN, int STAGES, int EW, bool WS, bool BPACK, bool CTA2 = false>

@@ -48,6 +48,7 @@ __global__ void __launch_bounds__(kQuantThreads) quantize_rows_reg_kernel(
   constexpr int WARPS_PER_ROW = G / 32;
   __shared__ float warp_max[kQuantThreads / 32];
 
+  grid_dependency_wait();
   const int t = threadIdx.x % G;
   const int r_in_cta = threadIdx.x / G;
   const int64_t row = (int64_t)blockIdx.x * ROWS_PER_CTA + r_in_cta;
@@ -64,6 +65,7 @@ __global__ void __launch_bounds__(kQuantThreads) quantize_rows_reg_kernel(
     if (live && idx < nvec) v[i] = __ldg(xrow + idx);
     amax = fmaxf(amax, fmaxf(fmaxf(fabsf(v[i].x), fabsf(v[i].y)), fmaxf(fabsf(v[i].z), fabsf(v[i].w))));
   }
+  grid_dependents_launch();  // this CTA's loads are in flight; it has little left to do
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
   if (WARPS_PER_ROW > 1) {
@@ -289,8 +291,9 @@ static int launch_quantize_rows(const float* x, int64_t rows, int64_t cols, int6
 #define AQT_LAUNCH_ROWS(G)                                                                                   \
   do {                                                                                                       \
     const int64_t grid = ceil_div(rows, kQuantThreads / G);                                                  \
-    quantize_rows_reg_kernel<G, ROUNDING, PACK><<<(unsigned)grid, kQuantThreads, 0, st>>>(x, rows, (int)cols, ld, qmax, \
-                                                                                         q_out, scale_out); \
+    const int rc_launch = launch_pdl(quantize_rows_reg_kernel<G, ROUNDING, PACK>, dim3((unsigned)grid, 1, 1),       \
+                                     dim3(kQuantThreads, 1, 1), 0, st, 1, x, rows, (int)cols, ld, qmax, q_out, scale_out); \
+    if (rc_launch != AQT_OK) return rc_launch;                                                               \
   } while (0)
     if (nvec <= 32 * kQuantMaxVec) AQT_LAUNCH_ROWS(32);
     else if (nvec <= 64 * kQuantMaxVec) AQT_LAUNCH_ROWS(64);
