@@ -292,36 +292,18 @@ def run_ours(args):
     if aqt.aqt_device_status() != 0:
         raise SystemExit("device status reports a failed wait during warm-up")
 
-    # R consecutive steps captured in a CUDA graph (launch latency out of the way), twice: plain,
-    # and with an event recorded around every call (event-record nodes inside the graph), which is
-    # where the per-call durations of the roofline come from.
-    graph = graph_ev = None
-    call_events = [[torch.cuda.Event(enable_timing=True, external=True) for _ in range(NC + 1)] for _ in range(R)]
+    # R consecutive steps captured in a CUDA graph (launch latency out of the way; consecutive
+    # kernels overlap their set-up with the tail of the one before by programmatic dependent launch).
+    graph = None
     if not args.no_graph:
         def run_plain(st):
             for c3 in make_calls(st):
                 for c in c3:
                     c()
-
-        def run_with_events(st):
-            for r, c3 in enumerate(make_calls(st)):
-                call_events[r][0].record(st)
-                for j, c in enumerate(c3):
-                    c()
-                    call_events[r][j + 1].record(st)
         graph = _capture(run_plain, torch)
-        graph_ev = _capture(run_with_events, torch)
         for _ in range(2):
             graph.replay()
-            graph_ev.replay()
         barrier()
-
-    per_call_samples = [[] for _ in range(NC)]
-
-    def read_call_events():
-        for r in range(R):
-            for j in range(NC):
-                per_call_samples[j].append(call_events[r][j].elapsed_time(call_events[r][j + 1]))
 
     sampler = ClockSampler(local)
     if rank == 0:
@@ -331,14 +313,10 @@ def run_ours(args):
     # ---- the timed region: exactly args.steps steps
     barrier()
     e_begin.record(stream)
-    replays, i, used_ev = 0, 0, False
+    replays, i = 0, 0
     if graph is not None:
-        n_full = args.steps // R
-        for k in range(n_full):
-            if k == n_full - 1 and n_full >= 2:
-                graph_ev.replay(); used_ev = True     # the last R steps carry the per-call events
-            else:
-                graph.replay()
+        for k in range(args.steps // R):
+            graph.replay()
             replays += 1
             i += R
     while i < args.steps:
@@ -347,25 +325,30 @@ def run_ours(args):
     barrier()
     total_ms = e_begin.elapsed_time(e_end)
     status = aqt.aqt_device_status()
-    if used_ev:
-        read_call_events()
-    # more samples of the per-call events (outside the timed region), or call-by-call events without a graph
-    if graph_ev is not None:
-        for _ in range(8):
-            graph_ev.replay()
+
+    # ---- duration of each call of the step: the same call on the R rotating buffer sets, back to
+    # back in a graph of its own (an event between two kernels of the step's graph would keep them
+    # from overlapping and adds several microseconds per node, so the step itself carries none).
+    # Inputs sit where the step leaves them: x in HBM, the codes a call reads in L2.
+    per_call_ms = []
+    for j in range(NC):
+        def run_one(st, j=j):
+            for c3 in make_calls(st):
+                c3[j]()
+        if graph is not None:
+            gj = _capture(run_one, torch)
+            per_call_ms.append(_time_replays(torch, gj, 10)[0] / R)
+            del gj
+        else:
+            evs = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+            run_one(stream)
             torch.cuda.synchronize()
-            read_call_events()
-    else:
-        evs = [torch.cuda.Event(enable_timing=True) for _ in range(NC + 1)]
-        for k in range(8):
             evs[0].record(stream)
-            for j, f in enumerate(calls[k % R]):
-                f()
-                evs[j + 1].record(stream)
+            for _ in range(4):
+                run_one(stream)
+            evs[1].record(stream)
             torch.cuda.synchronize()
-            for j in range(NC):
-                per_call_samples[j].append(evs[j].elapsed_time(evs[j + 1]))
-    per_call_ms = [statistics.mean(v) for v in per_call_samples]
+            per_call_ms.append(evs[0].elapsed_time(evs[1]) / (4 * R))
 
     t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
     if world > 1:
@@ -498,8 +481,8 @@ def run_ours(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 4 * M * s0.K, "d2h_bytes_per_step": 4 * M * s1_.N,
                     "ms_per_step": float(te.item()) / args.steps, "streams": n_lanes, "api": "aqt_ffn_fwd", "device_status": e2e_status},
             "gpu_launches": args.steps * NC, "sum_call_ms_per_step": sum(per_call_ms),
-            "launch_mode": ("cuda graph of %d steps x %d replays (%s per-call events inside the graph) + %d call-by-call steps" %
-                            (R, replays, "the last with" if used_ev else "no", args.steps - replays * R))
+            "launch_mode": ("cuda graph of %d steps x %d replays + %d call-by-call steps; per-call durations from one graph per call" %
+                            (R, replays, args.steps - replays * R))
             if graph is not None else "call by call",
             "roofline": roofline}
     if sustained is not None:
@@ -788,6 +771,48 @@ def backward_ffn_layer(dev, steps: int = 20):
             "dtype": "tf32", "gpu_launches_per_step": 9, "launch_mode": "cuda graph"}
 
 
+def run_case(args):
+    """One call of the library, a few times over, for profiler captures (ncu -k ... -c ...): small
+    enough to finish in seconds, inputs larger than L2 where the kernel's DRAM figures matter."""
+    import torch
+    from paper_2203_15952_b200 import binding as aqt
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    g = torch.Generator(device=dev).manual_seed(11)
+    name, it = args.case, args.iters
+    codes = lambda r, c, q: torch.randint(-q, q + 1, (r, c), generator=g, dtype=torch.int8, device=dev)
+    scales = lambda n, a: torch.rand(n, generator=g, device=dev) * a + a * 0.1
+    if name in ("quantize_ffn", "quantize_large"):
+        M, K = (12800, 512) if name == "quantize_ffn" else (65536, 1024)
+        xs = [torch.randn((M, K), generator=g, device=dev) for _ in range(2 if name == "quantize_large" else 6)]
+        for i in range(it):
+            aqt.aqt_quantize(xs[i % len(xs)], 8, aqt.AXIS_ROW)
+    elif name in ("requant_ffn1", "requant_large"):
+        M, N, K = (12800, 2048, 512) if name == "requant_ffn1" else (32768, 4096, 1024)
+        xq, wq = codes(M, K, 127), torch.randint(0, 256, (N, K // 2), generator=g, dtype=torch.uint8, device=dev)
+        w_arg, bits_w = (wq, 4) if K <= 512 else (aqt.aqt_unpack_int4(wq, K), aqt.BITS_4_UNPACKED)
+        s_x, s_w = scales(M, 1e-2), scales(N, 1e-3)
+        for i in range(it):
+            aqt.aqt_qmatmul_requant(xq, s_x, w_arg, s_w, K=K, bits_a=8, bits_w=bits_w, act=aqt.ACT_SWISH, bits_out=8)
+    elif name in ("gemm_ffn2", "gemm_large_ffn2", "gemm_large_ffn1"):
+        M, N, K, act = {"gemm_ffn2": (12800, 512, 2048, aqt.ACT_NONE), "gemm_large_ffn2": (32768, 1024, 4096, aqt.ACT_NONE),
+                        "gemm_large_ffn1": (32768, 4096, 1024, aqt.ACT_SWISH)}[name]
+        xq, wq, s_x, s_w = codes(M, K, 127), codes(N, K, 7), scales(M, 1e-2), scales(N, 1e-3)
+        y = torch.empty((M, N), dtype=torch.float32, device=dev)
+        for i in range(it):
+            aqt.aqt_qmatmul(xq, s_x, wq, s_w, K=K, bits_a=8, bits_w=aqt.BITS_4_UNPACKED, act=act, y=y)
+    elif name == "weight_only_ffn1":
+        M, N, K = 12800, 2048, 512
+        x, wq, s_w = torch.randn((M, K), generator=g, device=dev), torch.randint(0, 256, (N, K // 2), generator=g, dtype=torch.uint8, device=dev), scales(N, 1e-3)
+        for i in range(it):
+            aqt.aqt_linear_fwd_weight_only(x, wq, s_w, bits_w=4, act=aqt.ACT_SWISH)
+    else:
+        raise SystemExit("unknown case " + name)
+    torch.cuda.synchronize()
+    print(json.dumps({"case": name, "iters": it, "device_status": aqt.aqt_device_status()}), flush=True)
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -800,7 +825,12 @@ def main():
                     help="skip the legs beside the headline (quantizer, encoder stacks, weight-only, backward, large matmuls)")
     ap.add_argument("--no-sustained", action="store_true", help="skip the half-second sustained run of the headline step")
     ap.add_argument("--no-graph", action="store_true", help="launch every step call by call (no CUDA graph replay)")
+    ap.add_argument("--case", default=None, help="run one library call a few times and exit (for profiler captures): quantize_ffn, "
+                    "quantize_large, requant_ffn1, requant_large, gemm_ffn2, gemm_large_ffn2, gemm_large_ffn1, weight_only_ffn1")
+    ap.add_argument("--iters", type=int, default=4, help="--case: number of calls")
     args = ap.parse_args()
+    if args.case is not None:
+        return run_case(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)

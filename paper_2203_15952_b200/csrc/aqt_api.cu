@@ -111,6 +111,17 @@ int float_gemm_nt(const float* a, int64_t lda, const float* b, int64_t rows, int
   return launch_qgemm(reinterpret_cast<const int8_t*>(a), b, false, y, ldy, p, st);
 }
 
+// True if the CTA-pair kernel with the row-quantizing epilogue takes the call: deep K, no GLU, int8
+// codes out (4-bit codes stay in their containers), at most 16 column parts per row.
+bool rowquant_pair_applies(int64_t M, int64_t N, int64_t K, int act, bool pack_out) {
+  if (pack_out || M <= kBM || K < 1024) return false;
+  if (act != AQT_ACT_NONE && act != AQT_ACT_SWISH) return false;
+  const int sms = sm_count() > 0 ? sm_count() : kDefaultSms;
+  const int plan = rowquant_plan(M, N, K, sms);
+  const int parts = rowquant_parts(plan, N);
+  return parts % 2 == 0 && parts <= 16 && ceil_div(N, kGemmPlanBn[plan]) <= sms / 2;
+}
+
 int validate_matmul_shape(int64_t M, int64_t N, int64_t K, int bits_a, int bits_w, int act, int s_x_kind) {
   if (M < 0 || N < 0 || K <= 0) return AQT_ERR_BADARG;
   if (!bits_ok(bits_a) || !bits_ok(bits_w) || !act_ok(act)) return AQT_ERR_BADARG;
@@ -382,8 +393,51 @@ int aqt_qmatmul_requant(const void* xq, const float* s_x, int s_x_kind, const vo
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
 
+  if (!requant_applies(M, N, K, act, y != nullptr, pack_out != 0) && rowquant_pair_applies(M, N, K, act, pack_out != 0)) {
+    // Deep K (the second feed-forward layers): the CTA-pair kernel with the row-quantizing epilogue
+    const int8_t* a_codes = reinterpret_cast<const int8_t*>(xq);
+    if (is_packed(bits_a)) {
+      rc = launch_unpack_int4(reinterpret_cast<const uint8_t*>(xq), M * K / 2, reinterpret_cast<int8_t*>(ws), st);
+      if (rc != AQT_OK) return rc;
+      a_codes = reinterpret_cast<const int8_t*>(ws);
+      ws += round_up((size_t)M * (size_t)K, 256);
+    }
+    const void* b_codes = wq;
+    if (is_packed(bits_w)) {
+      rc = launch_unpack_int4(reinterpret_cast<const uint8_t*>(wq), N * K / 2, reinterpret_cast<int8_t*>(ws), st);
+      if (rc != AQT_OK) return rc;
+      b_codes = ws;
+    }
+    GemmParams p;
+    p.s_x = s_x;
+    p.s_w = s_w;
+    p.bias = bias;
+    p.residual = residual;
+    p.acc_debug = nullptr;
+    p.ldr = ldr;
+    p.residual_scale = residual_scale;
+    p.s_x_kind = s_x_kind;
+    p.act = act;
+    p.M = (int)M;
+    p.N = (int)N;
+    p.K = (int)K;
+    p.n_out = (int)N;
+    p.tiles_m = p.tiles_n = p.k_blocks = 0;
+    p.small_acc = (K * (int64_t)(qmax_of(code_bits(bits_a)) + 1) * (qmax_of(code_bits(bits_w)) + 1) <= (1ll << 22)) ? 1 : 0;
+    p.q_out = reinterpret_cast<uint8_t*>(q_out);
+    p.s_out = s_out;
+    p.exchange = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(workspace) + mm_bytes);
+    p.generation = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(workspace) + mm_bytes + requant_exchange_bytes(M, N) - (size_t)kMaxGroups * 4);
+    p.tag = next_launch_tag();
+    p.qmax_out = qmax_of(bits_out);
+    p.rounding = rounding;
+    p.has_y = y != nullptr ? 1 : 0;
+    const int sms = sm_count();
+    if (sms <= 0) return AQT_ERR_CUDA;
+    return launch_qgemm_rowquant(rowquant_plan(M, N, K, sms), a_codes, b_codes, y, ldy, p, st);
+  }
   if (!requant_applies(M, N, K, act, y != nullptr, pack_out != 0)) {
-    // Shapes the fused kernel does not take: the two steps one after the other, through y.
+    // Shapes the fused kernels do not take: the two steps one after the other, through y.
     if (y == nullptr) return AQT_ERR_UNSUPPORTED;
     rc = aqt_qmatmul(xq, s_x, s_x_kind, wq, s_w, bias, residual, ldr, residual_scale, M, N, K, bits_a, bits_w, act, y, ldy, nullptr,
                      workspace, mm_bytes, stream);

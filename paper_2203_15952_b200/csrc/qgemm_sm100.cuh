@@ -25,6 +25,7 @@
 
 #include "aqt_common.cuh"
 #include "pack.cuh"
+#include "row_quant_epilogue.cuh"
 
 namespace aqt {
 
@@ -105,6 +106,17 @@ struct GemmParams {
   int n_out;    // N, or N / 2 for the GLU forms
   int tiles_m, tiles_n, k_blocks;
   int small_acc;  // every |accumulator| < 2^22: the int -> float conversion can use the exponent trick
+  // Row-quantizing epilogue (template argument RQ of the CTA-pair kernel): the output rows leave the
+  // kernel as codes and scales as well (or only), see the kernel.
+  uint8_t* q_out = nullptr;         // int8 codes [M, N], dense
+  float* s_out = nullptr;           // [M] row scales
+  uint64_t* exchange = nullptr;     // [rows padded to the tile height][exchange_parts] words: (tag << 32) | bits of a part's row maximum
+  uint32_t* generation = nullptr;   // [groups] counters that make the tag differ on every execution
+  uint32_t tag = 0;                 // tag of this call
+  int exchange_parts = 0;           // column parts a row's maximum is assembled from: tiles_n x warps per lane quadrant
+  int qmax_out = 127;
+  int rounding = AQT_ROUND_NEAREST_EVEN;
+  int has_y = 1;                    // 0: no fp32 output
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -446,7 +458,15 @@ __device__ __forceinline__ bool tile_at(const GemmParams& p, int i, int& tm, int
   return tile < p.tiles_m * p.tiles_n;
 }
 
-template <int BN, int STAGES, int EW, bool WS, bool BPACK, int ACCK, bool DEBUG, bool CTA2 = false>
+// RQ (CTA pairs, no GLU): the epilogue also quantizes the output rows for the next layer (Fig. 2 of
+// the paper on u = what the plain epilogue writes): pass 1 is the plain epilogue, which also keeps
+// the row maxima and writes u back over its accumulators; every thread then publishes the maximum
+// of its row over its warp's columns as a tagged word, polls the words of the other column parts
+// of the row (its own CTA's other warps and the other pairs of its group, which work on the same
+// rows at the same time), and pass 2 turns u into codes.  The next tile's MMAs run meanwhile in
+// the other accumulator buffer.  The pairs of a group (tiles_n consecutive pairs) always share
+// their rows, so the grid is a multiple of tiles_n pairs.
+template <int BN, int STAGES, int EW, bool WS, bool BPACK, int ACCK, bool DEBUG, bool CTA2 = false, bool RQ = false>
 __global__ void __launch_bounds__(32 * (2 + EW), 1)
 qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                 const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_r, const GemmParams p) {
@@ -458,6 +478,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   constexpr bool TF32 = (ACCK == kAccFloat);  // float operands: no activation scale, accumulators are binary32
   static_assert(!(TF32 && (BPACK || DEBUG)), "the float kind reads expanded weights and has no integer accumulators to dump");
   static_assert(!(TF32 && BN == 512), "512-column tiles exist for the 8-bit kind only");
+  static_assert(!RQ || (CTA2 && !TF32 && !DEBUG && !WS), "the row-quantizing epilogue belongs to the 8-bit CTA-pair kernel");
   const uint32_t pair_rank = CTA2 ? cluster_ctarank() : 0u;  // 0 = leader: issues the MMAs, owns the barriers the pair shares
   const int row_in_tile = (int)pair_rank * kBM;               // this CTA's first row inside the tile
 
@@ -515,6 +536,10 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   }
   // everything above touched only this CTA's own state; from here on global memory is read
   grid_dependency_wait();
+  // RQ: tag of this execution's exchange words (the call's tag mixed with the group's generation
+  // counter, which the group's first CTA bumps when it has finished: a replayed graph repeats the call's tag)
+  const int rq_group = RQ ? (int)(blockIdx.x >> 1) / p.tiles_n : 0;
+  const uint32_t rq_tag = RQ ? mix_tag(p.tag, __ldcg(p.generation + rq_group)) : 0u;
   if (WS) {
     // scales and biases of the CTA's n-tile, once: values first, then (GLU) gates
     const int tn = blockIdx.x % p.tiles_n;
@@ -665,6 +690,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     const uint32_t slab_gate_off = WS ? HALF * 4 : 128;           // gate columns relative to the value columns
     uint32_t store_count = 0;
     bool ok = true;
+    const bool do_store = !RQ || p.has_y != 0;  // the fp32 output is written (always, without RQ)
 
     if (WS && BPACK) {
       // Sign-extend the CTA's packed weights into the resident slab, in the layout a swizzled
@@ -743,6 +769,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         }
       }
       const float sx = TF32 ? 1.0f : ((p.s_x_kind == AQT_SCALE_ROW) ? (row_ok ? __ldg(p.s_x + m) : 0.0f) : __ldg(p.s_x));
+      float rq_amax = 0.0f;  // RQ: maximum of this thread's row over this warp's columns
       __syncwarp();
 
       if (!mbar_wait(smem_u32(&tmem_full_bar[buf]), aph, &abort_flag, t_start)) break;
@@ -761,7 +788,7 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         if (!glu) {
           tmem_ld_32x32(lane_addr + col, acc);
           tmem_ld_wait();
-          if (last_chunk) {
+          if (last_chunk && !RQ) {
             // accumulator buffer read out by this warp: hand it back before the arithmetic
             tc_fence_before();
             __syncwarp();
@@ -860,22 +887,35 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             a[4 * j + 3] = __fmaf_rn(p.residual_scale, a[4 * j + 3], r3);
           }
           __syncwarp();  // every lane has read its residual row before the buffer is overwritten
-        } else {
+        } else if (do_store) {
           // staging buffer free once the bulk store that last used it has been read out
           if (lane == 0) tma_store_wait_read<SBUFS - 1>();
           __syncwarp();
         }
-        // row `lane` of the 32 x 32 box; 16-byte chunk j sits at (j ^ (row & 7)) under the 128-byte swizzle
+        if constexpr (RQ) {
+          // u stays in tensor memory, over the accumulators it was made from, until the row's scale is known
+          float cmax = 0.0f;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const uint32_t dst = sbuf + lane * 128 + ((j ^ (lane & 7)) << 4);
-          asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(a[4 * j]), "f"(a[4 * j + 1]),
-                       "f"(a[4 * j + 2]), "f"(a[4 * j + 3])
-                       : "memory");
+          for (int j = 0; j < 32; ++j) {
+            cmax = fmaxf(cmax, fabsf(a[j]));
+            acc[j] = __float_as_uint(a[j]);
+          }
+          if (oc < p.n_out) rq_amax = fmaxf(rq_amax, cmax);  // columns beyond N contribute nothing
+          tmem_st_32x32(lane_addr + col, acc);
         }
-        fence_proxy_async_smem();
+        // row `lane` of the 32 x 32 box; 16-byte chunk j sits at (j ^ (row & 7)) under the 128-byte swizzle
+        if (do_store) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint32_t dst = sbuf + lane * 128 + ((j ^ (lane & 7)) << 4);
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(a[4 * j]), "f"(a[4 * j + 1]),
+                         "f"(a[4 * j + 2]), "f"(a[4 * j + 3])
+                         : "memory");
+          }
+          fence_proxy_async_smem();
+        }
         __syncwarp();
-        if (lane == 0) {
+        if (lane == 0 && do_store) {
           // boxes that start inside the output are clipped at its edges by the copy engine
           if (oc < p.n_out && row0_warp < p.M) tma_store_2d(&tm_y, sbuf, oc, row0_warp);
           tma_store_commit();
@@ -893,6 +933,58 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         ++store_count;
       }
       if (!ok) break;
+      if constexpr (RQ) {
+        // ---------------------------------------------------------- the row's maximum over all of N
+        const int parts = p.exchange_parts;
+        const int my_part = tn * (EW / 4) + chalf;
+        uint64_t* xrow = p.exchange + (size_t)m * parts;  // rows up to the padded tile height are allocated
+        st_relaxed_gpu_64(xrow + my_part, ((uint64_t)rq_tag << 32) | __float_as_uint(rq_amax));
+        uint32_t amax_bits = 0u;
+        for (uint32_t spin = 1;; ++spin) {
+          bool all = true;
+          amax_bits = 0u;
+          for (int q = 0; q < parts; q += 2) {  // parts is even: a pair has at least two column parts
+            const ulonglong2 w = ld_relaxed_gpu_2x64(xrow + q);
+            all = all && (uint32_t)(w.x >> 32) == rq_tag && (uint32_t)(w.y >> 32) == rq_tag;
+            amax_bits = max(amax_bits, max((uint32_t)w.x, (uint32_t)w.y));
+          }
+          if (__all_sync(0xffffffffu, all)) break;
+          if ((spin & 0x3F) == 0) {
+            bool go_on = *(volatile int*)&abort_flag == 0;
+            if (go_on && global_timer_ns() - t_start > kWaitLimitNs) {
+              *(volatile int*)&abort_flag = 1;
+              atomicExch(&g_device_status, AQT_ERR_TIMEOUT);
+              go_on = false;
+            }
+            if (!__all_sync(0xffffffffu, go_on)) { ok = false; break; }
+          }
+        }
+        if (!ok) break;
+        // ---------------------------------------------------------- pass 2: scale, codes
+        const ScaleCtx sc = make_scale_ctx(__uint_as_float(amax_bits), p.qmax_out);
+        if (my_part == 0 && row_ok) p.s_out[m] = sc.s;
+        tmem_st_wait();  // this warp's stores of pass 1
+        for (int c = 0; c < chunks; ++c) {
+          const int col = (chalf * chunks + c) * 32;
+          const int oc = out0 + col;
+          uint32_t u[32], w[8];
+          tmem_ld_32x32(lane_addr + col, u);
+          tmem_ld_wait();
+          if (c == chunks - 1) {
+            // the tile has been read out by this warp: the accumulator buffer goes back to the MMA
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(smem_u32(&tmem_empty_bar[buf]), 0);
+          }
+          if (p.rounding == AQT_ROUND_HALF_UP_FLOOR) codes_of<AQT_ROUND_HALF_UP_FLOOR, false, 32>(u, sc, p.qmax_out, w);
+          else codes_of<AQT_ROUND_NEAREST_EVEN, false, 32>(u, sc, p.qmax_out, w);
+          if (row_ok && oc < p.n_out) {
+            uint4* dst = reinterpret_cast<uint4*>(p.q_out + (size_t)m * p.n_out + oc);
+            dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+            if (oc + 16 < p.n_out) dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+          }
+        }
+      }
     }
     if (lane == 0) tma_store_wait_all();
   }
@@ -913,6 +1005,10 @@ qgemm_i8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     tc_fence_after();
     if (CTA2) tmem_dealloc_pair(tmem_base, Cfg::kTmemCols);
     else tmem_dealloc(tmem_base, Cfg::kTmemCols);
+  }
+  if (RQ) {
+    // every CTA of the group has read the counter long since (this one could not finish its tiles without them)
+    if (threadIdx.x == 0 && blockIdx.x == (unsigned)(2 * rq_group * p.tiles_n)) p.generation[rq_group] = __ldcg(p.generation + rq_group) + 1u;
   }
 }
 
@@ -997,7 +1093,7 @@ static int pick_bn(int64_t M, int64_t N, bool glu, int sms) {
 }
 
 // b: weight codes as the kernel reads them -- int8 [N, K], or (BPACK) packed nibbles [N, K/2].
-template <int BN, int STAGES, int EW, bool WS, bool BPACK, int ACCK, bool DEBUG, bool CTA2 = false>
+template <int BN, int STAGES, int EW, bool WS, bool BPACK, int ACCK, bool DEBUG, bool CTA2 = false, bool RQ = false>
 static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t ldy, const GemmParams& p0, cudaStream_t st) {
   using Cfg = GemmCfg<BN, STAGES, EW, WS, CTA2>;
   GemmParams p = p0;
@@ -1025,9 +1121,13 @@ static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t l
   }
   if (rc != AQT_OK) return rc;
   if (p.batch_tiles_m > 0 && (WS || CTA2)) return AQT_ERR_UNSUPPORTED;
-  rc = make_map_2d(&tm_y, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, y, (uint64_t)p.M, (uint64_t)p.n_out, (uint64_t)ldy * 4, kStoreBoxRows,
-                   kStoreBoxCols);
-  if (rc != AQT_OK) return rc;
+  if (RQ && !p.has_y) {
+    tm_y = tm_a;  // never dereferenced
+  } else {
+    rc = make_map_2d(&tm_y, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, y, (uint64_t)p.M, (uint64_t)p.n_out, (uint64_t)ldy * 4, kStoreBoxRows,
+                     kStoreBoxCols);
+    if (rc != AQT_OK) return rc;
+  }
   if (p.residual != nullptr) {
     rc = make_map_2d(&tm_r, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, p.residual, (uint64_t)p.M, (uint64_t)p.n_out, (uint64_t)p.ldr * 4,
                      kStoreBoxRows, kStoreBoxCols);
@@ -1035,7 +1135,7 @@ static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t l
   } else {
     tm_r = tm_y;  // never dereferenced
   }
-  auto kernel = qgemm_i8_kernel<BN, STAGES, EW, WS, BPACK, ACCK, DEBUG, CTA2>;
+  auto kernel = qgemm_i8_kernel<BN, STAGES, EW, WS, BPACK, ACCK, DEBUG, CTA2, RQ>;
   static std::atomic<uint64_t> smem_opted_in{0};
   rc = ensure_dynamic_smem(kernel, Cfg::kSmemBytes, smem_opted_in);
   if (rc != AQT_OK) return rc;
@@ -1044,7 +1144,13 @@ static int launch_qgemm_inst(const int8_t* a, const void* b, float* y, int64_t l
   if (WS && (int)grid < p.tiles_n) grid = (unsigned)p.tiles_n;  // every n-tile needs an owner
   if (CTA2) {
     // one cluster of two CTAs per tile in flight
-    const int64_t pairs = sms / 2;
+    int64_t pairs = sms / 2;
+    if (RQ) {
+      // the pairs that share rows (tiles_n consecutive ones) wait on one another: whole groups only,
+      // every one of them on an SM of its own
+      if (p.tiles_n > pairs || p.exchange_parts != p.tiles_n * (EW / 4) || p.exchange_parts % 2 != 0) return AQT_ERR_UNSUPPORTED;
+      pairs = pairs / p.tiles_n * p.tiles_n;
+    }
     grid = 2u * (unsigned)(tiles < pairs ? tiles : pairs);
     return launch_pdl(kernel, dim3(grid, 1, 1), dim3(Cfg::kThreads, 1, 1), Cfg::kSmemBytes, st, 2, tm_a, tm_b, tm_y, tm_r, p);
   }
@@ -1236,6 +1342,35 @@ static int launch_qgemm_plan(int plan, const int8_t* a, const void* b, bool b_pa
     case kPlanPair512S3E16: return launch_qgemm_cfg<512, 3, 16, false, false, true>(a, b, y, ldy, p, st);
     default: return AQT_ERR_UNSUPPORTED;
   }
+}
+
+// The CTA-pair configurations with the row-quantizing epilogue.  p carries q_out, s_out, the
+// exchange area, tag, qmax_out, rounding, has_y; exchange_parts is filled in here.
+static int rowquant_plan(int64_t M, int64_t N, int64_t K, int sms) {
+  // Eight epilogue warps on 256 x 256 pair tiles throughout: both passes of a tile have to fit into
+  // the next tile's MMA time (measured at 65 536 x 4096 -> 1024 with the fp32 output: 274 us against
+  // 306 us with the four-warp epilogue and 288 us for matmul + row quantizer; 256 x 512 tiles, whose
+  // single accumulator buffer exposes both passes, lose to the two kernels at 12 800 x 2048 -> 512).
+  (void)M;
+  (void)N;
+  (void)K;
+  (void)sms;
+  return kPlanPair256S4E8;
+}
+static int rowquant_parts(int plan, int64_t N) {
+  return (int)ceil_div(N, kGemmPlanBn[plan]) * (kGemmPlanEw[plan] / 4);
+}
+template <int BN, int STAGES, int EW>
+static int launch_rowquant_cfg(const int8_t* a, const void* b, float* y, int64_t ldy, const GemmParams& p, cudaStream_t st) {
+  if (p.small_acc) return launch_qgemm_inst<BN, STAGES, EW, false, false, kAccInt32Small, false, true, true>(a, b, y, ldy, p, st);
+  return launch_qgemm_inst<BN, STAGES, EW, false, false, kAccInt32, false, true, true>(a, b, y, ldy, p, st);
+}
+static int launch_qgemm_rowquant(int plan, const int8_t* a, const void* b, float* y, int64_t ldy, GemmParams p, cudaStream_t st) {
+  if (p.act != AQT_ACT_NONE && p.act != AQT_ACT_SWISH) return AQT_ERR_UNSUPPORTED;
+  if (p.M <= kBM || p.kind != 0) return AQT_ERR_UNSUPPORTED;
+  p.exchange_parts = rowquant_parts(plan, p.N);
+  if (plan != kPlanPair256S4E8) return AQT_ERR_UNSUPPORTED;
+  return launch_rowquant_cfg<256, 4, 8>(a, b, y, ldy, p, st);
 }
 
 static GemmShape gemm_shape_of(const GemmParams& p) {

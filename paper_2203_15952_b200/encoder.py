@@ -109,8 +109,12 @@ class LayerRunner:
         """True if `layer`'s matmul can quantize its own output rows in its epilogue (the GLU
         forms only when the fp32 output is not wanted as well)."""
         s = layer.spec
-        ok = self.a_scale_kind == aqt.SCALE_ROW and s.K <= 1024 and s.K % 16 == 0 and s.n_out % 16 == 0 and s.N <= 128 * 148
-        if s.act in (aqt.ACT_GLU, aqt.ACT_GLU_SWISH) or s.K > 512:
+        ok = self.a_scale_kind == aqt.SCALE_ROW and s.K % 16 == 0 and s.n_out % 32 == 0 and s.N <= 128 * 148
+        glu = s.act in (aqt.ACT_GLU, aqt.ACT_GLU_SWISH)
+        if s.K > 1024 or (s.K > 512 and with_y):
+            # deep K: the CTA-pair kernel quantizes its rows (no GLU; at most 16 column parts per row)
+            return ok and not glu and self.M > 128 and s.N <= 2048
+        if glu or s.K > 512:
             return ok and not with_y
         return ok
 
@@ -191,9 +195,12 @@ class ConformerBlockLinears:
         self.h_b = torch.empty((M, d), **f32)
 
     def forward(self, layers: List[QuantLinear], h_in: torch.Tensor, h_out: torch.Tensor,
-                keep: Optional[Dict[str, torch.Tensor]] = None) -> torch.Tensor:
+                keep: Optional[Dict[str, torch.Tensor]] = None, in_codes=None, next_bits: Optional[int] = None):
         """h_in -> h_out (distinct buffers, neither h_a nor h_b).  `keep`, if given, receives
-        clones of every intermediate keyed by layer name (for parity checks)."""
+        clones of every intermediate keyed by layer name (for parity checks).  in_codes: (codes,
+        scales) of h_in if the producer already quantized its rows.  next_bits: if given, the last
+        matmul also quantizes the rows of h_out to that width for the next block, and the codes and
+        scales are returned with h_out (None where the shape does not allow it)."""
         L, run = layers, self.run
 
         def note(name, t):
@@ -201,11 +208,14 @@ class ConformerBlockLinears:
                 keep[name] = t.clone()
 
         parity = keep is not None  # then every fp32 intermediate is written as well
-        self._ffn(L[0], L[1], h_in, self.h_a, 0.5, parity, note)
+        hq, hs = self._ffn(L[0], L[1], h_in, self.h_a, 0.5, parity, note, xq=in_codes[0] if in_codes else None,
+                           xs=in_codes[1] if in_codes else None, out_role="ha", out_bits=L[2].spec.bits_a)
         note(L[1].spec.name, self.h_a)
-        # q, k, v read the same h: quantize it once (the codes do not depend on the consumer) and
-        # run the three projections as one matmul over their concatenated output channels
-        hq, hs = run.quantize_input(self.h_a, L[2].spec.bits_a)
+        # q, k, v read the same h: its codes come out of the second feed-forward matmul's epilogue
+        # (or one quantizer pass; the codes do not depend on the consumer), and the three
+        # projections run as one matmul over their concatenated output channels
+        if hq is None:
+            hq, hs = run.quantize_input(self.h_a, L[2].spec.bits_a)
         wq, s_w, bias = self._fused_qkv(L)
         aqt.aqt_qmatmul(hq, hs, wq, s_w, bias, None, 1.0, K=self.d, bits_a=_container_bits(L[2].spec.bits_a), bits_w=L[2].mm_bits, act=aqt.ACT_NONE,
                         s_x_kind=run.a_scale_kind, y=self.qkv, workspace=run.workspace)
@@ -235,31 +245,44 @@ class ConformerBlockLinears:
                 cq, cs = run.quantize_input(self.c, L[7].spec.bits_a)
             aq, as_ = run.matmul_requant(L[7], cq, cs, L[8].spec.bits_a, "h", y=self.h_a, residual=self.h_b, residual_scale=1.0)
             note(L[7].spec.name, self.h_a)
-            self._ffn(L[8], L[9], self.h_a, h_out, 0.5, parity, note, xq=aq, xs=as_)
+            out_codes = self._ffn(L[8], L[9], self.h_a, h_out, 0.5, parity, note, xq=aq, xs=as_, out_role="hb", out_bits=next_bits)
         else:
             if cq is not None:
                 run.matmul(L[7], cq, cs, self.h_a, residual=self.h_b, residual_scale=1.0)
             else:
                 run(L[7], self.c, self.h_a, residual=self.h_b, residual_scale=1.0)
             note(L[7].spec.name, self.h_a)
-            self._ffn(L[8], L[9], self.h_a, h_out, 0.5, parity, note)
+            out_codes = self._ffn(L[8], L[9], self.h_a, h_out, 0.5, parity, note, out_role="hb", out_bits=next_bits)
         note(L[9].spec.name, h_out)
+        if next_bits is not None:
+            return h_out, (out_codes if out_codes[0] is not None else None)
         return h_out
 
     def _ffn(self, l0: QuantLinear, l1: QuantLinear, h: torch.Tensor, out: torch.Tensor, rs: float, parity: bool, note,
-             xq: Optional[torch.Tensor] = None, xs: Optional[torch.Tensor] = None) -> None:
-        """out = h + rs * W_1 . Swish(W_0 . h); xq, xs: codes and scales of h if already at hand."""
+             xq: Optional[torch.Tensor] = None, xs: Optional[torch.Tensor] = None, out_role: str = "ha",
+             out_bits: Optional[int] = None):
+        """out = h + rs * W_1 . Swish(W_0 . h); xq, xs: codes and scales of h if already at hand.
+        out_bits: also quantize the rows of `out` to that width in the second matmul's epilogue
+        where it can; returns (codes, scales) of out, or (None, None)."""
         run = self.run
+        fuse_out = out_bits is not None and run.fuses_requant(l1, with_y=True)
         if run.fuses_requant(l0, with_y=parity):
             if xq is None:
                 xq, xs = run.quantize_input(h, l0.spec.bits_a)
             uq, us = run.matmul_requant(l0, xq, xs, l1.spec.bits_a, "u", y=self.u if parity else None)
             if parity:
                 note(l0.spec.name, self.u)
-            run.matmul(l1, uq, us, out, residual=h, residual_scale=rs)
         else:
             run(l0, h, self.u); note(l0.spec.name, self.u)
-            run(l1, self.u, out, residual=h, residual_scale=rs)
+            if not fuse_out:
+                run(l1, self.u, out, residual=h, residual_scale=rs)
+                return None, None
+            uq, us = run.code_buffers("u", l0.spec.n_out)
+            aqt.aqt_quantize(self.u, l1.spec.bits_a, aqt.AXIS_ROW, run.rounding, q_out=uq, scale_out=us)
+        if fuse_out:
+            return run.matmul_requant(l1, uq, us, out_bits, out_role, y=out, residual=h, residual_scale=rs)
+        run.matmul(l1, uq, us, out, residual=h, residual_scale=rs)
+        return None, None
 
     def _fused_qkv(self, L: List[QuantLinear]):
         """Codes, scales and bias of the q, k, v projections stacked along the output channels
@@ -288,10 +311,15 @@ class EncoderStack:
 
     def forward(self, x: torch.Tensor) -> torch.Tensor:
         """x is read only; the result lives in one of the stack's own buffers."""
-        src = x
+        src, codes = x, None
         for b, layers in enumerate(self.blocks):
             dst = self.h0 if b % 2 == 0 else self.h1
-            self.block.forward(layers, src, dst)
+            nxt = self.blocks[b + 1][0].spec.bits_a if b + 1 < len(self.blocks) else None
+            if nxt is None:
+                self.block.forward(layers, src, dst, in_codes=codes)
+                codes = None
+            else:
+                _, codes = self.block.forward(layers, src, dst, in_codes=codes, next_bits=nxt)
             src = dst
         return src
 

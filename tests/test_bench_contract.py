@@ -52,8 +52,8 @@ def test_gpu_arm_prints_the_contract_line_with_roofline_and_e2e():
     r = d["roofline"]
     assert r["bound"] in ("hbm", "tensor", "alu") and 0 < r["frac"] < 1.5 and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
     assert len(r["calls"]) == 3 and abs(sum(c["share"] for c in r["calls"]) - 1.0) < 1e-9
-    # per-call durations come from events inside the replayed graph: together they are the step
-    assert 0.7 < d["sum_call_ms_per_step"] / d["sustained"]["ms_per_step"] < 1.3
+    # the calls timed one by one add up to the step (they overlap a little inside it)
+    assert 0.8 < d["sum_call_ms_per_step"] / d["sustained"]["ms_per_step"] < 1.25
     assert d["sustained"]["seconds"] >= 0.5 and d["clocks"]["samples"] >= 4
     e = d["e2e"]
     assert e["h2d_bytes_per_step"] == 4 * 12800 * 512 and e["d2h_bytes_per_step"] == 4 * 12800 * 512 and 0 < e["value"] < d["value"]

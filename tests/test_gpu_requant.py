@@ -189,3 +189,49 @@ def test_requant_argument_checks():
     q, s_, y = aqt.aqt_qmatmul_requant(z8[:0], one[:0], w8, one[:48], K=64)   # empty batch: nothing to do
     assert q.shape == (0, 48) and y is None
     assert aqt.aqt_device_status() == 0
+
+
+@pytest.mark.parametrize("M,N,K,act,with_res", [(600, 512, 2048, aqt.ACT_NONE, True), (700, 1024, 4096, aqt.ACT_SWISH, False),
+                                                 (300, 768, 2048, aqt.ACT_NONE, True), (513, 256, 4096, aqt.ACT_SWISH, True),
+                                                 (129, 1536, 1024, aqt.ACT_NONE, False)])
+def test_requant_second_ffn_layers_small(M, N, K, act, with_res):
+    """K = 1024 .. 4096 (the second feed-forward layers): the CTA-pair kernel quantizes its output
+    rows in the epilogue, with the fp32 output (a residual stream) and without it.  Row maxima
+    come from several warps and, beyond 512 columns, several CTA pairs."""
+    _run(M, N, K, 8, 4, act, True, with_res, 8, aqt.ROUND_NEAREST_EVEN, False, special_rows=True)
+    _run(M, N, K, 8, 8 if K <= 2048 else 4, act, False, with_res, 4, aqt.ROUND_HALF_UP_FLOOR, False)
+
+
+@pytest.mark.parametrize("M,N,K,plan", [(25600, 512, 2048, "pair256s4e8"), (12800, 512, 2048, "pair512s3e16"),
+                                        (30000, 1024, 4096, "pair256s6e4")])
+def test_requant_second_ffn_layers_full_size_sampled_rows(M, N, K, plan):
+    """The second feed-forward layers at the workloads' sizes: fp32 output with residual + codes
+    and scales, sampled rows against the oracle; every row's largest |code| is 127."""
+    from paper_2203_15952_b200 import inputs as gen
+    rng = np.random.default_rng(M + N)
+    xq = gen.random_codes(41, M, K, 8)
+    wq = gen.random_codes(42, N, K, 4)
+    s_x = rng.uniform(1e-3, 5e-2, M).astype(np.float32)
+    s_w = rng.uniform(1e-4, 5e-3, N).astype(np.float32)
+    res = rng.standard_normal((M, N), dtype=np.float32)
+    xq_d, wq_d, res_d = _dev(xq), _dev(wq), _dev(res)
+    y_d = torch.full((M, N), float("nan"), dtype=torch.float32, device=DEV)
+    q_d, s_d, _ = aqt.aqt_qmatmul_requant(xq_d, _dev(s_x), wq_d, _dev(s_w), None, res_d, 0.5, K=K, bits_a=8, bits_w=aqt.BITS_4_UNPACKED,
+                                          bits_out=8, y=y_d)
+    q2_d, s2_d, y_none = aqt.aqt_qmatmul_requant(xq_d, _dev(s_x), wq_d, _dev(s_w), None, None, 0.5, K=K, bits_a=8,
+                                                 bits_w=aqt.BITS_4_UNPACKED, bits_out=8)
+    assert aqt.aqt_device_status() == 0 and y_none is None
+    rows = sorted(set([0, 127, 128, 255, 256, 511, M - 257, M - 129, M - 1]) | set(rng.integers(0, M, 30).tolist()))
+    acc_ref = orc.int_matmul(xq[rows], wq)
+    y_ref = orc.epilogue_f32(acc_ref, s_x[rows], aqt.SCALE_ROW, s_w, None, res[rows], 0.5, aqt.ACT_NONE)
+    assert np.array_equal(y_d[rows].cpu().numpy().view(np.uint32), y_ref.view(np.uint32))
+    q_ref, s_ref = orc.quantize(y_ref, 8, orc.AXIS_ROW)
+    assert np.array_equal(q_d[rows].cpu().numpy(), q_ref) and np.array_equal(s_d[rows].cpu().numpy(), s_ref.reshape(-1))
+    # without residual and fp32 output
+    u_ref = orc.epilogue_f32(acc_ref, s_x[rows], aqt.SCALE_ROW, s_w, None, None, 0.0, aqt.ACT_NONE)
+    q_ref2, s_ref2 = orc.quantize(u_ref, 8, orc.AXIS_ROW)
+    assert np.array_equal(q2_d[rows].cpu().numpy(), q_ref2) and np.array_equal(s2_d[rows].cpu().numpy(), s_ref2.reshape(-1))
+    assert int(q_d.abs().max(dim=1).values.min()) == 127 and int(q2_d.abs().max(dim=1).values.min()) == 127
+    # the GPU row quantizer on the fp32 output gives the same codes everywhere
+    q3, s3 = aqt.aqt_quantize(y_d, 8, aqt.AXIS_ROW)
+    assert torch.equal(q3, q_d) and torch.equal(s3.view(torch.int32), s_d.view(torch.int32))
