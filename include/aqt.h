@@ -68,6 +68,12 @@ extern "C" {
                                   aqt_unpack_int4 produce.  Same layout as 8-bit codes; the smaller range lets the
                                   epilogue convert accumulators on the plain ALUs up to a deeper K. */
 
+#define AQT_STATIC_WEIGHTS 0x100 /* may be OR-ed into bits_w of the matmul entry points: the weight codes, their scales and
+                                    the bias were complete before the work that precedes this call on the stream was enqueued
+                                    (weights of a trained model, as opposed to weights re-quantized by the preceding call).
+                                    The kernels then fetch their weights while the preceding kernel is still draining;
+                                    everything else they touch still waits for it. */
+
 /* operations for aqt_workspace_bytes */
 #define AQT_OP_QMATMUL 1
 #define AQT_OP_LINEAR_FWD 2

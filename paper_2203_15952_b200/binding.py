@@ -23,6 +23,7 @@ ACT_NONE, ACT_SWISH, ACT_GLU, ACT_GLU_SWISH = 0, 1, 2, 3
 OP_QMATMUL, OP_LINEAR_FWD, OP_QMATMUL_REQUANT, OP_LINEAR_WEIGHT_ONLY, OP_LINEAR_WEIGHT_ONLY_X2, OP_LINEAR_BWD, OP_FFN_FWD = 1, 2, 3, 4, 5, 6, 7
 FLOAT_TF32, FLOAT_TF32X2 = 0, 1
 BITS_4_UNPACKED = 48  # 4-bit codes, one per int8 container
+STATIC_WEIGHTS = 0x100  # OR into bits_w: the weights were complete before the preceding work on the stream was enqueued
 
 EXPORTS = ("aqt_version", "aqt_status_string", "aqt_quantize", "aqt_pack_int4", "aqt_unpack_int4", "aqt_qmatmul",
            "aqt_linear_fwd", "aqt_linear_fwd_host", "aqt_workspace_bytes", "aqt_device_status", "aqt_qmatmul_w4_noalloc",

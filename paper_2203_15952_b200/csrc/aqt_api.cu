@@ -296,6 +296,7 @@ static int qmatmul_entry(const void* xq, const float* s_x, int s_x_kind, const v
                          const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K, int bits_a,
                          int bits_w, int act, float* y, int64_t ldy, int32_t* acc_debug, void* workspace, size_t workspace_bytes,
                          void* stream, int forced_plan) {
+  bits_w &= ~AQT_STATIC_WEIGHTS;
   int rc = validate_matmul_shape(M, N, K, bits_a, bits_w, act, s_x_kind);
   if (rc != AQT_OK) return rc;
   if (M == 0 || N == 0) return AQT_OK;
@@ -369,6 +370,8 @@ int aqt_qmatmul_requant(const void* xq, const float* s_x, int s_x_kind, const vo
                         const float* residual, int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K, int bits_a,
                         int bits_w, int act, int bits_out, int rounding, int pack_out, void* q_out, float* s_out, float* y,
                         int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+  const int static_w = (bits_w & AQT_STATIC_WEIGHTS) ? 1 : 0;
+  bits_w &= ~AQT_STATIC_WEIGHTS;
   int rc = validate_matmul_shape(M, N, K, bits_a, bits_w, act, s_x_kind);
   if (rc != AQT_OK) return rc;
   if (!quant_bits_ok(bits_out) || (pack_out != 0 && pack_out != 1) || (pack_out == 1 && bits_out != 4)) return AQT_ERR_BADARG;
@@ -480,6 +483,7 @@ int aqt_qmatmul_requant(const void* xq, const float* s_x, int s_x_kind, const vo
   p.n_out = (int)n_out;
   p.tiles_m = p.tiles_n = p.k_blocks = 0;
   p.small_acc = (K * (int64_t)(qmax_of(code_bits(bits_a)) + 1) * (qmax_of(code_bits(bits_w)) + 1) <= (1ll << 22)) ? 1 : 0;
+  p.static_w = (static_w && (!is_packed(bits_w) || b_packed)) ? 1 : 0;  // not for weights unpacked into the workspace just now
   rp.q_out = nullptr;
   rp.s_out = s_out;
   rp.exchange = nullptr;
@@ -493,6 +497,7 @@ int aqt_linear_fwd(const float* x, int64_t ldx, const void* wq, const float* s_w
                    int64_t ldr, float residual_scale, int64_t M, int64_t N, int64_t K, int bits_a, int bits_w,
                    int a_scale_kind, int rounding, int act, float* y, int64_t ldy, void* workspace, size_t workspace_bytes,
                    void* stream) {
+  bits_w &= ~AQT_STATIC_WEIGHTS;
   int rc = validate_matmul_shape(M, N, K, bits_a, bits_w, act, a_scale_kind);
   if (rc != AQT_OK) return rc;
   if (rounding != AQT_ROUND_HALF_UP_FLOOR && rounding != AQT_ROUND_NEAREST_EVEN) return AQT_ERR_BADARG;
@@ -559,6 +564,9 @@ int aqt_ffn_fwd(const float* x, int x_on_host, const void* w1q, const float* s_w
                 const void* w2q, const float* s_w2, const float* bias2, int bits_w2, int64_t M, int64_t d, int64_t ff,
                 int bits_a, int rounding, int act, float* y, int y_on_host, void* workspace, size_t workspace_bytes,
                 void* stream) {
+  const int static_flag = (bits_w1 | bits_w2) & AQT_STATIC_WEIGHTS;
+  bits_w1 &= ~AQT_STATIC_WEIGHTS;
+  bits_w2 &= ~AQT_STATIC_WEIGHTS;
   if (M < 0 || d <= 0 || ff <= 0 || !quant_bits_ok(bits_a) || !bits_ok(bits_w1) || !bits_ok(bits_w2)) return AQT_ERR_BADARG;
   if (act != AQT_ACT_NONE && act != AQT_ACT_SWISH) return AQT_ERR_BADARG;
   if (rounding != AQT_ROUND_HALF_UP_FLOOR && rounding != AQT_ROUND_NEAREST_EVEN) return AQT_ERR_BADARG;
@@ -589,7 +597,7 @@ int aqt_ffn_fwd(const float* x, int x_on_host, const void* w1q, const float* s_w
   rc = aqt_quantize(x_dev, M, d, d, bits_a, AQT_AXIS_ROW, rounding, 0, q1, s1, stream);
   if (rc != AQT_OK) return rc;
   const int bits_mm = bits_a == 8 ? 8 : AQT_BITS_4_UNPACKED;
-  rc = aqt_qmatmul_requant(q1, s1, AQT_SCALE_ROW, w1q, s_w1, bias1, nullptr, 0, 0.0f, M, ff, d, bits_mm, bits_w1, act, bits_a, rounding, 0,
+  rc = aqt_qmatmul_requant(q1, s1, AQT_SCALE_ROW, w1q, s_w1, bias1, nullptr, 0, 0.0f, M, ff, d, bits_mm, bits_w1 | static_flag, act, bits_a, rounding, 0,
                            q2, s2, nullptr, 0, ws + L.mm, mm_bytes, stream);
   if (rc != AQT_OK) return rc;
   rc = aqt_qmatmul(q2, s2, AQT_SCALE_ROW, w2q, s_w2, bias2, nullptr, 0, 0.0f, M, d, ff, bits_mm, bits_w2, AQT_ACT_NONE, y_dev, d, nullptr,

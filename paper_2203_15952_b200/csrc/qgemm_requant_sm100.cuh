@@ -210,12 +210,13 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     tmem_alloc(smem_u32(&tmem_base_slot), Cfg::kTmemCols);
     tmem_relinquish();
   }
-  // everything above touched only this CTA's own state; from here on global memory is read
-  grid_dependency_wait();
-  // Tag of this execution's exchange words.  A replayed CUDA graph repeats the call's own tag, so the
-  // group's generation counter goes into it: every CTA of the group reads it here, and the group's
-  // first CTA bumps it after its last tile, which it cannot finish before all of them have started.
-  const uint32_t tag = mix_tag(rp.tag, __ldcg(rp.generation + group));
+  // Everything above touched only this CTA's own state; from here on global memory is read.  The
+  // weights (codes, scales, bias) may be read before the kernel ahead of this one in the stream has
+  // finished if the caller says they were complete before that kernel was enqueued (static_w): the
+  // weight slab then loads and unpacks while that kernel drains, and every role waits for it only
+  // before its first access to anything else.
+  const bool early_w = p.static_w != 0;
+  if (!early_w) grid_dependency_wait();
   for (int t = threadIdx.x; t < BN; t += blockDim.x) {
     // scales and biases of the tile's weight rows: (GLU) values first, then gates
     const int n = !GLU ? tn * BN + t : (t < HALF ? tn * HALF + t : p.N / 2 + tn * HALF + (t - HALF));
@@ -255,6 +256,7 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
           }
         }
       }
+      if (early_w) grid_dependency_wait();  // the activation codes come from the kernel ahead
       for (int i = 0; ok && i < n_my; ++i) {
         const int tm = group + i * groups;
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
@@ -297,6 +299,11 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     // 64h + 2l + 1, i.e. one 16-byte load (two words) per n-tile, kExchangeBatch of them in flight.
     const int xh = warp - (2 + EW);
     bool ok = true;
+    if (early_w) grid_dependency_wait();
+    // Tag of this execution's exchange words.  A replayed CUDA graph repeats the call's own tag, so the
+    // group's generation counter goes into it: every CTA of the group reads it at its start, and the
+    // group's first CTA bumps it after its last tile, which it cannot finish before all of them have started.
+    const uint32_t tag = mix_tag(rp.tag, __ldcg(rp.generation + group));
     for (int i = 0; ok && i < n_my; ++i) {
       const int tm = group + i * groups;
       const uint32_t par = i % kSlots, ph = (i / kSlots) & 1;
@@ -385,6 +392,8 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       }
     }
 
+    if (early_w) grid_dependency_wait();  // scales of the activations, residual, outputs: everything but the weights
+    const uint32_t tag = mix_tag(rp.tag, __ldcg(rp.generation + group));  // see the exchange warps
     uint32_t res_count = 0;  // residual boxes this warp has consumed (phase of its barrier)
     if (ok && has_res && lane == 0 && set < n_my) {
       const int r0 = (group + set * groups) * kBM + quad * 32;

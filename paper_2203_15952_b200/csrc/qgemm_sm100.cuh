@@ -117,6 +117,9 @@ struct GemmParams {
   int qmax_out = 127;
   int rounding = AQT_ROUND_NEAREST_EVEN;
   int has_y = 1;                    // 0: no fp32 output
+  // The weights (codes, scales, bias) were complete before the kernel ahead of this one in the stream
+  // was enqueued, so a kernel may read them before that kernel has finished (see grid_dependency_wait).
+  int static_w = 0;
 };
 
 // ------------------------------------------------------------------------------------------------

@@ -102,3 +102,33 @@ def test_argument_errors_of_the_float_entry_points_need_no_device():
     assert L.aqt_workspace_bytes(4, i64(128), i64(256), i64(128), 0, 4) == 4 * 256 * 128
     assert L.aqt_workspace_bytes(5, i64(128), i64(256), i64(128), 0, 4) == 8 * 256 * 128 + 8 * 128 * 128
     assert L.aqt_workspace_bytes(6, i64(12800), i64(2048), i64(512), 0, 0) > 4 * (512 * 2048 + (2048 + 512) * 12800)
+
+
+def test_plan_query_and_new_entry_points_reject_bad_arguments():
+    """The plan query is host-only; the entry points added beside the named calls validate like them."""
+    import ctypes
+    from paper_2203_15952_b200 import binding as b
+    L = ctypes.CDLL(aqt_build.build())
+    i64, vp = ctypes.c_int64, ctypes.c_void_p
+    one = vp(256)
+    buf = ctypes.create_string_buffer(64)
+    assert L.aqt_plan_qmatmul(i64(1000), i64(512), i64(512), 8, 4, 0, 0, 148, buf, ctypes.c_size_t(64)) == 0 and buf.value == b"ws128e16"
+    assert L.aqt_plan_qmatmul(i64(1000), i64(512), i64(512), 8, 4, 0, 0, 148, buf, ctypes.c_size_t(4)) == -1      # name does not fit
+    assert L.aqt_plan_qmatmul(i64(0), i64(512), i64(512), 8, 4, 0, 0, 148, buf, ctypes.c_size_t(64)) == -1
+    assert L.aqt_plan_qmatmul(i64(8), i64(512), i64(512), 8, 5, 0, 0, 148, buf, ctypes.c_size_t(64)) == -1         # unknown width
+    assert b.aqt_plan_qmatmul(8, 512, 512, 8, b.BITS_4_UNPACKED) == "small_m"
+    # a named plan that does not exist; the 4-bit-in-container width and the static-weights flag pass validation
+    f = ctypes.c_float(1.0)
+    args = (one, one, 0, one, one, None, None, i64(0), f, i64(256), i64(256), i64(256), 8, b.BITS_4_UNPACKED | b.STATIC_WEIGHTS, 0, one,
+            i64(256), None, None, ctypes.c_size_t(0), None)
+    assert L.aqt_qmatmul_with_plan(ctypes.c_char_p(b"no_such_plan"), *args) == -1
+    bad = list(args); bad[13] = 5
+    assert L.aqt_qmatmul(*bad) == -1
+    # aqt_ffn_fwd: activation other than none / Swish, missing workspace
+    ffn = lambda act, ws, wsb: L.aqt_ffn_fwd(one, 0, one, one, None, 4, one, one, None, 4, i64(256), i64(512), i64(2048), 8, 1, act, one, 0,
+                                             ws, ctypes.c_size_t(wsb), None)
+    assert ffn(2, one, 1 << 30) == -1
+    assert ffn(1, None, 0) == -4
+    assert b.aqt_workspace_bytes(b.OP_FFN_FWD, 256, 2048, 512, 8, 4) > 2 * 4 * 256 * 512 + 256 * 2048
+    ops = ctypes.c_int64(0)
+    assert L.aqt_selftest_sfu_rate(0, one, ctypes.byref(ops), None) == -1

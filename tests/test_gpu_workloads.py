@@ -245,3 +245,40 @@ def test_cfg5_heavy_tailed_rows_of_the_large_encoder():
     q_ref, s_ref = orc.quantize(x[rows], 8, orc.AXIS_ROW)
     assert np.array_equal(q.cpu().numpy()[rows], q_ref) and np.array_equal(s.cpu().numpy()[rows], s_ref)
     assert float((q.abs() <= 16).float().mean()) > 0.5
+
+
+def test_ffn_fwd_entry_point_host_and_device_buffers():
+    """aqt_ffn_fwd (quantize -> matmul that quantizes its rows -> matmul, one call) gives the bits of
+    the three calls made one by one, with device buffers, with pinned host buffers, and with the
+    weights declared static (fetched before the preceding kernel has finished)."""
+    w = gen.WORKLOADS[2]
+    specs = gen.workload_layers(w)
+    M = 3000
+    gpu, cpu = _layers(w, 0, specs)
+    x = gen.workload_input(w, row_subset=range(M))
+    xd = _dev(x)
+    q1, s1 = aqt.aqt_quantize(xd, 8, aqt.AXIS_ROW)
+    u = aqt.aqt_qmatmul(q1, s1, gpu[0].wq, gpu[0].s_w, K=specs[0].K, bits_w=4, act=specs[0].act)
+    q2, s2 = aqt.aqt_quantize(u, 8, aqt.AXIS_ROW)
+    y_ref = aqt.aqt_qmatmul(q2, s2, gpu[1].wq, gpu[1].s_w, K=specs[1].K, bits_w=4)
+    for static in (0, aqt.STATIC_WEIGHTS):
+        y = torch.full_like(y_ref, float("nan"))
+        aqt.aqt_ffn_fwd(xd, gpu[0].wq, gpu[0].s_w, 4 | static, gpu[1].mm_weight, gpu[1].s_w, gpu[1].mm_bits | static, y)
+        assert aqt.aqt_device_status() == 0
+        assert torch.equal(y.view(torch.int32), y_ref.view(torch.int32))
+    xh = torch.from_numpy(x).pin_memory()
+    yh = torch.full((M, w.d), float("nan"), dtype=torch.float32).pin_memory()
+    aqt.aqt_ffn_fwd(xh, gpu[0].wq, gpu[0].s_w, 4, gpu[1].wq, gpu[1].s_w, 4, yh)
+    assert aqt.aqt_device_status() == 0
+    assert np.array_equal(yh.numpy().view(np.uint32), y_ref.cpu().numpy().view(np.uint32))
+    # and against the oracle: the second layer is IEEE operations only, fed the GPU's own u
+    rows = _sample_rows(M, n=16)
+    _check_layer(specs[0], cpu[0], x[rows], u.cpu().numpy()[rows])
+    _check_layer(specs[1], cpu[1], u.cpu().numpy()[rows], yh.numpy()[rows])
+
+
+def test_special_function_rate_measurement():
+    """The measurement aid reports a rate of the order of 16 operations per clock and SM."""
+    rate = aqt.aqt_selftest_sfu_rate(iterations=2048)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert 0.3 * 16 * sms * 1.0 < rate < 1.3 * 16 * sms * 2.2      # Gop/s at 1.0 .. 2.2 GHz
