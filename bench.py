@@ -792,6 +792,12 @@ def run_case(args):
         x, wq, s_w = torch.randn((M, K), generator=g, device=dev), torch.randint(0, 256, (N, K // 2), generator=g, dtype=torch.uint8, device=dev), scales(N, 1e-3)
         for i in range(it):
             aqt.aqt_linear_fwd_weight_only(x, wq, s_w, bits_w=4, act=aqt.ACT_SWISH)
+    elif name == "bwd_ffn1":
+        M, N, K = 12800, 2048, 512
+        dy, xq, wq = torch.randn((M, N), generator=g, device=dev), codes(M, K, 127), torch.randint(0, 256, (N, K // 2), generator=g, dtype=torch.uint8, device=dev)
+        s_x, s_w = scales(M, 1e-2), scales(N, 1e-3)
+        for i in range(it):
+            aqt.aqt_linear_bwd(dy, xq, s_x, wq, s_w, K=K, bits_a=8, bits_w=4)
     else:
         raise SystemExit("unknown case " + name)
     torch.cuda.synchronize()
@@ -812,7 +818,7 @@ def main():
     ap.add_argument("--no-sustained", action="store_true", help="skip the half-second sustained run of the headline step")
     ap.add_argument("--no-graph", action="store_true", help="launch every step call by call (no CUDA graph replay)")
     ap.add_argument("--case", default=None, help="run one library call a few times and exit (for profiler captures): quantize_ffn, "
-                    "quantize_large, requant_ffn1, requant_large, gemm_ffn2, gemm_large_ffn2, gemm_large_ffn1, weight_only_ffn1")
+                    "quantize_large, requant_ffn1, requant_large, gemm_ffn2, gemm_large_ffn2, gemm_large_ffn1, weight_only_ffn1, bwd_ffn1")
     ap.add_argument("--iters", type=int, default=4, help="--case: number of calls")
     args = ap.parse_args()
     if args.case is not None:
