@@ -302,7 +302,7 @@ int aqt_linear_fwd_weight_only(const float* x, int64_t ldx, const void* wq, cons
  *           aligned: the transposed, scaled operands (4 * (K * N + (N + K) * M) bytes and change)
  *           and, where the weight gradient's contraction is split over CTAs, the partial products.
  * Limits: K % 4 == 0, N % 4 == 0; lddy, lddx, lddw multiples of 4; dy, dx, dw, xq, wq 16-byte aligned;
- * M, N, K < 2^28.  M == 0 or N == 0 is a no-op.
+ * M, N < 2^23, K < 2^28 (larger sizes return AQT_ERR_UNSUPPORTED before anything is enqueued).  M == 0 or N == 0 is a no-op.
  */
 int aqt_linear_bwd(const float* dy, int64_t lddy, const void* xq, const float* s_x, int s_x_kind, int bits_a,
                    const void* wq, const float* s_w, int bits_w, int64_t M, int64_t N, int64_t K, float* dx,

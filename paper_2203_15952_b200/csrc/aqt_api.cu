@@ -114,7 +114,9 @@ int float_gemm_nt(const float* a, int64_t lda, const float* b, int64_t rows, int
 // True if the CTA-pair kernel with the row-quantizing epilogue takes the call: deep K, no GLU, int8
 // codes out (4-bit codes stay in their containers), at most 16 column parts per row.
 bool rowquant_pair_applies(int64_t M, int64_t N, int64_t K, int act, bool pack_out) {
-  if (pack_out || M <= kBM || K < 1024) return false;
+  // (from K = 2048: at K = 1024 a tile's MMAs are shorter than its two epilogue passes, and the
+  // two kernels are faster: 162 vs 209 us at 65 536 x 1024 -> 1024 with the fp32 output)
+  if (pack_out || M <= kBM || K < 2048) return false;
   if (act != AQT_ACT_NONE && act != AQT_ACT_SWISH) return false;
   const int sms = sm_count() > 0 ? sm_count() : kDefaultSms;
   const int plan = rowquant_plan(M, N, K, sms);
@@ -675,7 +677,8 @@ int aqt_linear_bwd(const float* dy, int64_t lddy, const void* xq, const float* s
   if (M < 0 || N < 0 || K <= 0 || !bits_ok(bits_a) || !bits_ok(bits_w)) return AQT_ERR_BADARG;
   if (s_x_kind != AQT_SCALE_ROW && s_x_kind != AQT_SCALE_TENSOR) return AQT_ERR_BADARG;
   if (K % 4 != 0 || N % 4 != 0) return AQT_ERR_BADARG;
-  if (M >= (1ll << 28) || N >= (1ll << 28) || K >= (1ll << 28) || M * N >= (1ll << 40)) return AQT_ERR_UNSUPPORTED;
+  // M and N are row counts of the transposing prepasses, whose 128-row blocks are a grid's y extent (at most 65 535)
+  if (M >= (1ll << 23) || N >= (1ll << 23) || K >= (1ll << 28) || M * N >= (1ll << 40)) return AQT_ERR_UNSUPPORTED;
   if (M == 0 || N == 0) return AQT_OK;
   if (dy == nullptr || lddy < N) return AQT_ERR_BADARG;
   if (dx != nullptr && (wq == nullptr || s_w == nullptr || lddx < K)) return AQT_ERR_BADARG;

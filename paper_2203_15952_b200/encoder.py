@@ -107,15 +107,16 @@ class LayerRunner:
 
     def fuses_requant(self, layer: QuantLinear, with_y: bool = True) -> bool:
         """True if `layer`'s matmul can quantize its own output rows in its epilogue (the GLU
-        forms only when the fp32 output is not wanted as well)."""
+        forms and 512 < K <= 1024 only when the fp32 output is not wanted as well; 1024 < K < 2048
+        not at all)."""
         s = layer.spec
         ok = self.a_scale_kind == aqt.SCALE_ROW and s.K % 16 == 0 and s.n_out % 32 == 0 and s.N <= 128 * 148
         glu = s.act in (aqt.ACT_GLU, aqt.ACT_GLU_SWISH)
-        if s.K > 1024 or (s.K > 512 and with_y):
+        if s.K >= 2048:
             # deep K: the CTA-pair kernel quantizes its rows (no GLU; at most 16 column parts per row)
             return ok and not glu and self.M > 128 and s.N <= 2048
         if glu or s.K > 512:
-            return ok and not with_y
+            return ok and not with_y and s.K <= 1024
         return ok
 
     def code_buffers(self, role: str, cols: int):

@@ -154,6 +154,16 @@ def test_requant_glu_forms(act, M, N, K, bits_w):
         assert np.array_equal(q_d.cpu().numpy(), q_ref), "fused codes differ: %d" % (q_d.cpu().numpy() != q_ref).sum()
 
 
+@pytest.mark.parametrize("M,N,K,act", [(300, 1024, 1024, aqt.ACT_NONE), (1500, 1024, 1024, aqt.ACT_SWISH), (129, 1040, 640, aqt.ACT_NONE),
+                                       (2000, 2064, 896, aqt.ACT_NONE)])
+def test_requant_deep_k_with_residual_stream(M, N, K, act):
+    """The d = 1024 encoder's attention output and second pointwise layers: 512 < K <= 1024 with
+    residual and fp32 output next to the codes (matmul, then the row quantizer, inside the one
+    call); N with a ragged last tile."""
+    _run(M, N, K, 8, 4, act, True, True, 8, aqt.ROUND_NEAREST_EVEN, False)
+    _run(M, N, K, 8, 8, act, False, True, 4, aqt.ROUND_NEAREST_EVEN, N % 32 == 0)
+
+
 def test_requant_unfused_shapes_go_through_y():
     """K > 1024 (and K > 512 or the GLU forms with an fp32 output) are not taken by the fused
     kernel: the call runs the two steps through y."""
