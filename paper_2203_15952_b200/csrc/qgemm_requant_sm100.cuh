@@ -161,8 +161,8 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
   __shared__ uint64_t b_loaded_bar;
   __shared__ uint64_t b_ready_bar;
   __shared__ __align__(16) uint32_t row_amax[kSlots][kBM];  // final row maxima (bit patterns) of a tile awaiting pass 2
-  __shared__ uint64_t ctx_ready_bar[kSlots];  // the exchange warp has filled row_amax[.]
-  __shared__ uint64_t ctx_free_bar[kSlots];   // the set's four warps have read their rows of row_amax[.]
+  __shared__ uint64_t ctx_ready_bar[kSlots][2];  // an exchange warp has filled its half of row_amax[.]
+  __shared__ uint64_t ctx_free_bar[kSlots][2];   // the set's two warps on that half of the rows have read theirs
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
@@ -200,8 +200,10 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     mbar_init(smem_u32(&b_loaded_bar), 1);
     mbar_init(smem_u32(&b_ready_bar), EW);
     for (int b = 0; b < kSlots; ++b) {
-      mbar_init(smem_u32(&ctx_ready_bar[b]), 2);  // both exchange warps
-      mbar_init(smem_u32(&ctx_free_bar[b]), 4);
+      for (int h = 0; h < 2; ++h) {
+        mbar_init(smem_u32(&ctx_ready_bar[b][h]), 1);
+        mbar_init(smem_u32(&ctx_free_bar[b][h]), 2);
+      }
     }
     fence_barrier_init();
     fence_proxy_async_smem();
@@ -307,7 +309,7 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     for (int i = 0; ok && i < n_my; ++i) {
       const int tm = group + i * groups;
       const uint32_t par = i % kSlots, ph = (i / kSlots) & 1;
-      if (!mbar_wait(smem_u32(&ctx_free_bar[par]), ph ^ 1, &abort_flag, t_start)) break;
+      if (!mbar_wait(smem_u32(&ctx_free_bar[par][xh]), ph ^ 1, &abort_flag, t_start)) break;
       const uint64_t* xt = rp.exchange + (size_t)tm * p.tiles_n * kBM + 64 * xh + 2 * lane;
       uint2 m2 = make_uint2(0u, 0u);
       for (int t0 = 0; ok && t0 < p.tiles_n; t0 += kExchangeBatch) {
@@ -339,7 +341,7 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       // final maxima of this warp's rows for the epilogue warps
       *reinterpret_cast<uint2*>(&row_amax[par][64 * xh + 2 * lane]) = m2;
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&ctx_ready_bar[par]));
+      if (lane == 0) mbar_arrive(smem_u32(&ctx_ready_bar[par][xh]));
     }
   } else {
     // ------------------------------------------------------------------ epilogue warps
@@ -508,10 +510,10 @@ qgemm_requant_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       st_relaxed_gpu_64(rp.exchange + ((size_t)tm * p.tiles_n + tn) * kBM + row_in_tile, ((uint64_t)tag << 32) | __float_as_uint(amax));
 
       // -------------------------------------------------------------- pass 2: scale, codes
-      if (!mbar_wait(smem_u32(&ctx_ready_bar[set]), aph, &abort_flag, t_start)) { ok = false; break; }
+      if (!mbar_wait(smem_u32(&ctx_ready_bar[set][quad >> 1]), aph, &abort_flag, t_start)) { ok = false; break; }
       const float amax_row = __uint_as_float(row_amax[set][row_in_tile]);
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&ctx_free_bar[set]));
+      if (lane == 0) mbar_arrive(smem_u32(&ctx_free_bar[set][quad >> 1]));
       const ScaleCtx sc = make_scale_ctx(amax_row, rp.qmax_out);
       if (tn == 0 && m < p.M) rp.s_out[m] = sc.s;
       tmem_st_wait();  // this warp's stores of pass 1
