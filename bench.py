@@ -30,10 +30,11 @@ sys.path.insert(0, ROOT)
 METRIC = "quantized Conformer linear TOPS (int4 weights, int8 activations)"
 UNIT = "TOPS"
 CFG = 2  # the Conformer FFN pair; fits one GPU many times over
-NCU_CAPTURE_VERSION = 200  # library version the ncu traffic figures below were captured at
+NCU_CAPTURE_VERSION = 201  # library version the ncu traffic figures below were captured at
 # call index -> DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the
-# ncu summaries under profiles/; empty until a capture of this library version is committed
-NCU_TRAFFIC = {}
+# ncu summaries under profiles/ (qgemm_requant_ffn1_ncu.md, qgemm_i8_ffn2_ncu.md); the quantizer of the
+# 12 800 x 512 input has no capture of its own (its 33 MB stay inside L2 under the profiler)
+NCU_TRAFFIC = {1: 7704320 + 2560, 2: 27355904 + 73984}
 INT8_NOMINAL_TOPS = 4500.0  # dense int8 tensor peak of the part, nominal
 
 

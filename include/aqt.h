@@ -32,7 +32,7 @@
 extern "C" {
 #endif
 
-#define AQT_VERSION 200
+#define AQT_VERSION 201
 
 /* status codes */
 #define AQT_OK 0
