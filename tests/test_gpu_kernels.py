@@ -210,6 +210,32 @@ def test_linear_fwd_conformer_s_width():
     assert np.array_equal(y.cpu().numpy().view(np.uint32), y_ref.view(np.uint32))
 
 
+def _random_matmul_case(seed, row_quantizing=False):
+    """A seeded random shape and operand mix inside the documented limits (K a multiple of 16, N a
+    multiple of 16 or, for the GLU forms, 32), small enough for the oracle: M N K <= 3e8."""
+    rng = np.random.default_rng(900 + seed)
+    act = [aqt.ACT_NONE, aqt.ACT_SWISH, aqt.ACT_GLU, aqt.ACT_GLU_SWISH][int(rng.integers(0, 4))]
+    K = int(rng.choice([16, 48, 96, 128, 144, 256, 384, 512, 640, 768, 1024, 1536, 2048, 4096]))
+    n_step = 64 if act in (aqt.ACT_GLU, aqt.ACT_GLU_SWISH) else 32
+    N = n_step * int(rng.integers(1, 2304 // n_step + 1))
+    M = int(rng.integers(1, 2600))
+    while M * N * K > 3e8:
+        if N > 4 * n_step:
+            N = n_step * max(1, (N // n_step) // 2)
+        else:
+            M = max(1, M // 2)
+    bits_a, bits_w = [(8, 8), (8, 4), (4, 4), (4, 8)][int(rng.integers(0, 4))]
+    return M, N, K, bits_a, bits_w, act, bool(rng.integers(0, 2)), bool(rng.integers(0, 2))
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_qmatmul_random_shapes(seed):
+    """Shapes nobody picked by hand: whatever kernel configuration the library chooses for them
+    must give the oracle's accumulators and outputs."""
+    M, N, K, bits_a, bits_w, act, with_bias, with_res = _random_matmul_case(seed)
+    _run_qmatmul(M, N, K, bits_a, bits_w, act, with_bias, with_res, seed=seed)
+
+
 def test_qmatmul_per_tensor_scale_and_deep_k():
     _run_qmatmul(256, 256, 4096, 8, 8, aqt.ACT_NONE, True, False, s_x_kind=aqt.SCALE_TENSOR, extremes=True)
 

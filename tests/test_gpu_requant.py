@@ -20,7 +20,8 @@ def _codes(rng, rows, K, bits):
     return rng.integers(-qm, qm + 1, (rows, K)).astype(np.int8)
 
 
-def _run(M, N, K, bits_a, bits_w, act, with_bias, with_res, bits_out, rounding, pack_out, special_rows=False):
+def _run(M, N, K, bits_a, bits_w, act, with_bias, with_res, bits_out, rounding, pack_out, special_rows=False,
+         may_refuse_without_y=False):
     rng = np.random.default_rng(7 + 1000 * M + N + K + bits_out)
     xq = _codes(rng, M, K, bits_a)
     wq = _codes(rng, N, K, bits_w)
@@ -77,7 +78,12 @@ def _run(M, N, K, bits_a, bits_w, act, with_bias, with_res, bits_out, rounding, 
     if res is None:
         q2_d = torch.full(q_shape, 0x55, dtype=q_d.dtype, device=DEV)
         s2_d = torch.full((M,), float("nan"), dtype=torch.float32, device=DEV)
-        _, _, y_none = aqt.aqt_qmatmul_requant(*args, **kw, q_out=q2_d, s_out=s2_d)
+        try:
+            _, _, y_none = aqt.aqt_qmatmul_requant(*args, **kw, q_out=q2_d, s_out=s2_d)
+        except aqt.AqtError as e:
+            # shapes no fused kernel takes need the fp32 output as the hand-over between the two steps
+            assert may_refuse_without_y and e.status == -3
+            return
         assert y_none is None
         assert aqt.aqt_device_status() == 0
         assert torch.equal(q2_d, q_d) and torch.equal(s2_d.view(torch.int32), s_d.view(torch.int32))
@@ -162,6 +168,29 @@ def test_requant_deep_k_with_residual_stream(M, N, K, act):
     call); N with a ragged last tile."""
     _run(M, N, K, 8, 4, act, True, True, 8, aqt.ROUND_NEAREST_EVEN, False)
     _run(M, N, K, 8, 8, act, False, True, 4, aqt.ROUND_NEAREST_EVEN, N % 32 == 0)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_requant_random_shapes(seed):
+    """Seeded random shapes inside the limits of the call (K a multiple of 16, output width a
+    multiple of 32): every form it dispatches to (fused K <= 512, eight-k-block, CTA pairs from
+    K = 2048, matmul + quantizer in between) against the oracle."""
+    rng = np.random.default_rng(400 + seed)
+    K = int(rng.choice([16, 64, 144, 256, 512, 640, 1024, 1536, 2048, 4096]))
+    N = 32 * int(rng.integers(1, 65))
+    M = int(rng.integers(1, 3000))
+    while M * N * K > 3e8:
+        if N > 128:
+            N = 32 * max(1, (N // 32) // 2)
+        else:
+            M = max(1, M // 2)
+    bits_a, bits_w = [(8, 8), (8, 4), (4, 4), (4, 8)][int(rng.integers(0, 4))]
+    act = [aqt.ACT_NONE, aqt.ACT_SWISH][int(rng.integers(0, 2))]
+    bits_out = [8, 4][int(rng.integers(0, 2))]
+    pack_out = bits_out == 4 and bool(rng.integers(0, 2))
+    rounding = [aqt.ROUND_NEAREST_EVEN, aqt.ROUND_HALF_UP_FLOOR][int(rng.integers(0, 2))]
+    _run(M, N, K, bits_a, bits_w, act, bool(rng.integers(0, 2)), bool(rng.integers(0, 2)), bits_out, rounding, pack_out,
+         may_refuse_without_y=K > 1024)
 
 
 def test_requant_unfused_shapes_go_through_y():
