@@ -366,6 +366,33 @@ def test_linear_fwd_matches_oracle(bits_a, bits_w, kind, rounding):
     assert np.array_equal(y.cpu().numpy().view(np.uint32), y_ref.view(np.uint32))
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_linear_fwd_random_shapes(seed):
+    """The whole layer (fp32 in, fp32 out, act = NONE so every output bit is fixed) on seeded
+    random shapes, scale kinds, bit widths and rounding rules, weights prepared on the GPU."""
+    rng = np.random.default_rng(1300 + seed)
+    K = 16 * int(rng.integers(1, 129))
+    N = 16 * int(rng.integers(1, 97))
+    M = int(rng.integers(1, 1500))
+    while M * N * K > 2e8:
+        M = max(1, M // 2)
+    bits_a, bits_w = [(8, 8), (8, 4), (4, 4), (4, 8)][int(rng.integers(0, 4))]
+    kind = [aqt.SCALE_ROW, aqt.SCALE_TENSOR][int(rng.integers(0, 2))]
+    rounding = [orc.ROUND_HALF_UP_FLOOR, orc.ROUND_NEAREST_EVEN][int(rng.integers(0, 2))]
+    x = gen.normal(40 + seed, 1, M, K)
+    wt = gen.weight(40 + seed, 2, K, N)
+    bias = gen.normal(40 + seed, 3, 1, N, std=0.01)[0] if rng.integers(0, 2) else None
+    res = gen.normal(40 + seed, 4, M, N) if rng.integers(0, 2) else None
+    wq, s_w = orc.quantize(wt, bits_w, orc.AXIS_ROW, rounding)
+    y_ref = orc.linear_fwd(x, wq, s_w, bias=bias, residual=res, residual_scale=0.5, bits_a=bits_a, a_scale_kind=kind, rounding=rounding)
+    wq_d, sw_d = aqt.aqt_quantize(_dev(wt), bits_w, aqt.AXIS_ROW, rounding, pack=(bits_w == 4))
+    assert np.array_equal(sw_d.cpu().numpy(), s_w)
+    y = aqt.aqt_linear_fwd(_dev(x), wq_d, sw_d, None if bias is None else _dev(bias), None if res is None else _dev(res), 0.5,
+                           bits_a=bits_a, bits_w=bits_w, a_scale_kind=kind, rounding=rounding)
+    _status_ok()
+    assert np.array_equal(y.cpu().numpy().view(np.uint32), y_ref.view(np.uint32))
+
+
 def test_linear_fwd_host_buffers():
     M, K, N = 256, 256, 256
     x = gen.normal(5, 1, M, K)
