@@ -76,6 +76,59 @@ class QuantLinear:
         return self.wq.numel() + 4 * self.s_w.numel()
 
 
+class WeightArena:
+    """The float weights W^T [N_i, K] of many linears kept in one tensor per (K, bit width), one
+    below the other, so that re-quantizing all of them (every training step when the model is
+    trained quantized from scratch, Section 2.2) is one quantizer call per group instead of one
+    per weight: the quantizer reduces over K row by row (one scale per output channel), so the
+    rows of different weights do not interact and the codes and scales are those of the
+    per-weight calls.  `float_view(i)` is weight i's slice of the arena (the optimizer writes
+    there); `quantize()` fills the code and scale arenas; `linear(i)` wraps weight i's slices."""
+
+    def __init__(self, specs: List[LinearSpec], device):
+        self.specs = list(specs)
+        self.groups: Dict[tuple, List[int]] = {}
+        for i, sp in enumerate(self.specs):
+            self.groups.setdefault((sp.K, sp.bits_w), []).append(i)
+        self.float_arena: Dict[tuple, torch.Tensor] = {}
+        self.code_arena: Dict[tuple, torch.Tensor] = {}
+        self.scale_arena: Dict[tuple, torch.Tensor] = {}
+        self._row0: Dict[int, int] = {}
+        for key, members in self.groups.items():
+            K, bits = key
+            rows = 0
+            for i in members:
+                self._row0[i] = rows
+                rows += self.specs[i].N
+            self.float_arena[key] = torch.empty((rows, K), dtype=torch.float32, device=device)
+            self.code_arena[key] = torch.empty((rows, K // 2 if bits == 4 else K), dtype=torch.uint8 if bits == 4 else torch.int8,
+                                               device=device)
+            self.scale_arena[key] = torch.empty(rows, dtype=torch.float32, device=device)
+
+    def _slice(self, arena: Dict[tuple, torch.Tensor], i: int) -> torch.Tensor:
+        sp = self.specs[i]
+        r0 = self._row0[i]
+        return arena[(sp.K, sp.bits_w)][r0:r0 + sp.N]
+
+    def float_view(self, i: int) -> torch.Tensor:
+        return self._slice(self.float_arena, i)
+
+    def quantize(self, rounding: int = aqt.ROUND_NEAREST_EVEN, stream=None) -> int:
+        """One quantizer call per group; returns the number of calls."""
+        for key, wt in self.float_arena.items():
+            aqt.aqt_quantize(wt, key[1], aqt.AXIS_ROW, rounding, pack=(key[1] == 4), q_out=self.code_arena[key],
+                             scale_out=self.scale_arena[key], stream=stream)
+        return len(self.float_arena)
+
+    def linear(self, i: int, bias: Optional[torch.Tensor] = None) -> "QuantLinear":
+        return QuantLinear(self.specs[i], self._slice(self.code_arena, i), self._slice(self.scale_arena, i), bias).prepare()
+
+    @property
+    def algorithmic_bytes(self) -> int:
+        """fp32 weights read, codes and scales written."""
+        return sum(4 * w.numel() + self.code_arena[k].numel() + 4 * self.scale_arena[k].numel() for k, w in self.float_arena.items())
+
+
 class LayerRunner:
     """Owns the scratch workspace shared by all layers of a workload and runs single layers."""
 

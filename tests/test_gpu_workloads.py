@@ -282,3 +282,27 @@ def test_special_function_rate_measurement():
     rate = aqt.aqt_selftest_sfu_rate(iterations=2048)
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     assert 0.3 * 16 * sms * 1.0 < rate < 1.3 * 16 * sms * 2.2      # Gop/s at 1.0 .. 2.2 GHz
+
+
+def test_weight_arena_quantizes_like_per_weight_calls_and_the_oracle():
+    """All weights of a block in one arena per contraction depth: one quantizer call per arena
+    must give every weight the codes and scales of its own call, which are the oracle's."""
+    from paper_2203_15952_b200.encoder import WeightArena
+    specs = gen.block_linears(128, 512, 4, 8, 8)          # FFN weights 4-bit, attention / pointwise 8-bit; K = 128 and 512
+    arena = WeightArena(specs, DEV)
+    host = []
+    for i, sp in enumerate(specs):
+        wt = gen.weight(77, i, sp.K, sp.N)
+        host.append(wt)
+        arena.float_view(i).copy_(_dev(wt))
+    calls = arena.quantize()
+    assert calls == len({(sp.K, sp.bits_w) for sp in specs}) < len(specs)
+    assert aqt.aqt_device_status() == 0
+    for i, sp in enumerate(specs):
+        lin = arena.linear(i)
+        q_ref, s_ref = orc.quantize(host[i], sp.bits_w, orc.AXIS_ROW)
+        want = orc.pack_int4(q_ref) if sp.bits_w == 4 else q_ref
+        assert np.array_equal(lin.wq.cpu().numpy().view(want.dtype), want), sp.name
+        assert np.array_equal(lin.s_w.cpu().numpy(), s_ref.reshape(-1)), sp.name
+        q_own, s_own = aqt.aqt_quantize(_dev(host[i]), sp.bits_w, aqt.AXIS_ROW, pack=(sp.bits_w == 4))
+        assert torch.equal(q_own.view(torch.uint8), lin.wq.view(torch.uint8)) and torch.equal(s_own, lin.s_w)
