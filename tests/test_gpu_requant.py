@@ -109,6 +109,13 @@ def test_requant_with_residual_stream(M, N, K, act):
     _run(M, N, K, 8, 4, act, True, True, 8, aqt.ROUND_NEAREST_EVEN, False)
 
 
+def test_requant_with_residual_stream_many_tiles_per_cta():
+    """Six tiles per CTA with residual and fp32 output: the sets overlap, so chunks of the residual
+    of several tiles are wanted at the same time while the residual ring holds two."""
+    _run(6000, 2048, 128, 8, 4, aqt.ACT_SWISH, True, True, 8, aqt.ROUND_NEAREST_EVEN, False)
+    _run(5000, 512, 256, 8, 8, aqt.ACT_NONE, False, True, 4, aqt.ROUND_HALF_UP_FLOOR, True)
+
+
 def test_requant_many_tiles_per_cta():
     """More m-tiles than groups of CTAs: every TMEM buffer and both exchange slots are reused."""
     _run(12800, 2048, 512, 8, 4, aqt.ACT_SWISH, False, False, 8, aqt.ROUND_NEAREST_EVEN, False)
