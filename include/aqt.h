@@ -183,12 +183,14 @@ int aqt_qmatmul_with_plan(const char* plan, const void* xq, const float* s_x, in
  *           a parity check).  residual != NULL requires y != NULL.
  * workspace at least aqt_workspace_bytes(AQT_OP_QMATMUL_REQUANT, ...) bytes, 256-byte aligned:
  *           what aqt_qmatmul needs plus the area through which CTAs exchange row maxima.
- * Limits: those of aqt_qmatmul, and N_out % 16 == 0 (N_out % 32 == 0 if pack_out).  The fused
- * kernel takes K <= 512 with act NONE or SWISH, the GLU forms when only int8 codes and scales
- * are asked for (y == NULL, pack_out == 0), and 512 < K <= 1024 when y == NULL; it is launched cooperatively (its CTAs wait on one
- * another, with the same bounded waits as everything else) on at most one CTA per SM.
- * Other calls run the two steps one after the other through y and return
- * AQT_ERR_UNSUPPORTED if y is NULL.
+ * Limits: those of aqt_qmatmul, and N_out % 16 == 0 (N_out % 32 == 0 if pack_out).  One kernel
+ * does both steps for: K <= 512 with act NONE or SWISH; the GLU forms when only int8 codes and
+ * scales are asked for (y == NULL, pack_out == 0); 512 < K <= 1024 when y == NULL; and K >= 2048
+ * with act NONE or SWISH, M > 128, N <= 2048 and pack_out == 0 (with or without y).  The CTAs of
+ * such a kernel wait on one another (row maxima cross CTAs), with the same bounded waits as
+ * everything else, so it runs on at most one CTA per SM and reports AQT_ERR_TIMEOUT through the
+ * device status word if other work keeps SMs from it for seconds.  Other calls run the two
+ * steps one after the other through y and return AQT_ERR_UNSUPPORTED if y is NULL.
  */
 int aqt_qmatmul_requant(const void* xq, const float* s_x, int s_x_kind, const void* wq, const float* s_w,
                         const float* bias, const float* residual, int64_t ldr, float residual_scale, int64_t M,
