@@ -256,6 +256,43 @@ def test_qmatmul_small_batch(M, N, K, act, bits_a, bits_w):
     _run_qmatmul(M, N, K, bits_a, bits_w, act, False, False, s_x_kind=aqt.SCALE_TENSOR)
 
 
+@pytest.mark.parametrize("M", [1, 5, 16, 17, 33, 48, 64])
+@pytest.mark.parametrize("N,K,act,bits_a,bits_w,kind,rounding", [
+    (256, 256, aqt.ACT_NONE, 8, 8, aqt.SCALE_TENSOR, orc.ROUND_NEAREST_EVEN),
+    (2048, 512, aqt.ACT_NONE, 8, 4, aqt.SCALE_ROW, orc.ROUND_HALF_UP_FLOOR),
+    (144, 144, aqt.ACT_NONE, 4, 4, aqt.SCALE_ROW, orc.ROUND_NEAREST_EVEN),
+    (512, 1024, aqt.ACT_NONE, 4, 8, aqt.SCALE_TENSOR, orc.ROUND_HALF_UP_FLOOR),
+    (1024, 512, aqt.ACT_GLU_SWISH, 8, 4, aqt.SCALE_ROW, orc.ROUND_NEAREST_EVEN),
+    (576, 16, aqt.ACT_SWISH, 8, 8, aqt.SCALE_ROW, orc.ROUND_NEAREST_EVEN)])
+def test_linear_fwd_few_rows(M, N, K, act, bits_a, bits_w, kind, rounding):
+    """One to 64 rows of fp32 activations (a streaming step) through the whole layer, across the
+    threshold between the small-batch and the tensor-core matmul.  Outputs bit-exact without a
+    transcendental, within the float bar with one; a zero row and a row of tiny values ride along."""
+    x = gen.normal(60 + M, 1, M, K)
+    if M > 2:
+        x[1, :] = 0.0
+        x[2, :] *= 1e-30
+    wt = gen.weight(60 + M, 2, K, N)
+    bias = gen.normal(60 + M, 3, 1, N, std=0.01)[0]
+    n_out = N // 2 if act in (aqt.ACT_GLU, aqt.ACT_GLU_SWISH) else N
+    res = gen.normal(60 + M, 4, M, n_out)
+    wq, s_w = orc.quantize(wt, bits_w, orc.AXIS_ROW, rounding)
+    y_ref, xq, sx, acc = orc.linear_fwd(x, wq, s_w, bias=bias, residual=res, residual_scale=0.5, bits_a=bits_a, a_scale_kind=kind,
+                                        rounding=rounding, act=act, return_parts=True)
+    wq_d = _dev(orc.pack_int4(wq)) if bits_w == 4 else _dev(wq)
+    y = aqt.aqt_linear_fwd(_dev(x), wq_d, _dev(s_w), _dev(bias), _dev(res), 0.5, bits_a=bits_a, bits_w=bits_w, a_scale_kind=kind,
+                           rounding=rounding, act=act)
+    _status_ok()
+    y = y.cpu().numpy()
+    if act == aqt.ACT_NONE:
+        assert np.array_equal(y.view(np.uint32), y_ref.view(np.uint32))
+    else:
+        y64 = orc.epilogue_f64(acc, sx, kind, s_w, bias, res, 0.5, act)
+        z = np.abs(orc.epilogue_f64(acc, sx, kind, s_w, None, None, 0.0, aqt.ACT_NONE))
+        mag = np.maximum(np.maximum(np.abs(y64), z[:, :n_out]), np.maximum(np.abs(bias[:n_out])[None, :], np.abs(res)))
+        assert np.all(np.abs(y - y64) <= 1e-6 * mag + 1e-30)
+
+
 def test_linear_fwd_small_batch_matches_oracle():
     M, K, N = 5, 512, 2048
     x = gen.normal(6, 1, M, K)
