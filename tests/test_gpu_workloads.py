@@ -306,3 +306,32 @@ def test_weight_arena_quantizes_like_per_weight_calls_and_the_oracle():
         assert np.array_equal(lin.s_w.cpu().numpy(), s_ref.reshape(-1)), sp.name
         q_own, s_own = aqt.aqt_quantize(_dev(host[i]), sp.bits_w, aqt.AXIS_ROW, pack=(sp.bits_w == 4))
         assert torch.equal(q_own.view(torch.uint8), lin.wq.view(torch.uint8)) and torch.equal(s_own, lin.s_w)
+
+
+def test_encoder_graph_replays_give_the_same_bits():
+    """A captured stack replayed many times: the row maxima cross CTAs through tagged words whose
+    tag changes on every execution of a captured launch, so every replay must give the output of
+    the first run, bit for bit, and leave the device status clean."""
+    w = gen.WORKLOADS[4]
+    specs = gen.workload_layers(w)
+    M, n_blocks = 128 * 23 + 40, 3
+    g = torch.Generator(device=DEV).manual_seed(11)
+    blocks = [[QuantLinear.from_float(s, torch.randn((s.N, s.K), generator=g, device=DEV) * (s.K ** -0.5)) for s in specs]
+              for _ in range(n_blocks)]
+    stack = EncoderStack(M, w.d, w.ff, blocks, DEV)
+    x = torch.randn((M, w.d), generator=g, device=DEV)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        ref_out = stack.forward(x).clone()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        out = stack.forward(x)
+    for r in range(60):
+        graph.replay()
+        if r % 10 == 9:
+            torch.cuda.synchronize()
+            assert torch.equal(out.view(torch.int32), ref_out.view(torch.int32)), "replay %d" % r
+    torch.cuda.synchronize()
+    assert aqt.aqt_device_status() == 0 and bool(torch.isfinite(out).all())
