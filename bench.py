@@ -304,6 +304,17 @@ def run_ours(args):
         graph = _capture(run_plain, torch)
         for _ in range(2):
             graph.replay()
+        # the steps left over when --steps is not a multiple of R: a graph of their own, so that the
+        # whole timed region is replayed from graphs whatever the step count
+        rem = args.steps % R
+        graph_rem = None
+        if rem:
+            def run_rem(st):
+                for c3 in make_calls(st)[:rem]:
+                    for c in c3:
+                        c()
+            graph_rem = _capture(run_rem, torch)
+            graph_rem.replay()
         barrier()
 
     sampler = ClockSampler(local)
@@ -320,6 +331,9 @@ def run_ours(args):
             graph.replay()
             replays += 1
             i += R
+        if graph_rem is not None:
+            graph_rem.replay()
+            i += rem
     while i < args.steps:
         step(i); i += 1
     e_end.record(stream)
@@ -482,7 +496,7 @@ def run_ours(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 4 * M * s0.K, "d2h_bytes_per_step": 4 * M * s1_.N,
                     "ms_per_step": float(te.item()) / args.steps, "streams": n_lanes, "api": "aqt_ffn_fwd", "device_status": e2e_status},
             "gpu_launches": args.steps * NC, "sum_call_ms_per_step": sum(per_call_ms),
-            "launch_mode": ("cuda graph of %d steps x %d replays + %d call-by-call steps; per-call durations from one graph per call" %
+            "launch_mode": ("cuda graph of %d steps x %d replays + one graph of the %d steps left over; per-call durations from one graph per call" %
                             (R, replays, args.steps - replays * R))
             if graph is not None else "call by call",
             "roofline": roofline}
